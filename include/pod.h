@@ -1,0 +1,158 @@
+/*
+ * pod.h -- C ABI of the PoD decode-attention library (CUDA, sm_100a, one GPU).
+ *
+ * PoD ("Proximal tokens over Distant tokens") keeps the full per-layer K and V of the
+ * proximal tokens of a sequence -- the first n_s ("sink") and the last n_r ("recent")
+ * tokens -- and stores the keys of all other ("distant") tokens once per block of
+ * consecutive layers; values are kept per layer (paper: abstract; Section 2.2).  At a decode
+ * step, layer l scores proximal tokens with its own query and keys, takes the distant scores
+ * from the lowest layer l_a of its block (query and keys of l_a), and applies one softmax
+ * over both groups to its own values (Section 2.2, Eq. 1 and Eq. 2; Appendix C shows the
+ * gate of Eq. 2 is exactly that single softmax).
+ *
+ * Conventions
+ *   - All tensors are bf16, row-major, contiguous; pointers named "device" are CUDA device
+ *     pointers owned by the caller, 16-byte aligned, valid until the stream work finishes.
+ *   - Layers, sequences, heads and positions are 0-based.  Blocks are runs of group_size
+ *     consecutive layers: block(l) = l / group_size, lowest layer l - l % group_size; the
+ *     last block is short when group_size does not divide n_layers.
+ *   - A sequence holding n tokens at a layer has sink positions [0, min(n, n_s)), recent
+ *     positions [max(n_s, n - n_r), n) and distant positions [n_s, n - n_r).  The token being
+ *     decoded is the last one: append its K/V with pod_cache_write, then call
+ *     pod_decode_attn (Eq. 1 ranges end at n, the current token included).
+ *   - q and K arrive with rotary position encoding already applied; distant scores pair
+ *     the lowest layer's query with the lowest layer's keys, so no re-rotation is needed.
+ *   - Calls return an int status: POD_OK (0), POD_DRY_RUN (1, host-only cache), or a
+ *     negative POD_ERR_* code.  Nothing throws, nothing aborts.  After an error the cache is
+ *     unchanged unless stated otherwise.
+ *   - Work is enqueued on the CUDA stream passed by the caller (NULL = default stream) and
+ *     is asynchronous unless stated.  All calls on one cache must be issued on one stream
+ *     (or be ordered by the caller); the library keeps sequence lengths both on the host
+ *     (validation, launch sizing) and on the device (read by the kernels in stream order).
+ *   - A cache object is not thread-safe.
+ */
+#ifndef POD_H_
+#define POD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define POD_OK            0
+#define POD_DRY_RUN       1   /* host-only cache: arguments were valid, bookkeeping advanced, nothing launched */
+#define POD_ERR_INVALID  (-1) /* null/misaligned pointer, index out of range, unsupported shape */
+#define POD_ERR_CAPACITY (-2) /* write would exceed a sequence's capacity; nothing written */
+#define POD_ERR_ORDER    (-3) /* block lengths differ, or lowest layer not decoded at these lengths */
+#define POD_ERR_ARENA    (-4) /* caller's arena is too small or misaligned */
+#define POD_ERR_CUDA     (-5) /* a CUDA runtime call failed; see pod_cache_last_cuda_error */
+#define POD_ERR_DEVICE   (-6) /* a kernel's bounded wait gave up; results of that call are invalid */
+
+/* pod_cache_bytes selector */
+#define POD_BYTES_LIVE        0 /* bytes of valid rows in the PoD layout */
+#define POD_BYTES_DENSE_EQUIV 1 /* bytes a per-layer K+V cache of the same lengths would hold */
+#define POD_BYTES_ALLOCATED   2 /* bytes of the arena (regions at capacity + library scratch) */
+
+/* pod_cache_read_region selector (logical regions of one sequence) */
+#define POD_REGION_SINK_K 0 /* [layer][kv_head][n_s][d]            position j            */
+#define POD_REGION_SINK_V 1
+#define POD_REGION_RING_K 2 /* [layer][kv_head][n_r][d]            slot (p - n_s) % n_r  */
+#define POD_REGION_RING_V 3
+#define POD_REGION_DIST_K 4 /* [block][kv_head][capacity-n_s-n_r][d] index p - n_s, key of the block's lowest layer */
+#define POD_REGION_DIST_V 5 /* [layer][kv_head][capacity-n_s-n_r][d] index p - n_s       */
+
+typedef struct pod_cache pod_cache; /* opaque: host bookkeeping + device arena */
+
+typedef struct {
+  int32_t n_layers;    /* L >= 1 */
+  int32_t n_q_heads;   /* H_q; H_q / H_kv must be 1, 2, 4 or 8 (grouped-query attention) */
+  int32_t n_kv_heads;  /* H_kv */
+  int32_t head_dim;    /* d: 64 or 128 */
+  int32_t group_size;  /* G >= 1 layers per block (G = 1: ordinary dense attention) */
+  int32_t n_sink;      /* n_s >= 0 */
+  int32_t n_recent;    /* n_r >= 1 */
+  int32_t batch;       /* number of sequences B >= 1 */
+  float   sm_scale;    /* logit scale; 0 means 1/sqrt(d) as in Eq. 1 */
+  int32_t device;      /* CUDA device ordinal; -1 = host-only cache (no CUDA call is made) */
+} pod_config;
+
+/* Bytes of device memory a cache with these per-sequence capacities (tokens, [batch]) needs:
+ * the regions of every sequence at capacity plus library scratch (device lengths, the
+ * per-block query stash, split-K partials).  Returns 0 on invalid arguments.  Host only. */
+size_t pod_cache_required_bytes(const pod_config* cfg, const int32_t* seq_capacity);
+
+/* Creates a cache.  arena: device memory of at least pod_cache_required_bytes, 256-byte
+ * aligned, owned by the caller and kept alive until pod_cache_destroy; or NULL to let the
+ * library allocate (and later free) it with cudaMalloc.  Region contents start undefined,
+ * lengths start at 0.  Synchronous.  The physical layout inside the arena is private; its
+ * logical content is what pod_cache_read_region returns.  Every region starts on a
+ * multiple of 128 bytes.  Errors: INVALID, ARENA, CUDA. */
+int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity,
+                     void* arena_device, size_t arena_bytes, pod_cache** out);
+
+/* Frees host state (and the arena if the library allocated it).  Synchronises the device. */
+int pod_cache_destroy(pod_cache* c);
+
+/* Appends n_tokens tokens to one layer of the cache (prefill, chunked prefill or decode
+ * append), scattering them into the PoD layout and moving rows that leave the recent window
+ * to the distant stores: values always, keys only when `layer` is the lowest layer of its
+ * block, so distant keys are written once per block (reading of the paper's cache-update
+ * figure, Fig. 2 right: a token is demoted when it falls out of the last n_r tokens).
+ *   seq >= 0 : k, v are device bf16 [n_tokens][H_kv][d] for that sequence.
+ *   seq == -1: n_tokens must be 1; k, v are device bf16 [B][H_kv][d], one token for every
+ *              sequence.
+ * Errors: INVALID, CAPACITY (length + n_tokens > capacity of a sequence; nothing written),
+ * CUDA. */
+int pod_cache_write(pod_cache* c, int layer, int seq, const void* k_device,
+                    const void* v_device, int n_tokens, void* cuda_stream);
+
+/* Decode-step attention of one layer for every sequence (Eq. 1 + Eq. 2 / Appendix C):
+ *   logits of proximal tokens  = sm_scale * <q[b][h], K_layer[p][h / r]>
+ *   logits of distant tokens   = sm_scale * <q_low[b][h], K_low[p][h / r]>, q_low being the q
+ *                                passed to this function for the block's lowest layer at the
+ *                                same step (the library stashes it), K_low the block's key store
+ *   out[b][h] = softmax over all logits applied to V_layer, fp32 accumulation, bf16 result.
+ * q_device, out_device: device bf16 [B][H_q][d].  A sequence of length 0 gives zeros.
+ * Call order inside a decode step: layers in increasing order within a block, lowest first;
+ * all layers of a block must hold the same lengths.  Errors: INVALID, ORDER, CUDA. */
+int pod_decode_attn(pod_cache* c, int layer, const void* q_device, void* out_device,
+                    void* cuda_stream);
+
+/* Byte accounting (host integers).  Live bytes of a sequence of length n (at the layer with
+ * the most tokens): row * H_kv * (L * (2 n_p + n_d) + ceil(L / G) * n_d), n_p = min(n, n_s+n_r),
+ * n_d = n - n_p; the saving against dense is (n_d / n) (1 - ceil(L/G)/L) / 2 -- only keys
+ * are shared (Section 2.2; Section 3 "KV Cache Memory").  Returns -1 on error. */
+int64_t pod_cache_bytes(const pod_cache* c, int which);
+
+/* Tokens currently held by (seq, layer); negative status on error.  Host only. */
+int pod_cache_seq_len(const pod_cache* c, int seq, int layer);
+
+/* Forgets the contents of one sequence (seq >= 0) or of all (seq == -1).  Synchronous. */
+int pod_cache_reset(pod_cache* c, int seq);
+
+/* Test/debug export: copies `count` rows (d bf16 each) starting at row `first` of a logical
+ * region to host memory.  Synchronises the device.  Only rows that hold a token are
+ * meaningful.  layer_or_block is a block index for POD_REGION_DIST_K, a layer otherwise. */
+int pod_cache_read_region(const pod_cache* c, int region, int layer_or_block, int seq,
+                          int kv_head, int first, int count, void* host_dst);
+
+/* Synchronises the device and reports POD_ERR_DEVICE if any kernel of this cache hit a
+ * bounded-wait limit since the last call (the flag is cleared), else POD_OK. */
+int pod_cache_device_status(pod_cache* c);
+
+/* Last CUDA runtime error code seen by this cache (0 if none). */
+int pod_cache_last_cuda_error(const pod_cache* c);
+
+/* Launch geometry of the most recent pod_decode_attn (diagnostics for benchmarks):
+ * tokens per split, CTAs launched, and kernels launched by that call. */
+int pod_cache_last_launch(const pod_cache* c, int32_t* split_tokens, int32_t* n_ctas,
+                          int32_t* n_kernels);
+
+const char* pod_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POD_H_ */

@@ -1,0 +1,163 @@
+"""Thin ctypes binding of the C ABI declared in ``include/pod.h``.
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+Tensors are passed as raw device pointers (``tensor.data_ptr()``); PyTorch supplies device
+memory and streams, nothing else.  There is no fallback: if the shared library is missing
+and cannot be built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_void_p
+
+from . import build as _build
+
+POD_OK, POD_DRY_RUN = 0, 1
+POD_ERR_INVALID, POD_ERR_CAPACITY, POD_ERR_ORDER = -1, -2, -3
+POD_ERR_ARENA, POD_ERR_CUDA, POD_ERR_DEVICE = -4, -5, -6
+POD_BYTES_LIVE, POD_BYTES_DENSE_EQUIV, POD_BYTES_ALLOCATED = 0, 1, 2
+(POD_REGION_SINK_K, POD_REGION_SINK_V, POD_REGION_RING_K, POD_REGION_RING_V,
+ POD_REGION_DIST_K, POD_REGION_DIST_V) = range(6)
+
+
+class pod_config(ctypes.Structure):
+    _fields_ = [("n_layers", c_int32), ("n_q_heads", c_int32), ("n_kv_heads", c_int32),
+                ("head_dim", c_int32), ("group_size", c_int32), ("n_sink", c_int32),
+                ("n_recent", c_int32), ("batch", c_int32), ("sm_scale", c_float),
+                ("device", c_int32)]
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path) or _build.needs_build():
+        try:
+            path = _build.build()
+        except Exception as e:  # no nvcc where the library is missing: fail loudly
+            if not os.path.exists(path):
+                raise ImportError(f"libpod_b200.so is missing and could not be built: {e}") from e
+    lib = ctypes.CDLL(path)
+    P = POINTER
+    sig = {
+        "pod_cache_required_bytes": (c_size_t, [P(pod_config), P(c_int32)]),
+        "pod_cache_create": (c_int, [P(pod_config), P(c_int32), c_void_p, c_size_t, P(c_void_p)]),
+        "pod_cache_destroy": (c_int, [c_void_p]),
+        "pod_cache_write": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_void_p]),
+        "pod_decode_attn": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
+        "pod_cache_bytes": (c_int64, [c_void_p, c_int]),
+        "pod_cache_seq_len": (c_int, [c_void_p, c_int, c_int]),
+        "pod_cache_reset": (c_int, [c_void_p, c_int]),
+        "pod_cache_read_region": (c_int, [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int, c_void_p]),
+        "pod_cache_device_status": (c_int, [c_void_p]),
+        "pod_cache_last_cuda_error": (c_int, [c_void_p]),
+        "pod_cache_last_launch": (c_int, [c_void_p, P(c_int32), P(c_int32), P(c_int32)]),
+        "pod_strerror": (c_char_p, [c_int]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    return lib
+
+
+lib = _load()
+EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_destroy", "pod_cache_write",
+           "pod_decode_attn", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
+           "pod_cache_read_region", "pod_cache_device_status", "pod_cache_last_cuda_error",
+           "pod_cache_last_launch", "pod_strerror"]
+
+
+class PodError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {pod_strerror(status)} ({status})")
+
+
+def pod_strerror(status: int) -> str:
+    return lib.pod_strerror(status).decode()
+
+
+def _check(status: int, where: str) -> int:
+    if status < 0:
+        raise PodError(status, where)
+    return status
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else (t if isinstance(t, int) else t.data_ptr())
+
+
+def make_config(*, n_layers, n_q_heads, n_kv_heads, head_dim, group_size, n_sink, n_recent, batch,
+                sm_scale=0.0, device=0) -> pod_config:
+    return pod_config(n_layers, n_q_heads, n_kv_heads, head_dim, group_size, n_sink, n_recent,
+                      batch, sm_scale, device)
+
+
+def _caps(cfg: pod_config, seq_capacity):
+    caps = list(seq_capacity)
+    if len(caps) != cfg.batch:
+        raise ValueError("one capacity per sequence")
+    return (c_int32 * cfg.batch)(*caps)
+
+
+def pod_cache_required_bytes(cfg: pod_config, seq_capacity) -> int:
+    return lib.pod_cache_required_bytes(ctypes.byref(cfg), _caps(cfg, seq_capacity))
+
+
+class PodCache:
+    """Owner of one ``pod_cache*``; methods carry the C names without the prefix."""
+
+    def __init__(self, cfg: pod_config, seq_capacity, arena=None):
+        self.cfg = cfg
+        self._arena = arena                       # keeps the caller's tensor alive
+        handle = c_void_p()
+        nbytes = 0 if arena is None else arena.numel() * arena.element_size()
+        st = lib.pod_cache_create(ctypes.byref(cfg), _caps(cfg, seq_capacity), _ptr(arena), nbytes,
+                                  ctypes.byref(handle))
+        _check(st, "pod_cache_create")
+        self._h = handle
+
+    def destroy(self):
+        if self._h is not None:
+            h, self._h = self._h, None
+            _check(lib.pod_cache_destroy(h), "pod_cache_destroy")
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def write(self, layer: int, seq: int, k, v, n_tokens: int, stream: int = 0) -> int:
+        return _check(lib.pod_cache_write(self._h, layer, seq, _ptr(k), _ptr(v), n_tokens, stream),
+                      "pod_cache_write")
+
+    def decode_attn(self, layer: int, q, out, stream: int = 0) -> int:
+        return _check(lib.pod_decode_attn(self._h, layer, _ptr(q), _ptr(out), stream), "pod_decode_attn")
+
+    def bytes(self, which: int) -> int:
+        return lib.pod_cache_bytes(self._h, which)
+
+    def seq_len(self, seq: int, layer: int) -> int:
+        return _check(lib.pod_cache_seq_len(self._h, seq, layer), "pod_cache_seq_len")
+
+    def reset(self, seq: int = -1) -> int:
+        return _check(lib.pod_cache_reset(self._h, seq), "pod_cache_reset")
+
+    def read_region(self, region: int, layer_or_block: int, seq: int, kv_head: int, first: int, count: int):
+        """Returns a numpy uint16 array [count][head_dim] of bf16 bit patterns."""
+        import numpy as np
+        dst = np.empty((count, self.cfg.head_dim), dtype=np.uint16)
+        _check(lib.pod_cache_read_region(self._h, region, layer_or_block, seq, kv_head, first, count,
+                                         dst.ctypes.data), "pod_cache_read_region")
+        return dst
+
+    def device_status(self) -> int:
+        return lib.pod_cache_device_status(self._h)
+
+    def last_cuda_error(self) -> int:
+        return lib.pod_cache_last_cuda_error(self._h)
+
+    def last_launch(self):
+        a, b, c = c_int32(), c_int32(), c_int32()
+        lib.pod_cache_last_launch(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+        return {"split_tokens": a.value, "n_ctas": b.value, "n_kernels": c.value}

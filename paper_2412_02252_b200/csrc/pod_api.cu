@@ -1,0 +1,399 @@
+// Host side of the PoD library: the C ABI of include/pod.h, argument validation, arena
+// carving, length bookkeeping, split planning and kernel launches.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/pod.h"
+#include "pod_common.h"
+
+using namespace pod;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+constexpr int MAX_SPLITS_CAP = 128;
+constexpr int TARGET_CTAS_FOR_SPLITS = 148 * 2 * 4;   // used only to size the partial buffers
+constexpr int SPLIT_OVERHEAD_TOKENS = 48;             // fixed cost of a CTA in the planner's model
+
+size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+bool config_ok(const pod_config* c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1 || c->batch < 1) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->n_q_heads % c->n_kv_heads != 0) return false;
+  if (c->n_q_heads / c->n_kv_heads > 8) return false;
+  if (c->group_size < 1 || c->n_sink < 0 || c->n_recent < 1) return false;
+  if (c->n_kv_heads > 65535 || c->batch > 65535) return false;
+  if (!(c->sm_scale >= 0.f) || isinf(c->sm_scale)) return false;
+  return true;
+}
+
+int max_splits_for(const pod_config& c) {
+  int per = (TARGET_CTAS_FOR_SPLITS + c.batch * c.n_kv_heads - 1) / (c.batch * c.n_kv_heads);
+  if (per < 16) per = 16;
+  if (per > MAX_SPLITS_CAP) per = MAX_SPLITS_CAP;
+  return per;
+}
+
+struct Carve {
+  std::vector<int64_t> seq_row_base;   // rows
+  std::vector<int32_t> seq_cap_d;
+  size_t off_len, off_rowbase, off_capd, off_stash, off_pacc, off_pml, off_err, total;
+  int n_blocks, max_splits;
+};
+
+bool carve(const pod_config& c, const int32_t* cap, Carve* out) {
+  const int64_t row_bytes = (int64_t)c.head_dim * 2;
+  const int n_blocks = (c.n_layers + c.group_size - 1) / c.group_size;
+  out->n_blocks = n_blocks;
+  out->max_splits = max_splits_for(c);
+  out->seq_row_base.resize(c.batch);
+  out->seq_cap_d.resize(c.batch);
+  int64_t rows = 0;
+  const int64_t SW = (int64_t)c.n_sink + c.n_recent;
+  for (int b = 0; b < c.batch; ++b) {
+    if (cap[b] < 1) return false;
+    const int64_t cap_d = cap[b] > SW ? cap[b] - SW : 0;
+    out->seq_row_base[b] = rows;
+    out->seq_cap_d[b] = (int32_t)cap_d;
+    rows += (int64_t)c.n_layers * 2 * c.n_kv_heads * SW + ((int64_t)c.n_layers + n_blocks) * c.n_kv_heads * cap_d;
+  }
+  size_t off = align_up((size_t)(rows * row_bytes));
+  out->off_len = off;      off = align_up(off + (size_t)c.n_layers * c.batch * 4);
+  out->off_rowbase = off;  off = align_up(off + (size_t)c.batch * 8);
+  out->off_capd = off;     off = align_up(off + (size_t)c.batch * 4);
+  out->off_stash = off;    off = align_up(off + (size_t)n_blocks * c.batch * c.n_q_heads * row_bytes);
+  out->off_pacc = off;     off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * c.head_dim * 4);
+  out->off_pml = off;      off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * 2 * 4);
+  out->off_err = off;      off = align_up(off + 4);
+  out->total = off;
+  return true;
+}
+
+}  // namespace
+
+struct pod_cache {
+  pod_config cfg;
+  std::vector<int32_t> cap;            // [B]
+  std::vector<int32_t> len;            // host mirror [L][B]
+  std::vector<int32_t> stash_len;      // [n_blocks][B]: lengths at which the block's q was stashed, -1 = none
+  Carve cv;
+  unsigned char* arena = nullptr;
+  bool owns_arena = false;
+  bool dry = false;
+  int last_cuda = 0;
+  int sm_count = 148, resident = 2;
+  float scale = 0.f;
+  Layout y{};
+  // last launch (diagnostics)
+  int32_t last_split_tokens = 0, last_ctas = 0, last_kernels = 0;
+  // planner memo
+  int64_t memo_sum = -1; int32_t memo_max = -1; DecodePlan memo_plan{};
+
+  int32_t* d_len(int layer) const { return reinterpret_cast<int32_t*>(arena + cv.off_len) + (size_t)layer * cfg.batch; }
+  int32_t& h_len(int layer, int b) { return len[(size_t)layer * cfg.batch + b]; }
+  int32_t h_len(int layer, int b) const { return len[(size_t)layer * cfg.batch + b]; }
+};
+
+namespace {
+
+int cuda_fail(pod_cache* c, cudaError_t e) {
+  c->last_cuda = (int)e;
+  return POD_ERR_CUDA;
+}
+
+// Picks the tokens-per-split that minimises a simple time model: the CTAs run in waves of
+// (SMs x resident CTAs), every CTA costs its tokens plus a fixed overhead.
+DecodePlan plan_decode(pod_cache* c, int layer) {
+  const pod_config& g = c->cfg;
+  int64_t sum = 0; int32_t nmax = 0;
+  for (int b = 0; b < g.batch; ++b) { const int32_t n = c->h_len(layer, b); sum += n; if (n > nmax) nmax = n; }
+  if (sum == c->memo_sum && nmax == c->memo_max) return c->memo_plan;
+  DecodePlan best{1, 1, 0};
+  if (nmax > 0) {
+    const int64_t slots = (int64_t)c->sm_count * c->resident;
+    double best_cost = 1e300;
+    int last_st = -1;
+    for (int k = 1; k <= c->cv.max_splits; ++k) {
+      const int st = (nmax + k - 1) / k;
+      if (st == last_st) continue;
+      last_st = st;
+      int64_t ctas = 0;
+      for (int b = 0; b < g.batch; ++b) ctas += ((int64_t)c->h_len(layer, b) + st - 1) / st;
+      ctas *= g.n_kv_heads;
+      const int64_t waves = (ctas + slots - 1) / slots;
+      const double cost = (double)waves * (st + SPLIT_OVERHEAD_TOKENS);
+      if (cost < best_cost * 0.999) { best_cost = cost; best = DecodePlan{st, (nmax + st - 1) / st, (int32_t)ctas}; }
+      if (st <= 64) break;
+    }
+  }
+  c->memo_sum = sum; c->memo_max = nmax; c->memo_plan = best;
+  return best;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pod_strerror(int status) {
+  switch (status) {
+    case POD_OK: return "ok";
+    case POD_DRY_RUN: return "host-only cache: validated, nothing launched";
+    case POD_ERR_INVALID: return "invalid argument";
+    case POD_ERR_CAPACITY: return "sequence capacity exceeded";
+    case POD_ERR_ORDER: return "decode order violated: block lengths differ or lowest layer not decoded";
+    case POD_ERR_ARENA: return "arena too small or misaligned";
+    case POD_ERR_CUDA: return "CUDA runtime error";
+    case POD_ERR_DEVICE: return "a kernel gave up a bounded wait";
+    default: return "unknown status";
+  }
+}
+
+size_t pod_cache_required_bytes(const pod_config* cfg, const int32_t* seq_capacity) {
+  if (!config_ok(cfg) || !seq_capacity) return 0;
+  Carve cv;
+  if (!carve(*cfg, seq_capacity, &cv)) return 0;
+  return cv.total;
+}
+
+int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* arena_device,
+                     size_t arena_bytes, pod_cache** out) {
+  if (!out) return POD_ERR_INVALID;
+  *out = nullptr;
+  if (!config_ok(cfg) || !seq_capacity) return POD_ERR_INVALID;
+  pod_cache* c = new (std::nothrow) pod_cache();
+  if (!c) return POD_ERR_INVALID;
+  c->cfg = *cfg;
+  if (!carve(*cfg, seq_capacity, &c->cv)) { delete c; return POD_ERR_INVALID; }
+  c->cap.assign(seq_capacity, seq_capacity + cfg->batch);
+  c->len.assign((size_t)cfg->n_layers * cfg->batch, 0);
+  c->stash_len.assign((size_t)c->cv.n_blocks * cfg->batch, -1);
+  c->scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)cfg->head_dim);
+  c->dry = cfg->device < 0;
+  Layout& y = c->y;
+  y.L = cfg->n_layers; y.H_kv = cfg->n_kv_heads; y.H_q = cfg->n_q_heads; y.D = cfg->head_dim;
+  y.G = cfg->group_size; y.S = cfg->n_sink; y.W = cfg->n_recent; y.B = cfg->batch;
+  y.n_blocks = c->cv.n_blocks;
+  if (c->dry) { *out = c; return POD_OK; }
+
+  cudaError_t e = cudaSetDevice(cfg->device);
+  if (e != cudaSuccess) { delete c; return POD_ERR_CUDA; }
+  if (arena_device) {
+    if (((uintptr_t)arena_device % ALIGN) != 0 || arena_bytes < c->cv.total) { delete c; return POD_ERR_ARENA; }
+    c->arena = static_cast<unsigned char*>(arena_device);
+  } else {
+    void* pmem = nullptr;
+    e = cudaMalloc(&pmem, c->cv.total);
+    if (e != cudaSuccess) { delete c; return POD_ERR_CUDA; }
+    c->arena = static_cast<unsigned char*>(pmem);
+    c->owns_arena = true;
+  }
+  y.seq_row_base = reinterpret_cast<const int64_t*>(c->arena + c->cv.off_rowbase);
+  y.seq_cap_d = reinterpret_cast<const int32_t*>(c->arena + c->cv.off_capd);
+  bool ok = true;
+  ok = ok && cudaMemset(c->arena + c->cv.off_len, 0, c->cv.total - c->cv.off_len) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->arena + c->cv.off_rowbase, c->cv.seq_row_base.data(), (size_t)cfg->batch * 8, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->arena + c->cv.off_capd, c->cv.seq_cap_d.data(), (size_t)cfg->batch * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  int sm = 0;
+  ok = ok && cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess;
+  const int res = ok ? decode_resident_ctas_per_sm(cfg->head_dim, cfg->n_q_heads / cfg->n_kv_heads) : 0;
+  ok = ok && res > 0 && cudaDeviceSynchronize() == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    if (c->owns_arena) cudaFree(c->arena);
+    delete c;
+    return POD_ERR_CUDA;
+  }
+  c->sm_count = sm; c->resident = res;
+  *out = c;
+  return POD_OK;
+}
+
+int pod_cache_destroy(pod_cache* c) {
+  if (!c) return POD_ERR_INVALID;
+  int st = POD_OK;
+  if (!c->dry) {
+    cudaSetDevice(c->cfg.device);
+    if (cudaDeviceSynchronize() != cudaSuccess) st = POD_ERR_CUDA;
+    if (c->owns_arena && cudaFree(c->arena) != cudaSuccess) st = POD_ERR_CUDA;
+  }
+  delete c;
+  return st;
+}
+
+int pod_cache_write(pod_cache* c, int layer, int seq, const void* k, const void* v, int n_tokens,
+                    void* stream) {
+  if (!c || !k || !v) return POD_ERR_INVALID;
+  const pod_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers || seq < -1 || seq >= g.batch || n_tokens < 1) return POD_ERR_INVALID;
+  if (seq == -1 && n_tokens != 1) return POD_ERR_INVALID;
+  if (((uintptr_t)k % 16) != 0 || ((uintptr_t)v % 16) != 0) return POD_ERR_INVALID;
+  const int b0 = seq < 0 ? 0 : seq, b1 = seq < 0 ? g.batch : seq + 1;
+  for (int b = b0; b < b1; ++b)
+    if ((int64_t)c->h_len(layer, b) + n_tokens > c->cap[b]) return POD_ERR_CAPACITY;
+  if (!c->dry) {
+    WriteParams p;
+    p.y = c->y;
+    p.arena = reinterpret_cast<uint16_t*>(c->arena);
+    p.k = static_cast<const uint16_t*>(k);
+    p.v = static_cast<const uint16_t*>(v);
+    p.len = c->d_len(layer);
+    p.layer = layer; p.seq = seq; p.n0 = seq < 0 ? 0 : c->h_len(layer, seq); p.T = n_tokens;
+    const int e = launch_write(p, static_cast<cudaStream_t>(stream));
+    if (e != 0) return cuda_fail(c, (cudaError_t)e);
+  }
+  for (int b = b0; b < b1; ++b) c->h_len(layer, b) += n_tokens;
+  c->memo_sum = -1;
+  return c->dry ? POD_DRY_RUN : POD_OK;
+}
+
+int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* stream) {
+  if (!c || !q || !out) return POD_ERR_INVALID;
+  const pod_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return POD_ERR_INVALID;
+  if (((uintptr_t)q % 16) != 0 || ((uintptr_t)out % 16) != 0) return POD_ERR_INVALID;
+  const int low = layer - layer % g.group_size, block = layer / g.group_size;
+  const bool lowest = (low == layer);
+  int32_t* sl = &c->stash_len[(size_t)block * g.batch];
+  if (!lowest) {
+    for (int b = 0; b < g.batch; ++b) {
+      const int32_t n = c->h_len(layer, b);
+      if (n != c->h_len(low, b)) return POD_ERR_ORDER;       // block must hold equal lengths
+      if (n > 0 && sl[b] != n) return POD_ERR_ORDER;         // lowest layer's q not stashed at this step
+    }
+  }
+  if (c->dry) {
+    if (lowest) for (int b = 0; b < g.batch; ++b) sl[b] = c->h_len(layer, b);
+    return POD_DRY_RUN;
+  }
+  const DecodePlan plan = plan_decode(c, layer);
+  DecodeParams p;
+  p.y = c->y;
+  p.arena = reinterpret_cast<const uint16_t*>(c->arena);
+  p.len = c->d_len(layer);
+  p.q = static_cast<const uint16_t*>(q);
+  uint16_t* stash = reinterpret_cast<uint16_t*>(c->arena + c->cv.off_stash) + (size_t)block * g.batch * g.n_q_heads * g.head_dim;
+  p.q_low = lowest ? p.q : stash;
+  p.stash = (lowest && g.group_size > 1) ? stash : nullptr;
+  p.part_acc = reinterpret_cast<float*>(c->arena + c->cv.off_pacc);
+  p.part_ml = reinterpret_cast<float*>(c->arena + c->cv.off_pml);
+  p.out = static_cast<uint16_t*>(out);
+  p.err_flag = reinterpret_cast<int32_t*>(c->arena + c->cv.off_err);
+  p.layer = layer; p.block = block;
+  p.split_tokens = plan.split_tokens; p.max_splits = c->cv.max_splits;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int kernels = 0;
+  if (plan.n_ctas > 0) {
+    const int e = launch_decode(p, plan.grid_splits, s);
+    if (e != 0) return cuda_fail(c, (cudaError_t)e);
+    ++kernels;
+  }
+  const int e2 = launch_combine(p, s);
+  if (e2 != 0) return cuda_fail(c, (cudaError_t)e2);
+  ++kernels;
+  if (lowest) for (int b = 0; b < g.batch; ++b) sl[b] = c->h_len(layer, b);
+  c->last_split_tokens = plan.split_tokens; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;
+  return POD_OK;
+}
+
+int64_t pod_cache_bytes(const pod_cache* c, int which) {
+  if (!c) return -1;
+  const pod_config& g = c->cfg;
+  const int64_t row = (int64_t)g.head_dim * 2;
+  if (which == POD_BYTES_ALLOCATED) return (int64_t)c->cv.total;
+  if (which != POD_BYTES_LIVE && which != POD_BYTES_DENSE_EQUIV) return -1;
+  const int64_t SW = (int64_t)g.n_sink + g.n_recent;
+  int64_t total = 0;
+  for (int b = 0; b < g.batch; ++b) {
+    // count what each layer and each block store actually holds
+    for (int l = 0; l < g.n_layers; ++l) {
+      const int64_t n = c->h_len(l, b);
+      const int64_t n_p = n < SW ? n : SW, n_d = n - n_p;
+      if (which == POD_BYTES_DENSE_EQUIV) { total += g.n_kv_heads * row * 2 * n; continue; }
+      total += g.n_kv_heads * row * (2 * n_p + n_d);
+      if (l % g.group_size == 0) total += g.n_kv_heads * row * n_d;
+    }
+  }
+  return total;
+}
+
+int pod_cache_seq_len(const pod_cache* c, int seq, int layer) {
+  if (!c || seq < 0 || seq >= c->cfg.batch || layer < 0 || layer >= c->cfg.n_layers) return POD_ERR_INVALID;
+  return c->h_len(layer, seq);
+}
+
+int pod_cache_reset(pod_cache* c, int seq) {
+  if (!c || seq < -1 || seq >= c->cfg.batch) return POD_ERR_INVALID;
+  const pod_config& g = c->cfg;
+  const int b0 = seq < 0 ? 0 : seq, b1 = seq < 0 ? g.batch : seq + 1;
+  for (int l = 0; l < g.n_layers; ++l)
+    for (int b = b0; b < b1; ++b) c->h_len(l, b) = 0;
+  for (int blk = 0; blk < c->cv.n_blocks; ++blk)
+    for (int b = b0; b < b1; ++b) c->stash_len[(size_t)blk * g.batch + b] = -1;
+  c->memo_sum = -1;
+  if (c->dry) return POD_DRY_RUN;
+  cudaError_t e = cudaSetDevice(g.device);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e == cudaSuccess)
+    e = cudaMemcpy(c->arena + c->cv.off_len, c->len.data(), c->len.size() * 4, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  return POD_OK;
+}
+
+int pod_cache_read_region(const pod_cache* c, int region, int layer_or_block, int seq, int kv_head,
+                          int first, int count, void* host_dst) {
+  if (!c || !host_dst || c->dry) return POD_ERR_INVALID;
+  const pod_config& g = c->cfg;
+  if (seq < 0 || seq >= g.batch || kv_head < 0 || kv_head >= g.n_kv_heads || first < 0 || count < 0) return POD_ERR_INVALID;
+  const bool is_block = (region == POD_REGION_DIST_K);
+  if (layer_or_block < 0 || layer_or_block >= (is_block ? c->cv.n_blocks : g.n_layers)) return POD_ERR_INVALID;
+  const int64_t cap_d = c->cv.seq_cap_d[seq];
+  int64_t row, extent;
+  switch (region) {
+    case POD_REGION_SINK_K: row = prox_row(c->y, layer_or_block, 0, kv_head); extent = g.n_sink; break;
+    case POD_REGION_SINK_V: row = prox_row(c->y, layer_or_block, 1, kv_head); extent = g.n_sink; break;
+    case POD_REGION_RING_K: row = prox_row(c->y, layer_or_block, 0, kv_head) + g.n_sink; extent = g.n_recent; break;
+    case POD_REGION_RING_V: row = prox_row(c->y, layer_or_block, 1, kv_head) + g.n_sink; extent = g.n_recent; break;
+    case POD_REGION_DIST_K: row = distk_row(c->y, layer_or_block, kv_head, cap_d); extent = cap_d; break;
+    case POD_REGION_DIST_V: row = distv_row(c->y, layer_or_block, kv_head, cap_d); extent = cap_d; break;
+    default: return POD_ERR_INVALID;
+  }
+  if ((int64_t)first + count > extent) return POD_ERR_INVALID;
+  if (count == 0) return POD_OK;
+  const size_t row_bytes = (size_t)g.head_dim * 2;
+  const unsigned char* src = c->arena + (size_t)(c->cv.seq_row_base[seq] + row + first) * row_bytes;
+  cudaError_t e = cudaSetDevice(g.device);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(host_dst, src, (size_t)count * row_bytes, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) { const_cast<pod_cache*>(c)->last_cuda = (int)e; return POD_ERR_CUDA; }
+  return POD_OK;
+}
+
+int pod_cache_device_status(pod_cache* c) {
+  if (!c) return POD_ERR_INVALID;
+  if (c->dry) return POD_DRY_RUN;
+  int32_t flag = 0;
+  cudaError_t e = cudaSetDevice(c->cfg.device);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(&flag, c->arena + c->cv.off_err, 4, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess && flag != 0) e = cudaMemset(c->arena + c->cv.off_err, 0, 4);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  return flag ? POD_ERR_DEVICE : POD_OK;
+}
+
+int pod_cache_last_cuda_error(const pod_cache* c) { return c ? c->last_cuda : (int)cudaErrorInvalidValue; }
+
+int pod_cache_last_launch(const pod_cache* c, int32_t* split_tokens, int32_t* n_ctas, int32_t* n_kernels) {
+  if (!c) return POD_ERR_INVALID;
+  if (split_tokens) *split_tokens = c->last_split_tokens;
+  if (n_ctas) *n_ctas = c->last_ctas;
+  if (n_kernels) *n_kernels = c->last_kernels;
+  return POD_OK;
+}
+
+}  // extern "C"

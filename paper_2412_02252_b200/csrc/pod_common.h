@@ -1,0 +1,75 @@
+// Shared declarations of the PoD library's translation units (host API, write kernel,
+// decode kernels).  Private to the library; the public surface is include/pod.h.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace pod {
+
+// Physical layout of the arena.  All offsets are in rows; one row is one head's d bf16
+// values (128 B at d = 64, 256 B at d = 128), so every region base is 128-byte aligned.
+//
+// Sequence b owns a contiguous block starting at row seq_row_base[b]:
+//   prox  [L][2 (K, V)][H_kv][n_s + n_r]     rows [0, n_s) = sink, row n_s + slot = ring slot
+//   distV [L][H_kv][cap_d[b]]                 index p - n_s
+//   distK [n_blocks][H_kv][cap_d[b]]          index p - n_s, key of the block's lowest layer
+// with cap_d[b] = max(0, capacity[b] - n_s - n_r).  Sink and ring of one (layer, head) are
+// adjacent so that the proximal tokens of a head are one contiguous stream (the softmax does
+// not care about token order, so ring slots are read in slot order).
+struct Layout {
+  int32_t L, H_kv, H_q, D, G, S, W, B, n_blocks;
+  const int64_t* seq_row_base;  // device [B]
+  const int32_t* seq_cap_d;     // device [B]
+};
+
+__host__ __device__ inline int64_t prox_row(const Layout& y, int layer, int kv /*0=K,1=V*/, int head) {
+  return (((int64_t)layer * 2 + kv) * y.H_kv + head) * (int64_t)(y.S + y.W);
+}
+__host__ __device__ inline int64_t dist_base_row(const Layout& y) {
+  return (int64_t)y.L * 2 * y.H_kv * (int64_t)(y.S + y.W);
+}
+__host__ __device__ inline int64_t distv_row(const Layout& y, int layer, int head, int64_t cap_d) {
+  return dist_base_row(y) + ((int64_t)layer * y.H_kv + head) * cap_d;
+}
+__host__ __device__ inline int64_t distk_row(const Layout& y, int block, int head, int64_t cap_d) {
+  return dist_base_row(y) + (((int64_t)y.L + block) * y.H_kv + head) * cap_d;
+}
+
+struct WriteParams {
+  Layout y;
+  uint16_t* arena;       // bf16 bit patterns
+  const uint16_t* k;     // [T][H_kv][D] (seq >= 0) or [B][H_kv][D] (seq == -1)
+  const uint16_t* v;
+  int32_t* len;          // device lengths of this layer, [B]
+  int32_t layer, seq, n0, T;
+};
+
+struct DecodeParams {
+  Layout y;
+  const uint16_t* arena;
+  const int32_t* len;      // device lengths of this layer, [B]
+  const uint16_t* q;       // [B][H_q][D] queries of this layer
+  const uint16_t* q_low;   // [B][H_q][D] queries of the block's lowest layer (== q if lowest)
+  uint16_t* stash;         // where a lowest layer saves q for its block, else nullptr
+  float* part_acc;         // [B][H_q][max_splits][D]
+  float* part_ml;          // [B][H_q][max_splits][2]  (running max in log2 units, sum)
+  uint16_t* out;           // [B][H_q][D]
+  int32_t* err_flag;
+  int32_t layer, block, split_tokens, max_splits;
+  float scale_log2;        // sm_scale * log2(e)
+};
+
+struct DecodePlan {
+  int32_t split_tokens;   // tokens per split
+  int32_t grid_splits;    // grid.x
+  int32_t n_ctas;         // CTAs that do work
+};
+
+// launchers (defined in the .cu files); return a cudaError_t as int
+int launch_write(const WriteParams& p, cudaStream_t s);
+int launch_decode(const DecodeParams& p, int grid_splits, cudaStream_t s);
+int launch_combine(const DecodeParams& p, cudaStream_t s);
+int decode_resident_ctas_per_sm(int D, int R);   // occupancy of the split-K kernel, 0 on error
+
+}  // namespace pod

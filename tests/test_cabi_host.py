@@ -1,0 +1,182 @@
+"""Host-side checks of the C-ABI library that need no GPU: exported symbols, argument
+validation, call-order rules and byte accounting on a host-only cache (device = -1)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from oracle import pod_oracle as O
+from paper_2412_02252_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "pod.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(pod_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared_functions()
+    assert "pod_cache_create" in names and "pod_decode_attn" in names
+    assert "pod_cache_write" in names and "pod_cache_bytes" in names
+    raw = ctypes.CDLL(B._build.LIB)
+    for n in names:
+        assert hasattr(raw, n), f"{n} declared in pod.h but not exported"
+    assert sorted(B.EXPORTS) == names
+
+
+def _cfg(**kw):
+    base = dict(n_layers=4, n_q_heads=8, n_kv_heads=2, head_dim=64, group_size=2, n_sink=16,
+                n_recent=64, batch=1, device=-1)
+    base.update(kw)
+    return B.make_config(**base)
+
+
+def test_strerror_covers_all_codes():
+    seen = {B.pod_strerror(s) for s in range(-6, 2)}
+    assert len(seen) == 8 and "unknown status" not in seen
+    assert B.pod_strerror(-99) == "unknown status"
+
+
+@pytest.mark.parametrize("bad", [dict(head_dim=96), dict(n_q_heads=7), dict(n_q_heads=32, n_kv_heads=2),
+                                 dict(group_size=0), dict(n_recent=0), dict(n_sink=-1), dict(batch=0),
+                                 dict(n_layers=0), dict(sm_scale=-1.0)])
+def test_invalid_configs_are_rejected(bad):
+    cfg = _cfg(**bad)
+    caps = [512] * max(1, cfg.batch)
+    if cfg.batch >= 1:
+        assert B.pod_cache_required_bytes(cfg, caps) == 0
+        with pytest.raises(B.PodError) as e:
+            B.PodCache(cfg, caps)
+        assert e.value.status == B.POD_ERR_INVALID
+    else:
+        h = ctypes.c_void_p()
+        st = B.lib.pod_cache_create(ctypes.byref(cfg), (ctypes.c_int32 * 1)(512), None, 0, ctypes.byref(h))
+        assert st == B.POD_ERR_INVALID
+
+
+def test_required_bytes_covers_regions_at_capacity():
+    cfg = _cfg()
+    need = B.pod_cache_required_bytes(cfg, [512])
+    live, _ = O.pod_cache_bytes([512], n_layers=4, n_kv_heads=2, head_dim=64, group_size=2, n_s=16, n_r=64)
+    assert need >= live and need % 256 == 0
+    assert B.pod_cache_required_bytes(cfg, [1024]) > need
+    # capacity below the proximal window still reserves the whole sink + ring
+    assert B.pod_cache_required_bytes(cfg, [8]) >= 4 * 2 * 2 * 80 * 128
+
+
+def _fake_ptr():
+    return 0x1000          # never dereferenced by a host-only cache
+
+
+def test_bytes_match_closed_form_and_oracle():
+    for lens, kw in [([512], dict()),
+                     ([100, 80, 512], dict(batch=3)),
+                     ([300], dict(n_layers=5, group_size=2)),          # short last block
+                     ([300], dict(group_size=1)),
+                     ([40], dict())]:
+        cfg = _cfg(**kw)
+        c = B.PodCache(cfg, [max(lens)] * cfg.batch)
+        for l in range(cfg.n_layers):
+            for b, n in enumerate(lens):
+                assert c.write(l, b, _fake_ptr(), _fake_ptr(), n) == B.POD_DRY_RUN
+        live, dense = O.pod_cache_bytes(lens, n_layers=cfg.n_layers, n_kv_heads=2, head_dim=64,
+                                        group_size=cfg.group_size, n_s=16, n_r=64)
+        assert c.bytes(B.POD_BYTES_LIVE) == live
+        assert c.bytes(B.POD_BYTES_DENSE_EQUIV) == dense
+        assert c.bytes(B.POD_BYTES_ALLOCATED) == B.pod_cache_required_bytes(cfg, [max(lens)] * cfg.batch)
+        assert c.bytes(7) == -1
+        for b, n in enumerate(lens):
+            assert c.seq_len(b, 0) == n
+    cfg = _cfg()
+    c = B.PodCache(cfg, [512])
+    for l in range(4):
+        c.write(l, 0, _fake_ptr(), _fake_ptr(), 512)
+    assert c.bytes(B.POD_BYTES_LIVE) == 827392 and c.bytes(B.POD_BYTES_DENSE_EQUIV) == 1048576
+
+
+def test_write_validation_and_capacity():
+    cfg = _cfg(batch=2)
+    c = B.PodCache(cfg, [10, 20])
+    p = _fake_ptr()
+    for args in [(4, 0, p, p, 1), (-1, 0, p, p, 1), (0, 2, p, p, 1), (0, -2, p, p, 1), (0, 0, p, p, 0),
+                 (0, -1, p, p, 2), (0, 0, 0, p, 1), (0, 0, p, 0, 1), (0, 0, p + 8, p, 1)]:
+        with pytest.raises(B.PodError) as e:
+            c.write(*args)
+        assert e.value.status == B.POD_ERR_INVALID
+    c.write(0, 0, p, p, 10)
+    with pytest.raises(B.PodError) as e:
+        c.write(0, 0, p, p, 1)
+    assert e.value.status == B.POD_ERR_CAPACITY
+    with pytest.raises(B.PodError) as e:      # batched append fails if any sequence is full; nothing advances
+        c.write(0, -1, p, p, 1)
+    assert e.value.status == B.POD_ERR_CAPACITY
+    assert c.seq_len(0, 0) == 10 and c.seq_len(1, 0) == 0
+    c.reset(0)
+    assert c.seq_len(0, 0) == 0
+    assert c.write(0, -1, p, p, 1) == B.POD_DRY_RUN
+    assert c.seq_len(0, 0) == 1 and c.seq_len(1, 0) == 1
+
+
+def test_decode_order_rules():
+    cfg = _cfg()
+    c = B.PodCache(cfg, [512])
+    p = _fake_ptr()
+    for l in range(4):
+        c.write(l, 0, p, p, 100)
+    # a non-lowest layer before its block's lowest layer: no stashed query
+    with pytest.raises(B.PodError) as e:
+        c.decode_attn(1, p, p)
+    assert e.value.status == B.POD_ERR_ORDER
+    assert c.decode_attn(0, p, p) == B.POD_DRY_RUN
+    assert c.decode_attn(1, p, p) == B.POD_DRY_RUN
+    with pytest.raises(B.PodError) as e:      # block 1 has its own stash
+        c.decode_attn(3, p, p)
+    assert e.value.status == B.POD_ERR_ORDER
+    # next step, interleaved write/decode per layer as a model would do it
+    c.write(0, 0, p, p, 1)
+    assert c.decode_attn(0, p, p) == B.POD_DRY_RUN
+    with pytest.raises(B.PodError) as e:      # layer 1 not yet appended: block lengths differ
+        c.decode_attn(1, p, p)
+    assert e.value.status == B.POD_ERR_ORDER
+    c.write(1, 0, p, p, 1)
+    assert c.decode_attn(1, p, p) == B.POD_DRY_RUN
+    # stale stash: lowest layer decoded at an older length
+    c.write(0, 0, p, p, 1)
+    c.write(1, 0, p, p, 1)
+    with pytest.raises(B.PodError) as e:
+        c.decode_attn(1, p, p)
+    assert e.value.status == B.POD_ERR_ORDER
+    for args in [(4, p, p), (-1, p, p), (0, 0, p), (0, p, 0), (0, p + 2, p)]:
+        with pytest.raises(B.PodError) as e:
+            c.decode_attn(*args)
+        assert e.value.status == B.POD_ERR_INVALID
+
+
+def test_dense_configuration_needs_no_order():
+    cfg = _cfg(group_size=1)
+    c = B.PodCache(cfg, [64])
+    p = _fake_ptr()
+    for l in range(4):
+        c.write(l, 0, p, p, 5)
+    for l in (3, 1, 0, 2):
+        assert c.decode_attn(l, p, p) == B.POD_DRY_RUN
+
+
+def test_host_only_cache_refuses_device_reads():
+    c = B.PodCache(_cfg(), [64])
+    with pytest.raises(B.PodError):
+        c.read_region(B.POD_REGION_SINK_K, 0, 0, 0, 0, 1)
+    assert c.device_status() == B.POD_DRY_RUN
+
+
+def test_null_handles():
+    assert B.lib.pod_cache_destroy(None) == B.POD_ERR_INVALID
+    assert B.lib.pod_cache_bytes(None, 0) == -1
+    assert B.lib.pod_cache_seq_len(None, 0, 0) == B.POD_ERR_INVALID
+    assert B.lib.pod_cache_reset(None, 0) == B.POD_ERR_INVALID
+    assert B.lib.pod_decode_attn(None, 0, None, None, None) == B.POD_ERR_INVALID
+    assert B.lib.pod_cache_write(None, 0, 0, None, None, 1, None) == B.POD_ERR_INVALID

@@ -1,0 +1,269 @@
+"""GPU parity: the CUDA path through the C ABI against the fp64 oracle on the same seeded
+inputs.  Layout is compared bit for bit; attention within max-abs 1e-2 and relative L2 5e-3."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pod_oracle as O
+from paper_2412_02252_b200 import binding as B
+from paper_2412_02252_b200 import synth
+from podtest import Case, assert_close
+
+pytestmark = pytest.mark.gpu
+
+REGIONS = [("sinkK", B.POD_REGION_SINK_K), ("sinkV", B.POD_REGION_SINK_V),
+           ("ringK", B.POD_REGION_RING_K), ("ringV", B.POD_REGION_RING_V),
+           ("distK", B.POD_REGION_DIST_K), ("distV", B.POD_REGION_DIST_V)]
+
+
+def _oracle_cache(case, b):
+    return O.PodCacheOracle(case.L, case.Hkv, case.d, case.G, case.S, case.W, case.caps[b])
+
+
+def _compare_layout(case, cache, oracles):
+    for b, oc in enumerate(oracles):
+        for name, rid in REGIONS:
+            count = oc.n_blocks if name == "distK" else case.L
+            for i in range(count):
+                for h in range(case.Hkv):
+                    ref, first = oc.valid_rows(name, i, h)
+                    got = cache.read_region(rid, i, b, h, first, ref.shape[0])
+                    np.testing.assert_array_equal(got, ref, err_msg=f"{name}[{i}] seq {b} head {h}")
+
+
+# --------------------------------------------------------------------------- layout
+@pytest.mark.parametrize("chunks", [[40], [1] * 40, [3, 17, 1, 1, 9, 9], [25, 15], [6, 30, 4]])
+@pytest.mark.parametrize("d", [64, 128])
+def test_cache_write_layout_bit_exact(chunks, d):
+    """Prefill, chunked prefill (chunks larger than the window too), appends and ring wraps."""
+    case = Case(seed=21, L=3, G=2, Hq=4, Hkv=2, d=d, S=3, W=7, lens=[sum(chunks)], caps=[sum(chunks) + 5])
+    cache = case.make_cache()
+    oc = _oracle_cache(case, 0)
+    at = 0
+    for t in chunks:
+        for l in range(case.L):
+            k = case.kv(synth.TAG_K, l, 0, at, at + t, "cuda")
+            v = case.kv(synth.TAG_V, l, 0, at, at + t, "cuda")
+            cache.write(l, 0, k, v, t)
+            oc.write(l, synth.bf16_bits(k), synth.bf16_bits(v))
+        at += t
+        _compare_layout(case, cache, [oc])
+        assert cache.seq_len(0, 0) == at
+    live, dense = O.pod_cache_bytes([at], n_layers=3, n_kv_heads=2, head_dim=d, group_size=2, n_s=3, n_r=7)
+    assert cache.bytes(B.POD_BYTES_LIVE) == live and cache.bytes(B.POD_BYTES_DENSE_EQUIV) == dense
+
+
+def test_batched_append_layout_bit_exact():
+    """seq = -1 appends one token to every sequence of a ragged batch, across ring wraps."""
+    lens = [0, 5, 11, 30]
+    case = Case(seed=22, L=2, G=2, Hq=8, Hkv=2, d=64, S=2, W=4, lens=lens, caps=[n + 12 for n in lens])
+    cache = case.make_cache()
+    ocs = [_oracle_cache(case, b) for b in range(case.B)]
+    case.prefill(cache, chunk=7)
+    for b, oc in enumerate(ocs):
+        for l in range(case.L):
+            if lens[b]:
+                oc.write(l, synth.bf16_bits(case.kv(synth.TAG_K, l, b, 0, lens[b], "cpu")),
+                         synth.bf16_bits(case.kv(synth.TAG_V, l, b, 0, lens[b], "cpu")))
+    _compare_layout(case, cache, ocs)
+    for step in range(12):
+        for l in range(case.L):
+            k = torch.stack([case.kv(synth.TAG_K, l, b, lens[b] + step, lens[b] + step + 1, "cuda")[0]
+                             for b in range(case.B)])
+            v = torch.stack([case.kv(synth.TAG_V, l, b, lens[b] + step, lens[b] + step + 1, "cuda")[0]
+                             for b in range(case.B)])
+            cache.write(l, -1, k, v, 1)
+            kb, vb = synth.bf16_bits(k), synth.bf16_bits(v)
+            for b, oc in enumerate(ocs):
+                oc.append(l, kb[b], vb[b])
+        _compare_layout(case, cache, ocs)
+    with pytest.raises(B.PodError) as e:
+        cache.write(0, -1, k, v, 1)
+    assert e.value.status == B.POD_ERR_CAPACITY
+
+
+# --------------------------------------------------------------------------- attention, small
+def _check_all_heads(case, outs, step=0, lens=None):
+    lens = case.lens if lens is None else lens
+    worst = (0.0, 0.0)
+    for l in range(case.L):
+        for b in range(case.B):
+            ref = np.stack([case.oracle_head(l, b, h, n=lens[b], step=step) for h in range(case.Hq)])
+            ma, rl = assert_close(outs[l, b], ref, f"layer {l} seq {b}")
+            worst = (max(worst[0], ma), max(worst[1], rl))
+    return worst
+
+
+def test_config1_tiny_all_heads():
+    """Batch 1, 4 layers, G = 2, 8/2 heads, d = 64, 512 tokens, S = 16, W = 64, seed 0."""
+    case = Case(seed=0, L=4, G=2, Hq=8, Hkv=2, d=64, S=16, W=64, lens=[512])
+    cache = case.make_cache()
+    case.prefill(cache)
+    outs = case.decode_all(cache)
+    _check_all_heads(case, outs)
+    assert cache.bytes(B.POD_BYTES_LIVE) == 827392
+    # the same answer from the layout oracle fed with the same bits
+    oc = _oracle_cache(case, 0)
+    for l in range(4):
+        oc.write(l, synth.bf16_bits(case.kv(synth.TAG_K, l, 0, 0, 512, "cpu")),
+                 synth.bf16_bits(case.kv(synth.TAG_V, l, 0, 0, 512, "cpu")))
+    for l in range(4):
+        q = case.q(l, 0, "cpu")[0].double().numpy()
+        ql = case.q(l - l % 2, 0, "cpu")[0].double().numpy()
+        assert_close(outs[l, 0], oc.attend(l, q, ql), f"layout oracle layer {l}")
+
+
+@pytest.mark.parametrize("d,Hq,Hkv", [(128, 8, 2), (64, 8, 2), (128, 4, 4), (128, 4, 2), (64, 16, 2),
+                                      (128, 16, 2), (128, 6, 2)])
+def test_shapes_and_ragged_batch(d, Hq, Hkv):
+    """Several GQA ratios and head sizes on a ragged batch whose lengths cover: empty, inside the
+    sink, partial ring, exactly S + W, first distant token, several tiles with a ragged tail."""
+    S, W = 4, 24
+    lens = [0, 1, 3, 4, 5, 20, 28, 29, 37, 100, 333, 1000]
+    case = Case(seed=3, L=3, G=2, Hq=Hq, Hkv=Hkv, d=d, S=S, W=W, lens=lens, caps=[max(n, 1) for n in lens])
+    cache = case.make_cache()
+    case.prefill(cache, chunk=97)
+    outs = case.decode_all(cache)
+    _check_all_heads(case, outs)
+    assert (outs[:, 0] == 0).all()          # empty sequence: zeros
+
+
+@pytest.mark.parametrize("G", [1, 3, 4])
+def test_group_sizes(G):
+    case = Case(seed=4, L=5, G=G, Hq=8, Hkv=2, d=128, S=8, W=32, lens=[700, 64])
+    cache = case.make_cache()
+    case.prefill(cache)
+    outs = case.decode_all(cache)
+    _check_all_heads(case, outs)
+
+
+def test_decode_steps_with_window_rollover():
+    """Appends and decodes interleaved per layer, as a model runs them, over ring wraps."""
+    lens0 = [30, 75, 9]
+    case = Case(seed=5, L=4, G=2, Hq=8, Hkv=2, d=128, S=4, W=16, lens=lens0, caps=[n + 40 for n in lens0])
+    cache = case.make_cache()
+    case.prefill(cache)
+    stream = torch.cuda.current_stream().cuda_stream
+    for step in range(1, 36):
+        lens = [n + step for n in lens0]
+        outs = torch.empty(case.L, case.B, case.Hq, case.d, dtype=torch.bfloat16, device="cuda")
+        for l in range(case.L):
+            k = torch.stack([case.kv(synth.TAG_K, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            v = torch.stack([case.kv(synth.TAG_V, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            cache.write(l, -1, k, v, 1, stream)
+            cache.decode_attn(l, case.q(l, step, "cuda"), outs[l], stream)
+        torch.cuda.synchronize()
+        if step in (1, 2, 7, 16, 17, 35):
+            _check_all_heads(case, outs, step=step, lens=lens)
+    assert cache.device_status() == B.POD_OK
+
+
+def test_custom_scale():
+    case = Case(seed=6, L=2, G=2, Hq=4, Hkv=1, d=64, S=2, W=6, lens=[50], scale=0.31)
+    cache = case.make_cache()
+    case.prefill(cache)
+    _check_all_heads(case, case.decode_all(cache))
+
+
+# --------------------------------------------------------------------------- planted keys
+@pytest.mark.parametrize("layer", [0, 1])
+def test_planted_key_at_every_boundary(layer):
+    """A key aligned with the query that scores it dominates the softmax: the output must be
+    that token's value row of the decoded layer.  Planted at region and split boundaries."""
+    L, G, Hq, Hkv, d, S, W, n = 2, 2, 4, 1, 128, 16, 64, 3000
+    seed = 9
+    cfg = B.make_config(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, group_size=G, n_sink=S,
+                        n_recent=W, batch=1, device=0)
+    K = [synth.gen_kv(seed, synth.TAG_K, l, 0, 0, n, Hkv, d, device="cuda") for l in range(L)]
+    V = [synth.gen_kv(seed, synth.TAG_V, l, 0, 0, n, Hkv, d, device="cuda") for l in range(L)]
+    q = [synth.gen_q(seed, l, 0, 1, Hq, d, device="cuda") for l in range(L)]
+    # make all four query heads of the group identical so one planted key serves them all
+    for l in range(L):
+        q[l][:, :] = q[l][:, :1]
+    ring_slot0 = next(p for p in range(n - W, n) if (p - S) % W == 0)
+    positions = [0, S - 1, S, S + 1, n - W - 1, n - W, n - 1, ring_slot0, ring_slot0 - 1,
+                 S + W - 1, S + W, 1500, 1501]
+    cache = B.PodCache(cfg, [n])
+    for l in range(L):
+        cache.write(l, 0, K[l], V[l], n)
+    out = torch.empty(1, Hq, d, dtype=torch.bfloat16, device="cuda")
+    tmp = torch.empty(1, Hq, d, dtype=torch.bfloat16, device="cuda")
+    cache.decode_attn(0, q[0], tmp)
+    st = cache.last_launch()["split_tokens"]
+    positions += [st - 1, st, 2 * st - 1, 2 * st]           # virtual split boundaries (approximate)
+    for pos in sorted(set(p for p in positions if 0 <= p < n)):
+        distant = S <= pos < n - W
+        src = 0 if (distant and layer == 1) else layer
+        Kp = [k.clone() for k in K]
+        qv = q[src][0, 0].float()
+        Kp[src][pos, 0] = (60.0 * qv / qv.norm()).to(torch.bfloat16)
+        cache.reset()
+        for l in range(L):
+            cache.write(l, 0, Kp[l], V[l], n)
+        cache.decode_attn(0, q[0], tmp)
+        cache.decode_attn(1, q[1], out)
+        got = tmp if layer == 0 else out
+        torch.cuda.synchronize()
+        want = V[layer][pos, 0].float()
+        for h in range(Hq):
+            err = (got[0, h].float() - want).abs().max().item()
+            assert err <= 1e-2, f"pos {pos} head {h}: {err}"
+
+
+def test_shared_scores_follow_lowest_layer_query():
+    """At a non-lowest layer, changing the layer's own query leaves an output dominated by a
+    distant planted key untouched; the distant scores are the lowest layer's."""
+    case = Case(seed=10, L=2, G=2, Hq=4, Hkv=1, d=64, S=4, W=8, lens=[400])
+    cache = case.make_cache()
+    K = [case.kv(synth.TAG_K, l, 0, 0, 400, "cuda") for l in range(2)]
+    V = [case.kv(synth.TAG_V, l, 0, 0, 400, "cuda") for l in range(2)]
+    q0, q1 = case.q(0, 0, "cuda"), case.q(1, 0, "cuda")
+    q0[:, :] = q0[:, :1]
+    K[0][200, 0] = (80.0 * q0[0, 0].float() / q0[0, 0].float().norm()).to(torch.bfloat16)
+    for l in range(2):
+        cache.write(l, 0, K[l], V[l], 400)
+    o0 = torch.empty_like(q0)
+    o1 = torch.empty_like(q0)
+    o1b = torch.empty_like(q0)
+    cache.decode_attn(0, q0, o0)
+    cache.decode_attn(1, q1, o1)
+    cache.decode_attn(1, -q1, o1b)
+    torch.cuda.synchronize()
+    want = V[1][200, 0].float()
+    assert (o1[0].float() - want).abs().max() <= 1e-2
+    assert (o1b[0].float() - want).abs().max() <= 1e-2
+
+
+# --------------------------------------------------------------------------- error paths on a device cache
+def test_error_paths_on_device_cache():
+    case = Case(seed=1, L=2, G=2, Hq=4, Hkv=1, d=64, S=2, W=4, lens=[10])
+    cache = case.make_cache()
+    k = case.kv(synth.TAG_K, 0, 0, 0, 10, "cuda")
+    q = case.q(0, 0, "cuda")
+    out = torch.empty_like(q)
+    cache.write(0, 0, k, k, 10)
+    with pytest.raises(B.PodError) as e:
+        cache.write(0, 0, k, k, 1)
+    assert e.value.status == B.POD_ERR_CAPACITY
+    with pytest.raises(B.PodError) as e:
+        cache.decode_attn(1, q, out)
+    assert e.value.status == B.POD_ERR_ORDER
+    arena = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.PodError) as e:
+        B.PodCache(case.cfg, case.caps, arena=arena)
+    assert e.value.status == B.POD_ERR_ARENA
+    need = B.pod_cache_required_bytes(case.cfg, case.caps)
+    arena = torch.empty(need, dtype=torch.uint8, device="cuda")
+    c2 = B.PodCache(case.cfg, case.caps, arena=arena)      # caller-owned arena works
+    c2.write(0, 0, k, k, 10)
+    c2.decode_attn(0, q, out)
+    torch.cuda.synchronize()
+    assert c2.device_status() == B.POD_OK
+    assert_close(out[0], np.stack([_dense_head(case, k, q, h) for h in range(4)]), "arena cache")
+
+
+def _dense_head(case, k, q, h):
+    kk = k[:, 0].double().cpu().numpy()
+    qq = q[0, h].double().cpu().numpy()
+    o, _ = O.pod_attention_joint(qq, qq, kk, kk, kk, case.S, case.W)
+    return o
