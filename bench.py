@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the PoD decode hot path (cache append + decode attention for every layer).
+
+One "step" is one decode step of the whole model's attention: for each layer, append the new
+token's K/V to the PoD cache (``pod_cache_write``) and run ``pod_decode_attn``.  The workload
+is the LLaMA-3-8B-shaped single-sequence decode at 32K context (32 layers, G = 2, 32/8 heads,
+d = 128, S = 16, W = 2048, seeded synthetic bf16 K/V with outlier channels).
+
+    python bench.py --gpus 1 --steps 50 --warmup 5
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference        # the fp64 CPU oracle on the host cores
+
+Prints ONE JSON line (rank 0).  Ranks hold independent sequences (no data-path collective):
+weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOADS = {
+    # name: (batch, context, layers, G, Hq, Hkv, d, S, W, outliers, seed)
+    "llama3-8b-32k": dict(B=1, n=32768, L=32, G=2, Hq=32, Hkv=8, d=128, S=16, W=2048, outliers=True, seed=2),
+    "llama3-8b-128k": dict(B=1, n=131072, L=32, G=2, Hq=32, Hkv=8, d=128, S=16, W=4096, outliers=True, seed=4),
+    "llama3-8b-32k-b16": dict(B=16, n=32768, L=32, G=4, Hq=32, Hkv=8, d=128, S=16, W=1024, outliers=False, seed=3),
+    "tiny": dict(B=1, n=512, L=4, G=2, Hq=8, Hkv=2, d=64, S=16, W=64, outliers=False, seed=0),
+}
+METRIC = "pod_decode_attn_us_per_layer_step"
+UNIT = "us/layer-step"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def _profile_traffic(workload):
+    """DRAM bytes per launch of the split-K kernel from the committed ncu summary, or None."""
+    path = os.path.join(ROOT, "profiles", f"pod_decode_splitk_{workload}.md")
+    try:
+        with open(path) as f:
+            for line in f:
+                if line.startswith("traffic_bytes_per_launch:"):
+                    return float(line.split(":")[1].split()[0])
+    except OSError:
+        pass
+    return None
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 6:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[2:6]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ------------------------------------------------------------------------------ our arm
+def run_ours(args):
+    from paper_2412_02252_b200 import binding as B
+    from paper_2412_02252_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the PoD library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    w = dict(WORKLOADS[args.workload])
+    Bn, n, L, G, Hq, Hkv, d, S, W = (w[k] for k in ("B", "n", "L", "G", "Hq", "Hkv", "d", "S", "W"))
+    seed = w["seed"] + 1000 * rank                       # every rank decodes its own sequences
+    total_steps = args.warmup + args.steps
+    e2e_steps = max(3, min(args.steps, 20))
+    extra = 2 * total_steps + 2 * (e2e_steps + 3) + 8     # headroom for every timed pass
+    dev = torch.device("cuda", local)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def build_cache(group):
+        cfg = B.make_config(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, group_size=group,
+                            n_sink=S, n_recent=W, batch=Bn, device=local)
+        cache = B.PodCache(cfg, [n + extra] * Bn)
+        for l in range(L):
+            for b in range(Bn):
+                at = 0
+                while at < n - 1:
+                    t = min(8192, n - 1 - at)
+                    k = synth.gen_kv(seed, synth.TAG_K, l, b, at, at + t, Hkv, d, outliers=w["outliers"], device=dev)
+                    v = synth.gen_kv(seed, synth.TAG_V, l, b, at, at + t, Hkv, d, outliers=w["outliers"], device=dev)
+                    cache.write(l, b, k, v, t, stream)
+                    at += t
+        torch.cuda.synchronize()
+        return cache
+
+    # per-step inputs, resident in HBM: [step][layer] -> k, v [B][Hkv][d], q [B][Hq][d]
+    n_in = 8
+    def step_inputs(device):
+        ks = torch.stack([torch.stack([torch.stack([
+            synth.gen_kv(seed, synth.TAG_K, l, b, n - 1 + s, n + s, Hkv, d, outliers=w["outliers"], device=device)[0]
+            for b in range(Bn)]) for l in range(L)]) for s in range(n_in)])
+        vs = torch.stack([torch.stack([torch.stack([
+            synth.gen_kv(seed, synth.TAG_V, l, b, n - 1 + s, n + s, Hkv, d, outliers=w["outliers"], device=device)[0]
+            for b in range(Bn)]) for l in range(L)]) for s in range(n_in)])
+        qs = torch.stack([torch.stack([synth.gen_q(seed, l, s, Bn, Hq, d, device=device) for l in range(L)])
+                          for s in range(n_in)])
+        return ks, vs, qs
+
+    ks, vs, qs = step_inputs(dev)
+    outs = torch.empty(L, Bn, Hq, d, dtype=torch.bfloat16, device=dev)
+    launches = [0]
+
+    def step(cache, s, events=None):
+        i = s % n_in
+        for l in range(L):
+            cache.write(l, -1, ks[i, l], vs[i, l], 1, stream)
+            if events is not None:
+                events[l][0].record()
+            cache.decode_attn(l, qs[i, l], outs[l], stream)
+            if events is not None:
+                events[l][1].record()
+        launches[0] += L * (1 + cache.last_launch()["n_kernels"])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(cache, steps, warmup, first_step, per_call=False):
+        """Returns (ms for `steps` steps, list of per-decode-call ms if per_call)."""
+        for s in range(warmup):
+            step(cache, first_step + s)
+        per = []
+        evs = None
+        if per_call:
+            evs = [[[torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)]
+                    for _ in range(L)] for _ in range(steps)]
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        launches[0] = 0
+        t0.record()
+        for s in range(steps):
+            step(cache, first_step + warmup + s, None if evs is None else evs[s])
+        t1.record()
+        barrier()
+        ms = t0.elapsed_time(t1)
+        if per_call:
+            per = [a.elapsed_time(b) for st in evs for (a, b) in st]
+        return ms, per
+
+    def reduce_max(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    cache = build_cache(G)
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.3)
+    # ---- headline: K steps, device-resident inputs ------------------------------------------------
+    ms, _ = timed(cache, args.steps, args.warmup, 0)
+    n_launch = launches[0]
+    ms = reduce_max(ms)
+    # ---- same steps again with an event pair around every decode call (roofline of the kernel) ----
+    ms_ev, per = timed(cache, args.steps, 1, total_steps, per_call=True)
+    clocks = sampler.stop() if sampler else None
+    geo = cache.last_launch()
+    # ---- e2e: host buffers, H2D of k/v/q and D2H of the outputs inside the timed region -----------
+    hk, hv, hq = (x.cpu().pin_memory() for x in (ks, vs, qs))
+    dk, dv, dq = torch.empty_like(ks[0]), torch.empty_like(vs[0]), torch.empty_like(qs[0])
+    hout = torch.empty(L, Bn, Hq, d, dtype=torch.bfloat16).pin_memory()
+
+    def e2e_step(s):
+        i = s % n_in
+        for l in range(L):
+            dk[l].copy_(hk[i, l], non_blocking=True)
+            dv[l].copy_(hv[i, l], non_blocking=True)
+            dq[l].copy_(hq[i, l], non_blocking=True)
+            cache.write(l, -1, dk[l], dv[l], 1, stream)
+            cache.decode_attn(l, dq[l], outs[l], stream)
+        hout.copy_(outs, non_blocking=True)
+        torch.cuda.current_stream().synchronize()      # the caller needs the outputs on the host
+
+    for s in range(3):
+        e2e_step(s)
+    barrier()
+    t0 = time.perf_counter()
+    for s in range(e2e_steps):
+        e2e_step(3 + s)
+    torch.cuda.synchronize()
+    e2e_ms = reduce_max((time.perf_counter() - t0) * 1e3)   # wall clock: the host waits for every step's output
+    barrier()
+    h2d = L * Bn * (2 * Hkv + Hq) * d * 2
+    d2h = L * Bn * Hq * d * 2
+    live = cache.bytes(B.POD_BYTES_LIVE)
+    dense_equiv = cache.bytes(B.POD_BYTES_DENSE_EQUIV)
+    n_now = cache.seq_len(0, 0)
+    assert cache.device_status() == B.POD_OK
+    cache.destroy()
+    del cache
+    torch.cuda.empty_cache()
+
+    # ---- dense-KV baseline: the same kernels with every layer its own block (G = 1) ---------------
+    dense_us = None
+    if world == 1 and not args.no_dense:
+        dcache = build_cache(1)
+        dms, _ = timed(dcache, args.steps, args.warmup, 0)
+        dense_us = dms * 1e3 / (args.steps * L)
+        dcache.destroy()
+        del dcache
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    us_layer = ms * 1e3 / (args.steps * L * world)
+    hbm_peak, peak_kind = _peaks()
+    n_avg = n + args.warmup + args.steps / 2.0
+    alg_bytes = Bn * 2 * n_avg * Hkv * d * 2              # K row-set + V row-set of every token
+    per_us = statistics.mean(per) * 1e3
+    achieved = alg_bytes / (per_us * 1e-6) / 1e9
+    traffic = _profile_traffic(args.workload)
+    line = {
+        "metric": METRIC, "value": round(us_layer, 3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4),
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "batch_per_gpu": Bn, "context": n_now, "layers": L,
+                   "group_size": G, "q_heads": Hq, "kv_heads": Hkv, "head_dim": d, "n_sink": S,
+                   "n_recent": W, "l2": "inputs larger than L2 (a step reads %.1f GiB)" % (L * alg_bytes / 2**30),
+                   "split_tokens": geo["split_tokens"], "ctas": geo["n_ctas"]},
+        "decode_tokens_per_s": round(world * Bn / (ms * 1e-3 / args.steps), 1),
+        "hbm_gbs_step": round(L * alg_bytes / (ms * 1e-3 / args.steps) / 1e9, 1),
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": hbm_peak, "unit": "GB/s",
+                     "frac": round(achieved / hbm_peak, 4), "traffic": traffic, "peak_kind": peak_kind,
+                     "kernel": "pod_decode_attn (split-K + combine)",
+                     "us_per_call": round(per_us, 3), "us_per_call_min": round(min(per) * 1e3, 3),
+                     "algorithmic_bytes_per_call": int(alg_bytes), "frac_of_8TBs": round(achieved / 8000.0, 4)},
+        "e2e": {"value": round(e2e_ms * 1e3 / (e2e_steps * L * world), 3), "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": n_launch,
+        "clocks": clocks,
+        "cache_bytes": {"pod_live": live, "dense_equiv": dense_equiv, "saving": round(1 - live / dense_equiv, 5)},
+        "dense_kv_baseline_us_per_layer_step": None if dense_us is None else round(dense_us, 3),
+    }
+    if not args.no_cpu and world == 1:
+        line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_budget)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------ CPU oracle legs
+def _oracle_block_inputs(workload, block=0, n=None):
+    """fp64 history of one block of layers for sequence 0 (host), and the step's queries."""
+    from paper_2412_02252_b200 import synth
+    w = WORKLOADS[workload]
+    n = w["n"] if n is None else n
+    G, Hkv, d, Hq = w["G"], w["Hkv"], w["d"], w["Hq"]
+    layers = list(range(block * G, min(w["L"], (block + 1) * G)))
+    K = torch.stack([synth.gen_kv(w["seed"], synth.TAG_K, l, 0, 0, n, Hkv, d, outliers=w["outliers"]) for l in layers])
+    V = torch.stack([synth.gen_kv(w["seed"], synth.TAG_V, l, 0, 0, n, Hkv, d, outliers=w["outliers"]) for l in layers])
+    q = torch.stack([synth.gen_q(w["seed"], l, 0, w["B"], Hq, d)[0] for l in layers])
+    return K.double().numpy(), V.double().numpy(), q.double().numpy(), layers
+
+
+def _oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        ts = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(ts) if ts else 1
+    except Exception:
+        return 1
+
+
+def cpu_baseline(workload, budget_s=15.0):
+    """The fp64 oracle, as it stands, on a bounded sample: whole layer-steps (all query heads of
+    one sequence) of the first block of layers, repeated until the budget is used."""
+    from oracle import pod_oracle as O
+    w = WORKLOADS[workload]
+    K, V, q, layers = _oracle_block_inputs(workload)
+    done, t_used = 0, 0.0
+    while t_used < budget_s and done < 64:
+        li = done % len(layers)
+        t0 = time.perf_counter()
+        O.pod_decode_layer(q, K, V, li, group_size=w["G"], n_s=w["S"], n_r=w["W"])
+        t_used += time.perf_counter() - t0
+        done += 1
+    return {"value": round(t_used * 1e6 / done / 1.0, 1), "unit": UNIT, "cores": _oracle_threads(),
+            "host_cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"{done} layer-steps (layers {layers}, all {w['Hq']} query heads, 1 sequence of "
+                      f"{w['n']} tokens) of the {workload} workload; batch scales linearly"}
+
+
+def run_reference(args):
+    """The reference arm of this build is the fp64 CPU oracle (the paper ships no code)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import pod_oracle as O
+    w = WORKLOADS[args.workload]
+    K, V, q, layers = _oracle_block_inputs(args.workload)
+    steps = max(1, min(args.steps, 8))
+    warm = max(0, min(args.warmup, 1))
+
+    def one(i):
+        O.pod_decode_layer(q, K, V, i % len(layers), group_size=w["G"], n_s=w["S"], n_r=w["W"])
+
+    for i in range(warm):
+        one(i)
+    t0 = time.perf_counter()
+    for i in range(steps):
+        one(i)
+    dt = time.perf_counter() - t0
+    us = dt * 1e6 / steps * w["B"]
+    sample = (f"each step = one layer-step of sequence 0 (all {w['Hq']} query heads, {w['n']} tokens), "
+              f"scaled by batch {w['B']}; {steps} steps")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(us, 1), "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": warm,
+        "ms_per_step": round(dt * 1e3 / steps, 3), "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload},
+        "cpu_baseline": {"value": round(us, 1), "unit": UNIT, "kind": "oracle", "cores": _oracle_threads(),
+                         "host_cores": os.cpu_count(), "sample": sample},
+        "e2e": {"value": round(us, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama3-8b-32k", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense-KV baseline leg")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -27,7 +27,7 @@ namespace {
 constexpr int NW = 8;            // warps per CTA
 constexpr int NSTAGE = 3;        // stages of each warp's ring
 constexpr int TILE_BYTES = 2048; // bytes of one K (or V) tile of a warp's stage
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint32_t WAIT_LIMIT = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
