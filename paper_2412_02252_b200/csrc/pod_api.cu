@@ -1,5 +1,6 @@
 // Host side of the PoD library: the C ABI of include/pod.h, argument validation, arena
 // carving, length bookkeeping, split planning and kernel launches.
+#include <cudaTypedefs.h>
 #include <math.h>
 #include <string.h>
 
@@ -13,8 +14,8 @@ using namespace pod;
 
 namespace {
 
-constexpr size_t ALIGN = 256;
-constexpr int MAX_SPLITS_CAP = 128;
+constexpr size_t ALIGN = 1024;        // internal offsets
+constexpr size_t ARENA_ALIGN = 256;   // what a caller's arena must satisfy
 constexpr int TARGET_CTAS_FOR_SPLITS = 148 * 2 * 4;   // used only to size the partial buffers
 constexpr int SPLIT_OVERHEAD_TOKENS = 48;             // fixed cost of a CTA in the planner's model
 
@@ -43,6 +44,7 @@ struct Carve {
   std::vector<int64_t> seq_row_base;   // rows
   std::vector<int32_t> seq_cap_d;
   size_t off_len, off_rowbase, off_capd, off_stash, off_pacc, off_pml, off_err, total;
+  int64_t total_rows;
   int n_blocks, max_splits;
 };
 
@@ -62,6 +64,8 @@ bool carve(const pod_config& c, const int32_t* cap, Carve* out) {
     out->seq_cap_d[b] = (int32_t)cap_d;
     rows += (int64_t)c.n_layers * 2 * c.n_kv_heads * SW + ((int64_t)c.n_layers + n_blocks) * c.n_kv_heads * cap_d;
   }
+  if (rows >= ((int64_t)1 << 31)) return false;   // tile coordinates are 32-bit row indices
+  out->total_rows = rows;
   size_t off = align_up((size_t)(rows * row_bytes));
   out->off_len = off;      off = align_up(off + (size_t)c.n_layers * c.batch * 4);
   out->off_rowbase = off;  off = align_up(off + (size_t)c.batch * 8);
@@ -89,6 +93,7 @@ struct pod_cache {
   int sm_count = 148, resident = 2;
   float scale = 0.f;
   Layout y{};
+  CUtensorMap tmap{};                  // the region rows of the arena as a [rows][d] bf16 tensor
   // last launch (diagnostics)
   int32_t last_split_tokens = 0, last_ctas = 0, last_kernels = 0;
   // planner memo
@@ -104,6 +109,26 @@ namespace {
 int cuda_fail(pod_cache* c, cudaError_t e) {
   c->last_cuda = (int)e;
   return POD_ERR_CUDA;
+}
+
+// One tensor map over all region rows: dims (d, rows), box (64 channels, tile rows), 128-byte
+// swizzle.  Loads past the last row are zero-filled.
+bool make_tensor_map(pod_cache* c) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr)
+    return false;
+  auto encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  const pod_config& g = c->cfg;
+  cuuint64_t dims[2] = {(cuuint64_t)g.head_dim, (cuuint64_t)c->cv.total_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)g.head_dim * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)decode_tile_tokens()};
+  cuuint32_t estr[2] = {1u, 1u};
+  const CUresult r = encode(&c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->arena, dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
 }
 
 // Picks the tokens-per-split that minimises a simple time model: the CTAs run in waves of
@@ -183,7 +208,7 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
   cudaError_t e = cudaSetDevice(cfg->device);
   if (e != cudaSuccess) { delete c; return POD_ERR_CUDA; }
   if (arena_device) {
-    if (((uintptr_t)arena_device % ALIGN) != 0 || arena_bytes < c->cv.total) { delete c; return POD_ERR_ARENA; }
+    if (((uintptr_t)arena_device % ARENA_ALIGN) != 0 || arena_bytes < c->cv.total) { delete c; return POD_ERR_ARENA; }
     c->arena = static_cast<unsigned char*>(arena_device);
   } else {
     void* pmem = nullptr;
@@ -195,12 +220,15 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
   y.seq_row_base = reinterpret_cast<const int64_t*>(c->arena + c->cv.off_rowbase);
   y.seq_cap_d = reinterpret_cast<const int32_t*>(c->arena + c->cv.off_capd);
   bool ok = true;
-  ok = ok && cudaMemset(c->arena + c->cv.off_len, 0, c->cv.total - c->cv.off_len) == cudaSuccess;
+  // Tiles of the decode kernel may extend past the rows a head holds into neighbouring rows;
+  // their logits are masked, but the rows must hold finite numbers, so the arena starts zeroed.
+  ok = ok && cudaMemset(c->arena, 0, c->cv.total) == cudaSuccess;
+  ok = ok && make_tensor_map(c);
   ok = ok && cudaMemcpy(c->arena + c->cv.off_rowbase, c->cv.seq_row_base.data(), (size_t)cfg->batch * 8, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->arena + c->cv.off_capd, c->cv.seq_cap_d.data(), (size_t)cfg->batch * 4, cudaMemcpyHostToDevice) == cudaSuccess;
   int sm = 0;
   ok = ok && cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess;
-  const int res = ok ? decode_resident_ctas_per_sm(cfg->head_dim, cfg->n_q_heads / cfg->n_kv_heads) : 0;
+  const int res = ok ? decode_resident_ctas_per_sm(cfg->head_dim) : 0;
   ok = ok && res > 0 && cudaDeviceSynchronize() == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
@@ -289,7 +317,7 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* str
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int kernels = 0;
   if (plan.n_ctas > 0) {
-    const int e = launch_decode(p, plan.grid_splits, s);
+    const int e = launch_decode(c->tmap, p, plan.grid_splits, s);
     if (e != 0) return cuda_fail(c, (cudaError_t)e);
     ++kernels;
   }

@@ -2,10 +2,13 @@
 // decode kernels).  Private to the library; the public surface is include/pod.h.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace pod {
+
+constexpr int MAX_SPLITS_CAP = 128;   // upper bound of splits per sequence (partial buffers, combine)
 
 // Physical layout of the arena.  All offsets are in rows; one row is one head's d bf16
 // values (128 B at d = 64, 256 B at d = 128), so every region base is 128-byte aligned.
@@ -68,8 +71,9 @@ struct DecodePlan {
 
 // launchers (defined in the .cu files); return a cudaError_t as int
 int launch_write(const WriteParams& p, cudaStream_t s);
-int launch_decode(const DecodeParams& p, int grid_splits, cudaStream_t s);
+int launch_decode(const CUtensorMap& tmap, const DecodeParams& p, int grid_splits, cudaStream_t s);
 int launch_combine(const DecodeParams& p, cudaStream_t s);
-int decode_resident_ctas_per_sm(int D, int R);   // occupancy of the split-K kernel, 0 on error
+int decode_resident_ctas_per_sm(int D);   // occupancy of the split-K kernel, 0 on error
+int decode_tile_tokens();                 // rows of the TMA box the split-K kernel loads
 
 }  // namespace pod

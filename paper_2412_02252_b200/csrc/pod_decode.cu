@@ -3,16 +3,20 @@
 // Grid (split, KV head, sequence).  A CTA owns a contiguous range of the sequence's tokens in
 // "virtual" order -- proximal rows first (sink, then ring slots), distant rows after -- and
 // its warps subdivide that range.  Each warp is an independent flash-decoding stream:
-//   * lane 0 stages tiles of K rows and V rows into the warp's private shared-memory ring
-//     with 1-D bulk async copies (TMA, no multicast) that complete on an mbarrier;
-//   * the lanes of a row group each hold 8 of the d channels of q (all r query heads of the
-//     KV head) in registers, multiply their 16-byte chunk of a K row against them with packed
-//     fp32 FMAs, and a transposing butterfly leaves one (token, head) logit per lane;
-//   * one online softmax in base 2 (logits pre-scaled by log2 e) runs over proximal and
-//     distant rows alike: only the query registers (own query for proximal rows, the block's
-//     lowest-layer query for distant rows) and the K/V base pointers change at the boundary;
-//   * probabilities go through a small shared buffer and are applied to the V chunk of
-//     each lane with packed fp32 FMAs.
+//   * lane 0 stages tiles of 16 K rows and 16 V rows into the warp's private shared-memory
+//     ring with tiled TMA loads (one tensor map views the whole arena as [rows][d]; 128-byte
+//     swizzle, no multicast) that complete on an mbarrier;
+//   * logits: S[16 x 16] = Q[16 x d] K^T with mma.sync m16n8k16 (bf16 in, fp32 out).  The rows
+//     of Q are the r <= 8 query heads of the KV head, zero-padded to 16; K fragments come from
+//     ldmatrix on the swizzled tile, so the bf16 data is never unpacked by ALU instructions;
+//   * one online softmax in base 2 runs over proximal and distant rows alike: at the boundary
+//     only the Q fragments (own query for proximal rows, the block's lowest-layer query for
+//     distant rows) and the tile coordinates change;
+//   * values: O[16 x d] += P[16 x 16] V[16 x d], P rounded to bf16 in the accumulator-to-A
+//     register layout, V fragments from ldmatrix.trans.
+// An earlier CUDA-core version of this kernel (packed fp32 FMAs on unpacked bf16) was bound by
+// instruction issue at half the memory rate; the tensor-core form needs about a tenth of the
+// instructions and leaves the kernel memory-bound.
 // Warps merge through shared memory; the CTA writes one fp32 partial (acc, max, sum) per
 // query head.  A second kernel merges the partials of a (sequence, head) and rounds to bf16.
 // Every mbarrier wait is bounded; a wait that gives up raises the cache's error flag.
@@ -24,9 +28,10 @@ namespace pod {
 
 namespace {
 
-constexpr int NW = 8;            // warps per CTA
+constexpr int NW = 4;            // warps per CTA
 constexpr int NSTAGE = 3;        // stages of each warp's ring
-constexpr int TILE_BYTES = 2048; // bytes of one K (or V) tile of a warp's stage
+constexpr int TOK = 16;          // tokens per tile (one mma k-step of P V)
+constexpr int CTAS_PER_SM = 2;
 constexpr uint32_t WAIT_LIMIT = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -53,12 +58,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   }
   return false;
 }
-// 1-D bulk copy global -> shared, completing `bytes` on the mbarrier.  Source, destination
-// and size are multiples of 16 bytes (rows are 128 or 256 bytes).
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+// Tiled TMA load of a [TOK rows][64 bf16] box at (x, y) = (channel, arena row).  x is 0 or
+// 64 elements, i.e. a multiple of 16 bytes as TMA requires.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar) {
   asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
@@ -66,60 +71,59 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
+__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
-// two packed bf16 -> two fp32 (exact)
-__device__ __forceinline__ float2 bf2(uint32_t w) {
-  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+__device__ __forceinline__ void ldsm4_t(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
-__device__ __forceinline__ void unpack8(const uint4& r, float2 (&f)[4]) {
-  f[0] = bf2(r.x); f[1] = bf2(r.y); f[2] = bf2(r.z); f[3] = bf2(r.w);
+// D = A (16x16, bf16, row) * B (16x8, bf16, col) + D, fp32 accumulate
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int D, int R>
+template <int D>
 struct Cfg {
-  static constexpr int LPR = D / 8;            // lanes per row
-  static constexpr int NG = 32 / LPR;          // row groups per warp
-  static constexpr int TG = LPR / R;           // tokens per row group per iteration
-  static constexpr int TOK_IT = NG * TG;       // tokens per iteration (= 32 / R)
-  static constexpr int ROWB = D * 2;
-  static constexpr int TILE_B = TILE_BYTES;    // bytes of one K (or V) tile
-  static constexpr int TOK = TILE_B / ROWB;    // tokens per stage
-  static constexpr int ITERS = TOK / TOK_IT;   // softmax iterations per stage
-  static constexpr int WARP_B = NSTAGE * 2 * TILE_B;
-  static constexpr int PS_FLOATS = 2 * TOK_IT * R;   // double-buffered probabilities
-  static constexpr int SMEM = NW * WARP_B + NW * PS_FLOATS * 4 + NW * NSTAGE * 8;
-  static_assert(TG >= 1, "r must not exceed d / 8");
-  static_assert(ITERS >= 1 && ITERS * TOK_IT == TOK, "a stage holds whole iterations");
-  static_assert(WARP_B >= (R * D + 2 * R) * 4, "merge scratch must fit the warp's ring");
+  static constexpr int NSUB = D / 64;                 // 128-byte wide sub-tiles per row
+  static constexpr int SUB_B = TOK * 128;             // bytes of one sub-tile (1024-byte multiple)
+  static constexpr int TILE_B = NSUB * SUB_B;         // bytes of one K (or V) tile
+  static constexpr int STAGE_B = 2 * TILE_B;
+  static constexpr int WARP_B = NSTAGE * STAGE_B;
+  static constexpr int SMEM = NW * WARP_B + NW * NSTAGE * 8 + 1024;   // + slack to align to 1024
+  static_assert(WARP_B >= (8 * D + 16) * 4, "merge scratch must fit the warp's ring");
 };
 
-template <int D, int R>
-__global__ void __launch_bounds__(NW * 32, (R > 4 ? 1 : 2)) pod_decode_splitk_kernel(const DecodeParams p) {
-  using C = Cfg<D, R>;
-  constexpr int LPR = C::LPR, TG = C::TG, TOK_IT = C::TOK_IT, TOK = C::TOK, ROWB = C::ROWB;
-  constexpr int ITERS = C::ITERS;
+template <int D>
+__global__ void __launch_bounds__(NW * 32, CTAS_PER_SM)
+pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams p) {
+  using C = Cfg<D>;
   const Layout& y = p.y;
-  const int r = y.H_q / y.H_kv;   // query heads per KV head; R >= r is the compute width
+  const int r = y.H_q / y.H_kv;   // query heads per KV head (<= 8): rows of the Q operand
 
   const int b = blockIdx.z, kvh = blockIdx.y, split = blockIdx.x;
   const int n = p.len[b];
   const int nsplit = min(p.max_splits, (n + p.split_tokens - 1) / p.split_tokens);
   if (split >= nsplit) return;
 
-  extern __shared__ __align__(128) unsigned char smem[];
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);   // swizzle atoms are 1024 B
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int gi = lane / LPR, sub = lane % LPR;
   unsigned char* wbuf = smem + warp * C::WARP_B;
-  float* ps = reinterpret_cast<float*>(smem + NW * C::WARP_B) + warp * C::PS_FLOATS;
-  const uint32_t bar0 = smem_u32(smem + NW * C::WARP_B + NW * C::PS_FLOATS * 4) + warp * NSTAGE * 8;
   const uint32_t wbuf_s = smem_u32(wbuf);
-  const uint32_t ps_s = smem_u32(ps);
+  const uint32_t bar0 = smem_u32(smem + NW * C::WARP_B) + warp * NSTAGE * 8;
 
-  // ---- token ranges -----------------------------------------------------------------
+  // ---- token ranges ---------------------------------------------------------------------
   const int n_p = min(n, y.S + y.W);
   const int c0 = (int)((int64_t)n * split / nsplit), c1 = (int)((int64_t)n * (split + 1) / nsplit);
   const int w0 = c0 + (int)((int64_t)(c1 - c0) * warp / NW);
@@ -129,27 +133,29 @@ __global__ void __launch_bounds__(NW * 32, (R > 4 ? 1 : 2)) pod_decode_splitk_ke
   const int ntp = (pa1 - pa0 + TOK - 1) / TOK, ntd = (da1 - da0 + TOK - 1) / TOK;
   const int nt = ntp + ntd;
 
+  // arena rows of this (sequence, layer, head): tile coordinates of the tensor map
   const int64_t cap_d = y.seq_cap_d[b];
-  const uint16_t* seq_base = p.arena + y.seq_row_base[b] * D;
-  const uint16_t* Kp = seq_base + prox_row(y, p.layer, 0, kvh) * D;
-  const uint16_t* Vp = seq_base + prox_row(y, p.layer, 1, kvh) * D;
-  const uint16_t* Kd = seq_base + distk_row(y, p.block, kvh, cap_d) * D;
-  const uint16_t* Vd = seq_base + distv_row(y, p.layer, kvh, cap_d) * D;
+  const int64_t seq_row = y.seq_row_base[b];
+  const int rowKp = (int)(seq_row + prox_row(y, p.layer, 0, kvh));
+  const int rowVp = (int)(seq_row + prox_row(y, p.layer, 1, kvh));
+  const int rowKd = (int)(seq_row + distk_row(y, p.block, kvh, cap_d));
+  const int rowVd = (int)(seq_row + distv_row(y, p.layer, kvh, cap_d));
 
   auto tile_rows = [&](int t) -> int {
     return t < ntp ? min(TOK, pa1 - (pa0 + t * TOK)) : min(TOK, da1 - (da0 + (t - ntp) * TOK));
   };
-  auto issue = [&](int t) {   // lane 0 only
-    const int stage = t % NSTAGE;
-    const int cnt = tile_rows(t);
-    const uint16_t *kp, *vp;
-    if (t < ntp) { const int64_t off = pa0 + (int64_t)t * TOK; kp = Kp + off * D; vp = Vp + off * D; }
-    else { const int64_t off = da0 + (int64_t)(t - ntp) * TOK; kp = Kd + off * D; vp = Vd + off * D; }
+  auto issue = [&](int t) {   // lane 0 only.  Rows past the piece are other (finite) cache rows
+    const int stage = t % NSTAGE;   // or zero fill past the arena; their logits are masked.
+    const int yk = t < ntp ? rowKp + pa0 + t * TOK : rowKd + da0 + (t - ntp) * TOK;
+    const int yv = t < ntp ? rowVp + pa0 + t * TOK : rowVd + da0 + (t - ntp) * TOK;
     const uint32_t bar = bar0 + stage * 8;
-    const uint32_t bytes = (uint32_t)cnt * ROWB;
-    mbar_expect_tx(bar, 2 * bytes);
-    bulk_g2s(wbuf_s + stage * 2 * C::TILE_B, kp, bytes, bar);
-    bulk_g2s(wbuf_s + stage * 2 * C::TILE_B + C::TILE_B, vp, bytes, bar);
+    const uint32_t dst = wbuf_s + stage * C::STAGE_B;
+    mbar_expect_tx(bar, C::STAGE_B);
+#pragma unroll
+    for (int s = 0; s < C::NSUB; ++s) {
+      tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yk, bar);
+      tma_load_2d(dst + C::TILE_B + s * C::SUB_B, &tmap, s * 64, yv, bar);
+    }
   };
 
   if (lane == 0) {
@@ -160,38 +166,40 @@ __global__ void __launch_bounds__(NW * 32, (R > 4 ? 1 : 2)) pod_decode_splitk_ke
   }
 
   // a lowest layer saves its query for the other layers of the block
-  if (p.stash != nullptr && split == 0 && warp == 0 && gi == 0) {
+  if (p.stash != nullptr && split == 0 && warp == 0 && lane < D / 8) {
     for (int h = 0; h < r; ++h) {
-      const int64_t o = ((int64_t)b * y.H_q + kvh * r + h) * D + sub * 8;
+      const int64_t o = ((int64_t)b * y.H_q + kvh * r + h) * D + lane * 8;
       *reinterpret_cast<uint4*>(p.stash + o) = *reinterpret_cast<const uint4*>(p.q + o);
     }
   }
   __syncwarp();
 
-  // ---- per-lane state -----------------------------------------------------------------
-  float2 qr[R][4];            // this lane's 8 channels of the r queries, scaled to log2 units
-  float2 acc[R][4];           // this lane's 8 channels of the r outputs (row group partial)
+  // ---- per-lane state -------------------------------------------------------------------
+  const int qrow = lane >> 2;          // query head (row of S and O) owned by this lane's quad
+  const int qcol = (lane & 3) * 2;     // first of the two columns this lane holds in a fragment
+  uint32_t qa[D / 16][2];              // A fragments of Q: rows 0..7 only (rows 8..15 are zero)
+  float o[D / 8][4];                   // O accumulators; [.][2], [.][3] belong to the zero rows
 #pragma unroll
-  for (int h = 0; h < R; ++h)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) acc[h][j] = make_float2(0.f, 0.f);
-  const int own_h = sub % R;  // the (token, head) pair whose logit lands in this lane
-  const int own_t = gi * TG + sub / R;
-  float m_own = -INFINITY, l_own = 0.f;
+  for (int c = 0; c < D / 8; ++c) { o[c][0] = o[c][1] = o[c][2] = o[c][3] = 0.f; }
+  float m_row = -INFINITY, l_row = 0.f;
   bool failed = false;
 
   auto load_q = [&](const uint16_t* qsrc) {
+    const uint16_t* base = qsrc + ((int64_t)b * y.H_q + kvh * r + qrow) * D + qcol;
 #pragma unroll
-    for (int h = 0; h < R; ++h) {
-      uint4 raw = make_uint4(0u, 0u, 0u, 0u);   // padded heads score 0 and are never written
-      if (h < r)
-        raw = *reinterpret_cast<const uint4*>(qsrc + ((int64_t)b * y.H_q + kvh * r + h) * D + sub * 8);
-      float2 f[4];
-      unpack8(raw, f);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) qr[h][j] = make_float2(f[j].x * p.scale_log2, f[j].y * p.scale_log2);
+    for (int kk = 0; kk < D / 16; ++kk) {
+      qa[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(base + kk * 16) : 0u;
+      qa[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(base + kk * 16 + 8) : 0u;
     }
   };
+
+  // ldmatrix lane addressing inside a [TOK][128 B] sub-tile with the 128-byte swizzle:
+  // 16-byte chunk c of row t lives at t * 128 + ((c ^ (t & 7)) << 4).
+  const int lm = lane >> 3, lr = lane & 7;
+  // K (non-transposed): matrices (tokens 0-7, chunk 2kk), (0-7, 2kk+1), (8-15, 2kk), (8-15, 2kk+1)
+  const int k_tok = (lm >> 1) * 8 + lr, k_chunk = lm & 1;
+  // V (transposed): matrices (tokens 0-7, chunk c), (8-15, c), (0-7, c+1), (8-15, c+1)
+  const int v_tok = (lm & 1) * 8 + lr, v_chunk = lm >> 1;
 
   int t = 0;
   for (; t < nt; ++t) {
@@ -199,88 +207,46 @@ __global__ void __launch_bounds__(NW * 32, (R > 4 ? 1 : 2)) pod_decode_splitk_ke
     const int stage = t % NSTAGE;
     if (!__all_sync(0xffffffffu, mbar_wait(bar0 + stage * 8, (t / NSTAGE) & 1))) { failed = true; break; }
     const int cnt = tile_rows(t);
-    const uint32_t ks = wbuf_s + stage * 2 * C::TILE_B + sub * 16;
+    const uint32_t ks = wbuf_s + stage * C::STAGE_B;
     const uint32_t vs = ks + C::TILE_B;
 
+    // ---- S = Q K^T ------------------------------------------------------------------------
+    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int it = 0; it < ITERS; ++it) {
-      if (it * TOK_IT >= cnt) break;
-      // ---- logits: TG rows of this row group against r queries -------------------------
-      float v[LPR];
+    for (int kk = 0; kk < D / 16; ++kk) {
+      const int chunk = 2 * kk + k_chunk;          // 16-byte chunk of the row
+      uint32_t bfr[4];
+      ldsm4(ks + (chunk >> 3) * C::SUB_B + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), bfr);
+      mma16816(s0, qa[kk][0], 0u, qa[kk][1], 0u, bfr[0], bfr[1]);
+      mma16816(s1, qa[kk][0], 0u, qa[kk][1], 0u, bfr[2], bfr[3]);
+    }
+    // ---- online softmax (base 2) over this lane's row -----------------------------------------
+    float a00 = (qcol < cnt) ? s0[0] * p.scale_log2 : -INFINITY;
+    float a01 = (qcol + 1 < cnt) ? s0[1] * p.scale_log2 : -INFINITY;
+    float a10 = (qcol + 8 < cnt) ? s1[0] * p.scale_log2 : -INFINITY;
+    float a11 = (qcol + 9 < cnt) ? s1[1] * p.scale_log2 : -INFINITY;
+    float mx = fmaxf(fmaxf(a00, a01), fmaxf(a10, a11));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    if (__any_sync(0xffffffffu, mx > m_row)) {
+      const float m_new = fmaxf(m_row, mx);
+      const float alpha = ex2(m_row - m_new);       // 0 on the first tile, 1 if unchanged
+      m_row = m_new;
+      l_row *= alpha;
 #pragma unroll
-      for (int tt = 0; tt < TG; ++tt) {
-        const int row = min(it * TOK_IT + gi * TG + tt, cnt - 1);
-        float2 kf[4];
-        unpack8(lds128(ks + row * ROWB), kf);
+      for (int c = 0; c < D / 8; ++c) { o[c][0] *= alpha; o[c][1] *= alpha; }
+    }
+    a00 = ex2(a00 - m_row); a01 = ex2(a01 - m_row); a10 = ex2(a10 - m_row); a11 = ex2(a11 - m_row);
+    l_row += (a00 + a01) + (a10 + a11);
+    const uint32_t pa0 = pack_bf16(a00, a01), pa2 = pack_bf16(a10, a11);
+    // ---- O += P V ---------------------------------------------------------------------------
 #pragma unroll
-        for (int h = 0; h < R; ++h) {
-          float2 a = __fmul2_rn(kf[0], qr[h][0]);
-          a = __ffma2_rn(kf[1], qr[h][1], a);
-          a = __ffma2_rn(kf[2], qr[h][2], a);
-          a = __ffma2_rn(kf[3], qr[h][3], a);
-          v[tt * R + h] = a.x + a.y;
-        }
-      }
-      // transposing butterfly over the LPR lanes of the row group: LPR values -> 1 per lane
-#pragma unroll
-      for (int o = LPR / 2; o >= 1; o >>= 1) {
-        const bool up = (lane & o) != 0;
-#pragma unroll
-        for (int i = 0; i < o; ++i) {
-          const float send = up ? v[i] : v[i + o];
-          const float keep = up ? v[i + o] : v[i];
-          v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-        }
-      }
-      float s = (it * TOK_IT + own_t < cnt) ? v[0] : -INFINITY;
-      // ---- online softmax ---------------------------------------------------------------
-      float mx = s;
-#pragma unroll
-      for (int o = R; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      if (__any_sync(0xffffffffu, mx > m_own)) {
-        const float m_new = fmaxf(m_own, mx);
-        const float alpha = ex2(m_own - m_new);     // 0 on the first tile, 1 if unchanged
-        l_own *= alpha;
-        m_own = m_new;
-#pragma unroll
-        for (int h = 0; h < R; ++h) {
-          const float ah = __shfl_sync(0xffffffffu, alpha, h);
-          const float2 a2 = make_float2(ah, ah);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) acc[h][j] = __fmul2_rn(acc[h][j], a2);
-        }
-      }
-      const float pr = ex2(s - m_own);
-      l_own += pr;
-      float* psb = ps + (it & 1) * (TOK_IT * R);
-      psb[own_t * R + own_h] = pr;
-      __syncwarp();
-      // ---- values -------------------------------------------------------------------------
-      const uint32_t psb_s = ps_s + (it & 1) * (TOK_IT * R * 4);
-#pragma unroll
-      for (int tt = 0; tt < TG; ++tt) {
-        const int row = min(it * TOK_IT + gi * TG + tt, cnt - 1);
-        float2 vf[4];
-        unpack8(lds128(vs + row * ROWB), vf);
-        float pw[R];
-        if constexpr (R == 8) {
-          const uint4 a = lds128(psb_s + (gi * TG + tt) * R * 4), c = lds128(psb_s + (gi * TG + tt) * R * 4 + 16);
-          pw[0] = __uint_as_float(a.x); pw[1] = __uint_as_float(a.y); pw[2] = __uint_as_float(a.z); pw[3] = __uint_as_float(a.w);
-          pw[4] = __uint_as_float(c.x); pw[5] = __uint_as_float(c.y); pw[6] = __uint_as_float(c.z); pw[7] = __uint_as_float(c.w);
-        } else if constexpr (R == 4) {
-          const uint4 a = lds128(psb_s + (gi * TG + tt) * R * 4);
-          pw[0] = __uint_as_float(a.x); pw[1] = __uint_as_float(a.y); pw[2] = __uint_as_float(a.z); pw[3] = __uint_as_float(a.w);
-        } else {
-#pragma unroll
-          for (int h = 0; h < R; ++h) pw[h] = psb[(gi * TG + tt) * R + h];
-        }
-#pragma unroll
-        for (int h = 0; h < R; ++h) {
-          const float2 p2 = make_float2(pw[h], pw[h]);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) acc[h][j] = __ffma2_rn(vf[j], p2, acc[h][j]);
-        }
-      }
+    for (int c = 0; c < D / 8; c += 2) {
+      const int chunk = c + v_chunk;
+      uint32_t bfr[4];
+      ldsm4_t(vs + (chunk >> 3) * C::SUB_B + v_tok * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), bfr);
+      mma16816(o[c], pa0, 0u, pa2, 0u, bfr[0], bfr[1]);
+      mma16816(o[c + 1], pa0, 0u, pa2, 0u, bfr[2], bfr[3]);
     }
     __syncwarp();                          // all lanes are done reading this stage
     if (lane == 0 && t + NSTAGE < nt) issue(t + NSTAGE);
@@ -292,46 +258,31 @@ __global__ void __launch_bounds__(NW * 32, (R > 4 ? 1 : 2)) pod_decode_splitk_ke
     for (int u = t; u < nt && u < t + NSTAGE; ++u) mbar_wait(bar0 + (u % NSTAGE) * 8, (u / NSTAGE) & 1);
   }
 
-  // ---- merge the row groups of the warp, then the warps of the CTA ------------------------
-#pragma unroll
-  for (int o = LPR; o < 32; o <<= 1)
-#pragma unroll
-    for (int h = 0; h < R; ++h)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        acc[h][j].x += __shfl_xor_sync(0xffffffffu, acc[h][j].x, o);
-        acc[h][j].y += __shfl_xor_sync(0xffffffffu, acc[h][j].y, o);
-      }
-#pragma unroll
-  for (int o = R; o < 32; o <<= 1) l_own += __shfl_xor_sync(0xffffffffu, l_own, o);
-
+  // ---- merge the warps of the CTA -------------------------------------------------------------
+  l_row += __shfl_xor_sync(0xffffffffu, l_row, 1);
+  l_row += __shfl_xor_sync(0xffffffffu, l_row, 2);
   __syncwarp();
-  float* mine = reinterpret_cast<float*>(wbuf);    // [R][D] acc, then [R] max, [R] sum
-  if (gi == 0) {
+  float* mine = reinterpret_cast<float*>(wbuf);    // [8][D] acc, then [8] max, [8] sum
 #pragma unroll
-    for (int h = 0; h < R; ++h)
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        *reinterpret_cast<float2*>(mine + h * D + sub * 8 + j * 2) = acc[h][j];
-  }
-  if (lane < R) { mine[R * D + lane] = m_own; mine[R * D + R + lane] = l_own; }
+  for (int c = 0; c < D / 8; ++c)
+    *reinterpret_cast<float2*>(mine + qrow * D + c * 8 + qcol) = make_float2(o[c][0], o[c][1]);
+  if ((lane & 3) == 0) { mine[8 * D + qrow] = m_row; mine[8 * D + 8 + qrow] = l_row; }
   __syncthreads();
 
-  for (int idx = threadIdx.x; idx < R * D; idx += NW * 32) {
+  for (int idx = threadIdx.x; idx < r * D; idx += NW * 32) {
     const int h = idx / D, c = idx % D;
-    if (h >= r) break;
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < NW; ++w)
-      M = fmaxf(M, reinterpret_cast<const float*>(smem + w * C::WARP_B)[R * D + h]);
+      M = fmaxf(M, reinterpret_cast<const float*>(smem + w * C::WARP_B)[8 * D + h]);
     float a = 0.f, l = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) {
-      const float* o = reinterpret_cast<const float*>(smem + w * C::WARP_B);
-      const float mw = o[R * D + h];
+      const float* ow = reinterpret_cast<const float*>(smem + w * C::WARP_B);
+      const float mw = ow[8 * D + h];
       const float sc = (mw == -INFINITY) ? 0.f : ex2(mw - M);
-      a += o[h * D + c] * sc;
-      l += o[R * D + R + h] * sc;
+      a += ow[h * D + c] * sc;
+      l += ow[8 * D + 8 + h] * sc;
     }
     const int64_t ph = ((int64_t)b * y.H_q + kvh * r + h) * p.max_splits + split;
     p.part_acc[ph * D + c] = a;
@@ -347,51 +298,76 @@ __global__ void __launch_bounds__(D) pod_combine_kernel(const DecodeParams p) {
   const int n = p.len[b];
   const int nsplit = min(p.max_splits, (n + p.split_tokens - 1) / p.split_tokens);
   const int64_t ph = ((int64_t)b * p.y.H_q + hq) * p.max_splits;
-  float M = -INFINITY;
-  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p.part_ml[(ph + s) * 2]);
-  float a = 0.f, l = 0.f;
-  for (int s = 0; s < nsplit; ++s) {
+  __shared__ float s_w[MAX_SPLITS_CAP];     // weight of each split: 2^(m_s - M)
+  __shared__ float s_red[2][4];
+  // pass 1: every thread takes some splits' (max, sum); block-wide max
+  float mloc = -INFINITY;
+  for (int s = c; s < nsplit; s += D) mloc = fmaxf(mloc, p.part_ml[(ph + s) * 2]);
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o));
+  if ((c & 31) == 0) s_red[0][c >> 5] = mloc;
+  __syncthreads();
+  float M = s_red[0][0];
+  for (int w = 1; w < D / 32; ++w) M = fmaxf(M, s_red[0][w]);
+  float lloc = 0.f;
+  for (int s = c; s < nsplit; s += D) {
     const float ms = p.part_ml[(ph + s) * 2];
-    const float sc = (ms == -INFINITY) ? 0.f : ex2(ms - M);
-    a += p.part_acc[(ph + s) * D + c] * sc;
-    l += p.part_ml[(ph + s) * 2 + 1] * sc;
+    const float wgt = (ms == -INFINITY) ? 0.f : ex2(ms - M);
+    s_w[s] = wgt;
+    lloc += p.part_ml[(ph + s) * 2 + 1] * wgt;
   }
-  const float o = (l > 0.f) ? a / l : 0.f;
-  reinterpret_cast<__nv_bfloat16*>(p.out)[((int64_t)b * p.y.H_q + hq) * D + c] = __float2bfloat16_rn(o);
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) lloc += __shfl_xor_sync(0xffffffffu, lloc, o);
+  if ((c & 31) == 0) s_red[1][c >> 5] = lloc;
+  __syncthreads();
+  float l = 0.f;
+  for (int w = 0; w < D / 32; ++w) l += s_red[1][w];
+  // pass 2: channel c over the splits, loads independent of one another
+  float a = 0.f;
+  int s = 0;
+  for (; s + 4 <= nsplit; s += 4) {
+    const float v0 = p.part_acc[(ph + s) * D + c], v1 = p.part_acc[(ph + s + 1) * D + c];
+    const float v2 = p.part_acc[(ph + s + 2) * D + c], v3 = p.part_acc[(ph + s + 3) * D + c];
+    a += v0 * s_w[s] + v1 * s_w[s + 1] + v2 * s_w[s + 2] + v3 * s_w[s + 3];
+  }
+  for (; s < nsplit; ++s) a += p.part_acc[(ph + s) * D + c] * s_w[s];
+  const float out = (l > 0.f) ? a / l : 0.f;
+  reinterpret_cast<__nv_bfloat16*>(p.out)[((int64_t)b * p.y.H_q + hq) * D + c] = __float2bfloat16_rn(out);
 }
 
-template <int D, int R>
-int launch_decode_t(const DecodeParams& p, int grid_splits, cudaStream_t s) {
-  using C = Cfg<D, R>;
+template <int D>
+int launch_decode_t(const CUtensorMap& tmap, const DecodeParams& p, int grid_splits, cudaStream_t s) {
+  using C = Cfg<D>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(pod_decode_splitk_kernel<D, R>,
+    cudaError_t e = cudaFuncSetAttribute(pod_decode_splitk_kernel<D>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return (int)e;
     configured = true;
   }
   dim3 grid(grid_splits, p.y.H_kv, p.y.B);
-  pod_decode_splitk_kernel<D, R><<<grid, NW * 32, C::SMEM, s>>>(p);
+  pod_decode_splitk_kernel<D><<<grid, NW * 32, C::SMEM, s>>>(tmap, p);
   return (int)cudaGetLastError();
 }
 
-template <int D, int R>
+template <int D>
 int resident_t() {
-  using C = Cfg<D, R>;
-  cudaError_t e = cudaFuncSetAttribute(pod_decode_splitk_kernel<D, R>,
+  using C = Cfg<D>;
+  cudaError_t e = cudaFuncSetAttribute(pod_decode_splitk_kernel<D>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
   if (e != cudaSuccess) return 0;
   int nb = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, pod_decode_splitk_kernel<D, R>, NW * 32, C::SMEM);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, pod_decode_splitk_kernel<D>, NW * 32, C::SMEM);
   return e == cudaSuccess ? nb : 0;
 }
 
 }  // namespace
 
-int launch_decode(const DecodeParams& p, int grid_splits, cudaStream_t s) {
-  const int D = p.y.D, r = p.y.H_q / p.y.H_kv;
-  if (D == 128) return r <= 4 ? launch_decode_t<128, 4>(p, grid_splits, s) : launch_decode_t<128, 8>(p, grid_splits, s);
-  if (D == 64) return r <= 4 ? launch_decode_t<64, 4>(p, grid_splits, s) : launch_decode_t<64, 8>(p, grid_splits, s);
+int decode_tile_tokens() { return TOK; }
+
+int launch_decode(const CUtensorMap& tmap, const DecodeParams& p, int grid_splits, cudaStream_t s) {
+  if (p.y.D == 128) return launch_decode_t<128>(tmap, p, grid_splits, s);
+  if (p.y.D == 64) return launch_decode_t<64>(tmap, p, grid_splits, s);
   return (int)cudaErrorInvalidValue;
 }
 
@@ -402,9 +378,9 @@ int launch_combine(const DecodeParams& p, cudaStream_t s) {
   return (int)cudaGetLastError();
 }
 
-int decode_resident_ctas_per_sm(int D, int r) {
-  if (D == 128) return r <= 4 ? resident_t<128, 4>() : resident_t<128, 8>();
-  if (D == 64) return r <= 4 ? resident_t<64, 4>() : resident_t<64, 8>();
+int decode_resident_ctas_per_sm(int D) {
+  if (D == 128) return resident_t<128>();
+  if (D == 64) return resident_t<64>();
   return 0;
 }
 
