@@ -2,6 +2,7 @@
 // carving, length bookkeeping, split planning and kernel launches.
 #include <cudaTypedefs.h>
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -43,7 +44,7 @@ int max_splits_for(const pod_config& c) {
 struct Carve {
   std::vector<int64_t> seq_row_base;   // rows
   std::vector<int32_t> seq_cap_d;
-  size_t off_len, off_rowbase, off_capd, off_stash, off_pacc, off_pml, off_err, total;
+  size_t off_len, off_rowbase, off_capd, off_stash, off_pacc, off_pml, off_err, off_tickets, total;
   int64_t total_rows;
   int n_blocks, max_splits;
 };
@@ -74,6 +75,7 @@ bool carve(const pod_config& c, const int32_t* cap, Carve* out) {
   out->off_pacc = off;     off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * c.head_dim * 4);
   out->off_pml = off;      off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * 2 * 4);
   out->off_err = off;      off = align_up(off + 4);
+  out->off_tickets = off;  off = align_up(off + (size_t)c.batch * c.n_kv_heads * 4);
   out->total = off;
   return true;
 }
@@ -91,6 +93,9 @@ struct pod_cache {
   bool dry = false;
   int last_cuda = 0;
   int sm_count = 148, resident = 2;
+  int64_t l2_keep_budget = 0;          // bytes of shared keys worth pinning in L2 (from the L2 size)
+  int force_split_tokens = 0;          // POD_SPLIT_TOKENS > 0 overrides the planner
+  bool two_launch = false;             // POD_COMBINE=separate: split-K and combine as two kernels
   float scale = 0.f;
   Layout y{};
   CUtensorMap tmap{};                  // the region rows of the arena as a [rows][d] bf16 tensor
@@ -139,7 +144,13 @@ DecodePlan plan_decode(pod_cache* c, int layer) {
   for (int b = 0; b < g.batch; ++b) { const int32_t n = c->h_len(layer, b); sum += n; if (n > nmax) nmax = n; }
   if (sum == c->memo_sum && nmax == c->memo_max) return c->memo_plan;
   DecodePlan best{1, 1, 0};
-  if (nmax > 0) {
+  if (nmax > 0 && c->force_split_tokens > 0) {      // POD_SPLIT_TOKENS: tuning experiments
+    int st = c->force_split_tokens;
+    if (st < (nmax + c->cv.max_splits - 1) / c->cv.max_splits) st = (nmax + c->cv.max_splits - 1) / c->cv.max_splits;
+    int64_t ctas = 0;
+    for (int b = 0; b < g.batch; ++b) ctas += ((int64_t)c->h_len(layer, b) + st - 1) / st;
+    best = DecodePlan{st, (nmax + st - 1) / st, (int32_t)(ctas * g.n_kv_heads)};
+  } else if (nmax > 0) {
     const int64_t slots = (int64_t)c->sm_count * c->resident;
     double best_cost = 1e300;
     int last_st = -1;
@@ -237,6 +248,13 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
     return POD_ERR_CUDA;
   }
   c->sm_count = sm; c->resident = res;
+  int l2 = 0;
+  if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, cfg->device) == cudaSuccess) c->l2_keep_budget = (int64_t)l2 * 3 / 4;
+  if (const char* kb = getenv("POD_L2_KEEP_MB")) c->l2_keep_budget = (int64_t)atoi(kb) << 20;
+  const char* comb = getenv("POD_COMBINE");
+  c->two_launch = comb != nullptr && strcmp(comb, "separate") == 0;
+  const char* fst = getenv("POD_SPLIT_TOKENS");
+  c->force_split_tokens = fst ? atoi(fst) : 0;
   *out = c;
   return POD_OK;
 }
@@ -311,9 +329,29 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* str
   p.part_ml = reinterpret_cast<float*>(c->arena + c->cv.off_pml);
   p.out = static_cast<uint16_t*>(out);
   p.err_flag = reinterpret_cast<int32_t*>(c->arena + c->cv.off_err);
+  p.tickets = c->two_launch ? nullptr : reinterpret_cast<int32_t*>(c->arena + c->cv.off_tickets);
   p.layer = layer; p.block = block;
   p.split_tokens = plan.split_tokens; p.max_splits = c->cv.max_splits;
   p.scale_log2 = c->scale * 1.4426950408889634f;
+  {
+    // Shared distant keys are read again by the next layer of the block within the same step.
+    // If the batch's key store of one block fits the L2 budget, ask L2 to keep those lines.
+    const int last_of_block = (low + g.group_size - 1 < g.n_layers - 1) ? low + g.group_size - 1 : g.n_layers - 1;
+    int64_t distk_bytes = 0;
+    const int64_t SW = (int64_t)g.n_sink + g.n_recent;
+    for (int b = 0; b < g.batch; ++b) {
+      const int64_t n = c->h_len(layer, b);
+      distk_bytes += (n > SW ? n - SW : 0) * g.n_kv_heads * g.head_dim * 2;
+    }
+    p.keep_distk = (layer < last_of_block && distk_bytes <= c->l2_keep_budget) ? 1 : 0;
+  }
+  p.by_value = g.batch <= SMALL_BATCH ? 1 : 0;
+  for (int b = 0; b < SMALL_BATCH; ++b) {
+    const bool in = p.by_value && b < g.batch;
+    p.v_len[b] = in ? c->h_len(layer, b) : 0;
+    p.v_cap_d[b] = in ? c->cv.seq_cap_d[b] : 0;
+    p.v_row_base[b] = in ? c->cv.seq_row_base[b] : 0;
+  }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int kernels = 0;
   if (plan.n_ctas > 0) {
@@ -321,9 +359,19 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* str
     if (e != 0) return cuda_fail(c, (cudaError_t)e);
     ++kernels;
   }
-  const int e2 = launch_combine(p, s);
-  if (e2 != 0) return cuda_fail(c, (cudaError_t)e2);
-  ++kernels;
+  if (c->two_launch) {
+    const int e2 = launch_combine(p, s);
+    if (e2 != 0) return cuda_fail(c, (cudaError_t)e2);
+    ++kernels;
+  } else {
+    bool any_empty = false;
+    for (int b = 0; b < g.batch; ++b) any_empty = any_empty || c->h_len(layer, b) == 0;
+    if (any_empty) {                      // no split CTA exists for an empty sequence
+      const int e2 = launch_zero_empty(p, s);
+      if (e2 != 0) return cuda_fail(c, (cudaError_t)e2);
+      ++kernels;
+    }
+  }
   if (lowest) for (int b = 0; b < g.batch; ++b) sl[b] = c->h_len(layer, b);
   c->last_split_tokens = plan.split_tokens; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;
   return POD_OK;

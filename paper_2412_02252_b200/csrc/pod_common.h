@@ -8,6 +8,7 @@
 
 namespace pod {
 
+constexpr int SMALL_BATCH = 8;        // batches up to this size pass per-sequence scalars by value
 constexpr int MAX_SPLITS_CAP = 128;   // upper bound of splits per sequence (partial buffers, combine)
 
 // Physical layout of the arena.  All offsets are in rows; one row is one head's d bf16
@@ -59,8 +60,16 @@ struct DecodeParams {
   float* part_ml;          // [B][H_q][max_splits][2]  (running max in log2 units, sum)
   uint16_t* out;           // [B][H_q][D]
   int32_t* err_flag;
+  int32_t* tickets;        // [B][H_kv] zeroed counters for the in-kernel combine; nullptr = two launches
   int32_t layer, block, split_tokens, max_splits;
   float scale_log2;        // sm_scale * log2(e)
+  // Small batches carry the per-sequence lengths and row offsets by value (the host mirrors the
+  // device lengths exactly), which takes two dependent global loads off every CTA's start-up.
+  int32_t keep_distk;      // 1: later layers of the block re-read the distant keys this step: keep them in L2
+  int32_t by_value;        // 1: use the arrays below instead of len / seq_row_base / seq_cap_d
+  int32_t v_len[SMALL_BATCH];
+  int32_t v_cap_d[SMALL_BATCH];
+  int64_t v_row_base[SMALL_BATCH];
 };
 
 struct DecodePlan {
@@ -73,6 +82,7 @@ struct DecodePlan {
 int launch_write(const WriteParams& p, cudaStream_t s);
 int launch_decode(const CUtensorMap& tmap, const DecodeParams& p, int grid_splits, cudaStream_t s);
 int launch_combine(const DecodeParams& p, cudaStream_t s);
+int launch_zero_empty(const DecodeParams& p, cudaStream_t s);   // zero outputs of empty sequences
 int decode_resident_ctas_per_sm(int D);   // occupancy of the split-K kernel, 0 on error
 int decode_tile_tokens();                 // rows of the TMA box the split-K kernel loads
 

@@ -18,7 +18,13 @@
 // instruction issue at half the memory rate; the tensor-core form needs about a tenth of the
 // instructions and leaves the kernel memory-bound.
 // Warps merge through shared memory; the CTA writes one fp32 partial (acc, max, sum) per
-// query head.  A second kernel merges the partials of a (sequence, head) and rounds to bf16.
+// query head.  The log-sum-exp combine of the partials (the gate of Eq. 2 generalised from two
+// parts to n_splits parts) runs in the same launch: every CTA takes a ticket of its
+// (sequence, KV head) after publishing its partial, and the CTA that draws the last ticket
+// merges all of them and writes the bf16 output.  Nobody waits for anybody, so nothing can hang.
+// A stand-alone combine kernel is kept for callers that want the two-launch form.
+// The kernels are launched with programmatic stream serialization: everything above
+// griddepcontrol.wait (barrier setup) overlaps the tail of the previous kernel in the stream.
 // Every mbarrier wait is bounded; a wait that gives up raises the cache's error flag.
 #include <cuda_bf16.h>
 
@@ -60,11 +66,38 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
 }
 // Tiled TMA load of a [TOK rows][64 bf16] box at (x, y) = (channel, arena row).  x is 0 or
 // 64 elements, i.e. a multiple of 16 bytes as TMA requires.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar) {
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar,
+                                            uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar), "l"(policy)
       : "memory");
+}
+// L2 eviction policies.  Rows that are read once per decode step stream through with
+// evict_first; the block's shared distant keys are kept with evict_last while later layers of
+// the block will read them again in the same step.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ float ld_cg(const float* p) {
+  float v;
+  asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float4 ld_cg4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.cg.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -100,6 +133,7 @@ struct Cfg {
   static constexpr int STAGE_B = 2 * TILE_B;
   static constexpr int WARP_B = NSTAGE * STAGE_B;
   static constexpr int SMEM = NW * WARP_B + NW * NSTAGE * 8 + 1024;   // + slack to align to 1024
+  static_assert(NW * WARP_B >= 8 * MAX_SPLITS_CAP * 4, "combine weights must fit the rings");
   static_assert(WARP_B >= (8 * D + 16) * 4, "merge scratch must fit the warp's ring");
 };
 
@@ -111,10 +145,6 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int r = y.H_q / y.H_kv;   // query heads per KV head (<= 8): rows of the Q operand
 
   const int b = blockIdx.z, kvh = blockIdx.y, split = blockIdx.x;
-  const int n = p.len[b];
-  const int nsplit = min(p.max_splits, (n + p.split_tokens - 1) / p.split_tokens);
-  if (split >= nsplit) return;
-
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);   // swizzle atoms are 1024 B
@@ -122,6 +152,20 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   unsigned char* wbuf = smem + warp * C::WARP_B;
   const uint32_t wbuf_s = smem_u32(wbuf);
   const uint32_t bar0 = smem_u32(smem + NW * C::WARP_B) + warp * NSTAGE * 8;
+  if (lane == 0) {
+    for (int s = 0; s < NSTAGE; ++s) mbar_init(bar0 + s * 8, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  // Everything below reads what earlier kernels of the stream wrote (lengths, cache rows, stash).
+  pdl_wait();
+  pdl_launch_dependents();
+
+  const int n = p.by_value ? p.v_len[b] : p.len[b];
+  const int64_t cap_d = p.by_value ? (int64_t)p.v_cap_d[b] : (int64_t)y.seq_cap_d[b];
+  const int64_t seq_row = p.by_value ? p.v_row_base[b] : y.seq_row_base[b];
+  const int nsplit = min(p.max_splits, (n + p.split_tokens - 1) / p.split_tokens);
+  if (split >= nsplit) return;
 
   // ---- token ranges ---------------------------------------------------------------------
   const int n_p = min(n, y.S + y.W);
@@ -134,12 +178,13 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int nt = ntp + ntd;
 
   // arena rows of this (sequence, layer, head): tile coordinates of the tensor map
-  const int64_t cap_d = y.seq_cap_d[b];
-  const int64_t seq_row = y.seq_row_base[b];
   const int rowKp = (int)(seq_row + prox_row(y, p.layer, 0, kvh));
   const int rowVp = (int)(seq_row + prox_row(y, p.layer, 1, kvh));
   const int rowKd = (int)(seq_row + distk_row(y, p.block, kvh, cap_d));
   const int rowVd = (int)(seq_row + distv_row(y, p.layer, kvh, cap_d));
+
+  const uint64_t pol_stream = policy_evict_first();
+  const uint64_t pol_distk = p.keep_distk ? policy_evict_last() : pol_stream;
 
   auto tile_rows = [&](int t) -> int {
     return t < ntp ? min(TOK, pa1 - (pa0 + t * TOK)) : min(TOK, da1 - (da0 + (t - ntp) * TOK));
@@ -151,17 +196,15 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     const uint32_t bar = bar0 + stage * 8;
     const uint32_t dst = wbuf_s + stage * C::STAGE_B;
     mbar_expect_tx(bar, C::STAGE_B);
+    const uint64_t pol_k = t < ntp ? pol_stream : pol_distk;
 #pragma unroll
     for (int s = 0; s < C::NSUB; ++s) {
-      tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yk, bar);
-      tma_load_2d(dst + C::TILE_B + s * C::SUB_B, &tmap, s * 64, yv, bar);
+      tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yk, bar, pol_k);
+      tma_load_2d(dst + C::TILE_B + s * C::SUB_B, &tmap, s * 64, yv, bar, pol_stream);
     }
   };
 
   if (lane == 0) {
-    for (int s = 0; s < NSTAGE; ++s) mbar_init(bar0 + s * 8, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     for (int t = 0; t < NSTAGE && t < nt; ++t) issue(t);
   }
 
@@ -288,12 +331,93 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     p.part_acc[ph * D + c] = a;
     if (c == 0) { p.part_ml[ph * 2] = M; p.part_ml[ph * 2 + 1] = l; }
   }
+  if (p.tickets == nullptr) return;      // two-launch form: a combine kernel follows
+
+  // ---- ticket: the CTA that publishes the last partial of this (sequence, KV head) combines ----
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int* tk = p.tickets + (int64_t)b * y.H_kv + kvh;
+    const int got = atomicAdd(tk, 1);
+    s_last = (got == nsplit - 1);
+    if (s_last) *tk = 0;                 // ready for the next launch
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  float* s_w = reinterpret_cast<float*>(smem);          // [8][MAX_SPLITS_CAP] split weights
+  for (int h = warp; h < r; h += NW) {
+    const int64_t ph = ((int64_t)b * y.H_q + kvh * r + h) * p.max_splits;
+    float mloc = -INFINITY;
+    for (int s = lane; s < nsplit; s += 32) mloc = fmaxf(mloc, ld_cg(p.part_ml + (ph + s) * 2));
+#pragma unroll
+    for (int o2 = 16; o2 >= 1; o2 >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o2));
+    float lloc = 0.f;
+    for (int s = lane; s < nsplit; s += 32) {
+      const float ms = ld_cg(p.part_ml + (ph + s) * 2);
+      const float wgt = (ms == -INFINITY) ? 0.f : ex2(ms - mloc);
+      s_w[h * MAX_SPLITS_CAP + s] = wgt;
+      lloc += ld_cg(p.part_ml + (ph + s) * 2 + 1) * wgt;
+    }
+#pragma unroll
+    for (int o2 = 16; o2 >= 1; o2 >>= 1) lloc += __shfl_xor_sync(0xffffffffu, lloc, o2);
+    __syncwarp();
+    const float inv = lloc > 0.f ? 1.f / lloc : 0.f;
+    // each lane owns 4 consecutive channels (d = 128) or 2 (d = 64)
+    constexpr int CPL = D / 32;
+    float acc[CPL];
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) acc[j] = 0.f;
+    const float* src = p.part_acc + ph * D + lane * CPL;
+    int s = 0;
+    for (; s + 4 <= nsplit; s += 4) {
+      float v[4][CPL];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if constexpr (CPL == 4) {
+          const float4 x = ld_cg4(src + (int64_t)(s + u) * D);
+          v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
+        } else {
+#pragma unroll
+          for (int j = 0; j < CPL; ++j) v[u][j] = ld_cg(src + (int64_t)(s + u) * D + j);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float wgt = s_w[h * MAX_SPLITS_CAP + s + u];
+#pragma unroll
+        for (int j = 0; j < CPL; ++j) acc[j] += v[u][j] * wgt;
+      }
+    }
+    for (; s < nsplit; ++s) {
+      const float wgt = s_w[h * MAX_SPLITS_CAP + s];
+#pragma unroll
+      for (int j = 0; j < CPL; ++j) acc[j] += ld_cg(src + (int64_t)s * D + j) * wgt;
+    }
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * y.H_q + kvh * r + h) * D + lane * CPL;
+#pragma unroll
+    for (int j = 0; j < CPL; j += 2)
+      *reinterpret_cast<__nv_bfloat162*>(dst + j) = __floats2bfloat162_rn(acc[j] * inv, acc[j + 1] * inv);
+  }
+}
+
+// Outputs of sequences that hold no token are zero (no split CTA exists to write them).
+__global__ void pod_zero_empty_kernel(const DecodeParams p) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int b = blockIdx.x;
+  if (p.len[b] != 0) return;
+  const int per = p.y.H_q * p.y.D;
+  for (int i = threadIdx.x; i < per; i += blockDim.x) p.out[(int64_t)b * per + i] = 0;
 }
 
 // Merge of the split partials of one (sequence, query head): the gate of Eq. 2 generalised
 // from two parts to n_splits parts.  Block = D threads, grid (H_q, B).
 template <int D>
 __global__ void __launch_bounds__(D) pod_combine_kernel(const DecodeParams p) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int hq = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
   const int n = p.len[b];
   const int nsplit = min(p.max_splits, (n + p.split_tokens - 1) / p.split_tokens);
@@ -335,6 +459,16 @@ __global__ void __launch_bounds__(D) pod_combine_kernel(const DecodeParams p) {
   reinterpret_cast<__nv_bfloat16*>(p.out)[((int64_t)b * p.y.H_q + hq) * D + c] = __float2bfloat16_rn(out);
 }
 
+cudaLaunchAttribute g_pdl_attr[1];
+cudaLaunchConfig_t pdl_config(dim3 grid, dim3 block, size_t smem, cudaStream_t s) {
+  g_pdl_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  g_pdl_attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cfg.attrs = g_pdl_attr; cfg.numAttrs = 1;
+  return cfg;
+}
+
 template <int D>
 int launch_decode_t(const CUtensorMap& tmap, const DecodeParams& p, int grid_splits, cudaStream_t s) {
   using C = Cfg<D>;
@@ -345,9 +479,8 @@ int launch_decode_t(const CUtensorMap& tmap, const DecodeParams& p, int grid_spl
     if (e != cudaSuccess) return (int)e;
     configured = true;
   }
-  dim3 grid(grid_splits, p.y.H_kv, p.y.B);
-  pod_decode_splitk_kernel<D><<<grid, NW * 32, C::SMEM, s>>>(tmap, p);
-  return (int)cudaGetLastError();
+  cudaLaunchConfig_t cfg = pdl_config(dim3(grid_splits, p.y.H_kv, p.y.B), dim3(NW * 32), C::SMEM, s);
+  return (int)cudaLaunchKernelEx(&cfg, pod_decode_splitk_kernel<D>, tmap, p);
 }
 
 template <int D>
@@ -372,10 +505,14 @@ int launch_decode(const CUtensorMap& tmap, const DecodeParams& p, int grid_split
 }
 
 int launch_combine(const DecodeParams& p, cudaStream_t s) {
-  dim3 grid(p.y.H_q, p.y.B);
-  if (p.y.D == 128) pod_combine_kernel<128><<<grid, 128, 0, s>>>(p);
-  else pod_combine_kernel<64><<<grid, 64, 0, s>>>(p);
-  return (int)cudaGetLastError();
+  cudaLaunchConfig_t cfg = pdl_config(dim3(p.y.H_q, p.y.B), dim3(p.y.D), 0, s);
+  if (p.y.D == 128) return (int)cudaLaunchKernelEx(&cfg, pod_combine_kernel<128>, p);
+  return (int)cudaLaunchKernelEx(&cfg, pod_combine_kernel<64>, p);
+}
+
+int launch_zero_empty(const DecodeParams& p, cudaStream_t s) {
+  cudaLaunchConfig_t cfg = pdl_config(dim3(p.y.B), dim3(128), 0, s);
+  return (int)cudaLaunchKernelEx(&cfg, pod_zero_empty_kernel, p);
 }
 
 int decode_resident_ctas_per_sm(int D) {

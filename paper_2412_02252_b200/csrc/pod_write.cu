@@ -17,6 +17,10 @@ __global__ void __launch_bounds__(256) pod_write_kernel(const WriteParams p) {
   const Layout& y = p.y;
   const int S = y.S, W = y.W, H = y.H_kv;
 
+  // Launched with programmatic stream serialization: wait for the previous kernel of the
+  // stream (it may still read rows this kernel overwrites) before touching global memory.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const bool batched = (p.seq < 0);
   const int b = batched ? (int)blockIdx.y : p.seq;
   const int n0 = batched ? p.len[b] : p.n0;
@@ -82,9 +86,14 @@ int launch_write(const WriteParams& p, cudaStream_t s) {
     if (blocks > 148 * 16) blocks = 148 * 16;
     grid.x = (unsigned)(blocks < 1 ? 1 : blocks);
   }
-  if (D == 128) pod_write_kernel<128><<<grid, 256, 0, s>>>(p);
-  else pod_write_kernel<64><<<grid, 256, 0, s>>>(p);
-  return (int)cudaGetLastError();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = s;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  if (D == 128) return (int)cudaLaunchKernelEx(&cfg, pod_write_kernel<128>, p);
+  return (int)cudaLaunchKernelEx(&cfg, pod_write_kernel<64>, p);
 }
 
 }  // namespace pod
