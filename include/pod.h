@@ -152,6 +152,42 @@ int pod_cache_last_launch(const pod_cache* c, int32_t* split_tokens, int32_t* n_
 
 const char* pod_strerror(int status);
 
+/* Decode attention without any allocation.  (The paper has no counterpart of this call; it is a
+ * packaging variant of pod_decode_attn for one sequence of ordinary, unshared K/V.)
+ *
+ * Some programs that embed this library cannot obtain device memory at the moment they need
+ * attention: a serving process whose own memory pool has already claimed the whole GPU, so a
+ * raw cudaMalloc would fail; a plug-in running under a host framework that forbids allocating
+ * behind its back; a latency-critical loop that cannot afford the implicit device-wide
+ * synchronisation an allocation or a free may cause.  pod_cache_create needs an arena with
+ * room for the split-K partial results; this call needs none.  Its partials live in a fixed
+ * array inside the library's device image (POD_STATIC_SCRATCH_BYTES, about 2.1 MB, held by
+ * every GPU that loads the library until the process exits).  It calls no cudaMalloc, no
+ * cudaFree and no allocating library routine.
+ *
+ *   kv_device : device bf16 [2][n_kv_heads][capacity][head_dim]: all keys, then all values,
+ *               head-major, token p of head h at row p.  Rows at or past n_tokens (up to the
+ *               next multiple of 16) are loaded and masked, so they must hold finite numbers:
+ *               zero the buffer once when it is created.
+ *   q_device  : device bf16 [n_q_heads][head_dim];  out_device: device bf16, same shape.
+ *   out[h] = softmax_p(sm_scale <q[h], K[p][h / r]>) V[.][h / r] over p < n_tokens (zeros when
+ *   n_tokens == 0); sm_scale 0 means 1/sqrt(head_dim).  Runs on the current device.
+ *
+ * Limits (POD_ERR_CAPACITY beyond them): n_q_heads <= 64, n_tokens <= capacity,
+ * 2 * n_kv_heads * capacity < 2^31.  Shapes as for pod_config (head_dim 64 or 128, at most 8
+ * query heads per KV head); other invalid arguments give POD_ERR_INVALID.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress) and
+ * the driver's tensor-map encoder; make that first call outside any stream capture.  All calls
+ * on a device share the one array, which keeps the previous call's contents; the call clears
+ * the counters that must start at zero on the given stream.  Two calls whose kernels may run at
+ * the same time on one device (different streams, different threads) race on the array: order
+ * them.  Asynchronous on cuda_stream like pod_decode_attn. */
+#define POD_STATIC_SCRATCH_BYTES 2130432
+int pod_dense_decode_attn_static(const void* kv_device, int capacity, int n_tokens,
+                                 const void* q_device, void* out_device, int n_q_heads,
+                                 int n_kv_heads, int head_dim, float sm_scale, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

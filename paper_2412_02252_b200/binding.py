@@ -52,6 +52,8 @@ def _load() -> ctypes.CDLL:
         "pod_cache_last_cuda_error": (c_int, [c_void_p]),
         "pod_cache_last_launch": (c_int, [c_void_p, P(c_int32), P(c_int32), P(c_int32)]),
         "pod_strerror": (c_char_p, [c_int]),
+        "pod_dense_decode_attn_static": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_int,
+                                                 c_int, c_float, c_void_p]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -63,7 +65,7 @@ lib = _load()
 EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_destroy", "pod_cache_write",
            "pod_decode_attn", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
            "pod_cache_read_region", "pod_cache_device_status", "pod_cache_last_cuda_error",
-           "pod_cache_last_launch", "pod_strerror"]
+           "pod_cache_last_launch", "pod_strerror", "pod_dense_decode_attn_static"]
 
 
 class PodError(RuntimeError):
@@ -161,3 +163,14 @@ class PodCache:
         a, b, c = c_int32(), c_int32(), c_int32()
         lib.pod_cache_last_launch(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
         return {"split_tokens": a.value, "n_ctas": b.value, "n_kernels": c.value}
+
+
+def pod_dense_decode_attn_static(kv, capacity: int, n_tokens: int, q, out, n_q_heads: int, n_kv_heads: int,
+                                 head_dim: int, sm_scale: float = 0.0, stream: int = 0) -> int:
+    """Decode attention over a caller-owned dense K/V buffer ``[2][n_kv_heads][capacity][head_dim]``
+    for programs that cannot allocate device memory when they need attention (their pool owns the
+    whole GPU, or an allocation's device-wide synchronisation is unaffordable): the split-K scratch
+    is a fixed array inside the library.  Rows past ``n_tokens`` must hold finite numbers."""
+    return _check(lib.pod_dense_decode_attn_static(_ptr(kv), capacity, n_tokens, _ptr(q), _ptr(out), n_q_heads,
+                                                   n_kv_heads, head_dim, sm_scale, stream),
+                  "pod_dense_decode_attn_static")
