@@ -61,6 +61,26 @@ def _profile_traffic(workload):
     return None
 
 
+def rank_seed(seed, rank):
+    """Every rank decodes its own sequences: disjoint seeds, no data-path collective."""
+    return seed + 1000 * rank
+
+
+def reduce_max(x, dist, device):
+    """Maximum of a per-rank timing over all ranks (identity without a process group)."""
+    if dist is None:
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate(*, ms, steps, layers, batch_per_rank, world):
+    """Whole-job figures from the slowest rank's time for `steps` steps."""
+    return {"us_per_layer_step": ms * 1e3 / (steps * layers * world),
+            "decode_tokens_per_s": world * batch_per_rank / (ms * 1e-3 / steps)}
+
+
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -129,7 +149,7 @@ def run_ours(args):
 
     w = dict(WORKLOADS[args.workload])
     Bn, n, L, G, Hq, Hkv, d, S, W = (w[k] for k in ("B", "n", "L", "G", "Hq", "Hkv", "d", "S", "W"))
-    seed = w["seed"] + 1000 * rank                       # every rank decodes its own sequences
+    seed = rank_seed(w["seed"], rank)
     total_steps = args.warmup + args.steps
     e2e_steps = max(3, min(args.steps, 20))
     extra = 2 * total_steps + 2 * (e2e_steps + 3) + 8     # headroom for every timed pass
@@ -217,12 +237,8 @@ def run_ours(args):
             per = [a.elapsed_time(b) for st in evs for (a, b) in st]
         return ms, per
 
-    def reduce_max(x):
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def rmax(x):
+        return reduce_max(x, dist, dev)
 
     cache = build_cache(G)
     sampler = ClockSampler(local) if rank == 0 else None
@@ -232,7 +248,7 @@ def run_ours(args):
     # ---- headline: K steps, device-resident inputs ------------------------------------------------
     ms, _ = timed(cache, args.steps, args.warmup, 0)
     n_launch = launches[0]
-    ms = reduce_max(ms)
+    ms = rmax(ms)
     # ---- same steps again with an event pair around every decode call (roofline of the kernel) ----
     ms_ev, per = timed(cache, args.steps, 1, total_steps, per_call=True)
     clocks = sampler.stop() if sampler else None
@@ -265,7 +281,7 @@ def run_ours(args):
     for s in range(e2e_steps):
         e2e_step(3 + s)
     torch.cuda.synchronize()
-    e2e_ms = reduce_max((time.perf_counter() - t0) * 1e3)   # wall clock: the host waits for every step's output
+    e2e_ms = rmax((time.perf_counter() - t0) * 1e3)   # wall clock: the host waits for every step's output
     barrier()
     h2d = L * Bn * (2 * Hkv + Hq) * d * 2
     d2h = L * Bn * Hq * d * 2
@@ -291,7 +307,8 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    us_layer = ms * 1e3 / (args.steps * L * world)
+    agg = aggregate(ms=ms, steps=args.steps, layers=L, batch_per_rank=Bn, world=world)
+    us_layer = agg["us_per_layer_step"]
     hbm_peak, peak_kind = _peaks()
     n_avg = n + args.warmup + args.steps / 2.0
     alg_bytes = Bn * 2 * n_avg * Hkv * d * 2              # K row-set + V row-set of every token
@@ -307,7 +324,7 @@ def run_ours(args):
                    "group_size": G, "q_heads": Hq, "kv_heads": Hkv, "head_dim": d, "n_sink": S,
                    "n_recent": W, "l2": "inputs larger than L2 (a step reads %.1f GiB)" % (L * alg_bytes / 2**30),
                    "split_tokens": geo["split_tokens"], "ctas": geo["n_ctas"]},
-        "decode_tokens_per_s": round(world * Bn / (ms * 1e-3 / args.steps), 1),
+        "decode_tokens_per_s": round(agg["decode_tokens_per_s"], 1),
         "hbm_gbs_step": round(L * alg_bytes / (ms * 1e-3 / args.steps) / 1e9, 1),
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": hbm_peak, "unit": "GB/s",
                      "frac": round(achieved / hbm_peak, 4), "traffic": traffic, "peak_kind": peak_kind,
