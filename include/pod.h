@@ -183,7 +183,7 @@ const char* pod_strerror(int status);
  * the counters that must start at zero on the given stream.  Two calls whose kernels may run at
  * the same time on one device (different streams, different threads) race on the array: order
  * them.  Asynchronous on cuda_stream like pod_decode_attn. */
-#define POD_STATIC_SCRATCH_BYTES 2130432
+#define POD_STATIC_SCRATCH_BYTES 2138368
 int pod_dense_decode_attn_static(const void* kv_device, int capacity, int n_tokens,
                                  const void* q_device, void* out_device, int n_q_heads,
                                  int n_kv_heads, int head_dim, float sm_scale, void* cuda_stream);

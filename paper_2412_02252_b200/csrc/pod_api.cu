@@ -38,13 +38,13 @@ int max_splits_for(const pod_config& c) {
   int per = (TARGET_CTAS_FOR_SPLITS + c.batch * c.n_kv_heads - 1) / (c.batch * c.n_kv_heads);
   if (per < 16) per = 16;
   if (per > MAX_SPLITS_CAP) per = MAX_SPLITS_CAP;
-  return per;
+  return (per + 1) & ~1;   // even: the combine's bulk copies move 16-byte multiples
 }
 
 struct Carve {
   std::vector<int64_t> seq_row_base;   // rows
   std::vector<int32_t> seq_cap_d;
-  size_t off_len, off_rowbase, off_capd, off_stash, off_pacc, off_pml, off_err, off_tickets, total;
+  size_t off_len, off_rowbase, off_capd, off_stash, off_pacc, off_pml, off_err, off_sched, total;
   int64_t total_rows;
   int n_blocks, max_splits;
 };
@@ -75,7 +75,7 @@ bool carve(const pod_config& c, const int32_t* cap, Carve* out) {
   out->off_pacc = off;     off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * c.head_dim * 4);
   out->off_pml = off;      off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * 2 * 4);
   out->off_err = off;      off = align_up(off + 4);
-  out->off_tickets = off;  off = align_up(off + (size_t)c.batch * c.n_kv_heads * 4);
+  out->off_sched = off;    off = align_up(off + (size_t)c.batch * c.n_kv_heads * SCHED_STRIDE * 4);
   out->total = off;
   return true;
 }
@@ -95,7 +95,8 @@ struct pod_cache {
   int sm_count = 148, resident = 2;
   int64_t l2_keep_budget = 0;          // bytes of shared keys worth pinning in L2 (from the L2 size)
   int force_split_tokens = 0;          // POD_SPLIT_TOKENS > 0 overrides the planner
-  bool two_launch = false;             // POD_COMBINE=separate: split-K and combine as two kernels
+  int force_chunk_tiles = 0;           // POD_CHUNK_TILES > 0 overrides the tiles per draw
+  int static_eighths = 5;              // POD_STATIC_EIGHTHS: share of a warp's chunks assigned without a draw
   float scale = 0.f;
   Layout y{};
   CUtensorMap tmap{};                  // the region rows of the arena as a [rows][d] bf16 tensor
@@ -251,8 +252,11 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
   int l2 = 0;
   if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, cfg->device) == cudaSuccess) c->l2_keep_budget = (int64_t)l2 * 3 / 4;
   if (const char* kb = getenv("POD_L2_KEEP_MB")) c->l2_keep_budget = (int64_t)atoi(kb) << 20;
-  const char* comb = getenv("POD_COMBINE");
-  c->two_launch = comb != nullptr && strcmp(comb, "separate") == 0;
+  if (const char* ct = getenv("POD_CHUNK_TILES")) c->force_chunk_tiles = atoi(ct);
+  if (const char* se = getenv("POD_STATIC_EIGHTHS")) {
+    const int v = atoi(se);
+    if (v >= 0 && v <= 8) c->static_eighths = v;
+  }
   const char* fst = getenv("POD_SPLIT_TOKENS");
   c->force_split_tokens = fst ? atoi(fst) : 0;
   *out = c;
@@ -329,9 +333,16 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* str
   p.part_ml = reinterpret_cast<float*>(c->arena + c->cv.off_pml);
   p.out = static_cast<uint16_t*>(out);
   p.err_flag = reinterpret_cast<int32_t*>(c->arena + c->cv.off_err);
-  p.tickets = c->two_launch ? nullptr : reinterpret_cast<int32_t*>(c->arena + c->cv.off_tickets);
+  p.sched = reinterpret_cast<int32_t*>(c->arena + c->cv.off_sched);
   p.layer = layer; p.block = block;
   p.split_tokens = plan.split_tokens; p.max_splits = c->cv.max_splits;
+  {
+    // A warp sees about split_tokens / (tile tokens x warps) tiles; it should make a dozen draws.
+    int tch = plan.split_tokens / (decode_tile_tokens() * decode_warps_per_cta() * 16);
+    if (c->force_chunk_tiles > 0) tch = c->force_chunk_tiles;
+    p.tiles_per_chunk = tch < 1 ? 1 : (tch > 16 ? 16 : tch);
+    p.static_eighths = c->static_eighths;
+  }
   p.scale_log2 = c->scale * 1.4426950408889634f;
   {
     // Shared distant keys are read again by the next layer of the block within the same step.
@@ -359,11 +370,7 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* str
     if (e != 0) return cuda_fail(c, (cudaError_t)e);
     ++kernels;
   }
-  if (c->two_launch) {
-    const int e2 = launch_combine(p, s);
-    if (e2 != 0) return cuda_fail(c, (cudaError_t)e2);
-    ++kernels;
-  } else {
+  {
     bool any_empty = false;
     for (int b = 0; b < g.batch; ++b) any_empty = any_empty || c->h_len(layer, b) == 0;
     if (any_empty) {                      // no split CTA exists for an empty sequence

@@ -11,6 +11,24 @@ namespace pod {
 constexpr int SMALL_BATCH = 8;        // batches up to this size pass per-sequence scalars by value
 constexpr int MAX_SPLITS_CAP = 128;   // upper bound of splits per sequence (partial buffers, combine)
 
+// Shape of the split-K decode kernel (compile-time; -D overrides are for tuning builds).
+#ifndef POD_DECODE_WARPS
+#define POD_DECODE_WARPS 4
+#endif
+#ifndef POD_DECODE_STAGES
+#define POD_DECODE_STAGES 3
+#endif
+#ifndef POD_DECODE_CTAS_PER_SM
+#define POD_DECODE_CTAS_PER_SM 2
+#endif
+constexpr int DECODE_WARPS = POD_DECODE_WARPS;              // warps per CTA, each an independent stream
+constexpr int DECODE_STAGES = POD_DECODE_STAGES;            // tiles in flight per warp
+constexpr int DECODE_CTAS_PER_SM = POD_DECODE_CTAS_PER_SM;  // register budget of the kernel
+
+// Scheduling words of one (sequence, KV head): 128 bytes apart so that heads do not share a line.
+constexpr int SCHED_STRIDE = 32;      // int32 per (sequence, KV head)
+constexpr int SCHED_TICKET = 16;      // [0] = chunk counter, [SCHED_TICKET] = finished-CTA tickets
+
 // Physical layout of the arena.  All offsets are in rows; one row is one head's d bf16
 // values (128 B at d = 64, 256 B at d = 128), so every region base is 128-byte aligned.
 //
@@ -60,8 +78,10 @@ struct DecodeParams {
   float* part_ml;          // [B][H_q][max_splits][2]  (running max in log2 units, sum)
   uint16_t* out;           // [B][H_q][D]
   int32_t* err_flag;
-  int32_t* tickets;        // [B][H_kv] zeroed counters for the in-kernel combine; nullptr = two launches
+  int32_t* sched;          // [B][H_kv][SCHED_STRIDE] zeroed chunk counters and tickets (the kernel re-zeroes them)
   int32_t layer, block, split_tokens, max_splits;
+  int32_t tiles_per_chunk; // tiles a warp takes per draw from the head's chunk counter
+  int32_t static_eighths;  // eighths of a warp's fair share of chunks that are assigned without a draw
   float scale_log2;        // sm_scale * log2(e)
   // Small batches carry the per-sequence lengths and row offsets by value (the host mirrors the
   // device lengths exactly), which takes two dependent global loads off every CTA's start-up.
@@ -81,9 +101,9 @@ struct DecodePlan {
 // launchers (defined in the .cu files); return a cudaError_t as int
 int launch_write(const WriteParams& p, cudaStream_t s);
 int launch_decode(const CUtensorMap& tmap, const DecodeParams& p, int grid_splits, cudaStream_t s);
-int launch_combine(const DecodeParams& p, cudaStream_t s);
 int launch_zero_empty(const DecodeParams& p, cudaStream_t s);   // zero outputs of empty sequences
 int decode_resident_ctas_per_sm(int D);   // occupancy of the split-K kernel, 0 on error
 int decode_tile_tokens();                 // rows of the TMA box the split-K kernel loads
+int decode_warps_per_cta();
 
 }  // namespace pod

@@ -1,31 +1,36 @@
-// Split-K decode attention over the PoD layout, and the log-sum-exp combine.
+// Split-K decode attention over the PoD layout with the log-sum-exp combine in the same launch.
 //
-// Grid (split, KV head, sequence).  A CTA owns a contiguous range of the sequence's tokens in
-// "virtual" order -- proximal rows first (sink, then ring slots), distant rows after -- and
-// its warps subdivide that range.  Each warp is an independent flash-decoding stream:
-//   * lane 0 stages tiles of 16 K rows and 16 V rows into the warp's private shared-memory
-//     ring with tiled TMA loads (one tensor map views the whole arena as [rows][d]; 128-byte
+// Grid (split, KV head, sequence); the CTAs of one (sequence, KV head) share that head's tokens.
+// The tokens are cut into tiles of 16 in "virtual" order -- proximal rows first (sink, then
+// ring slots), distant rows after -- and tiles into chunks of a few tiles.  Each warp is an
+// independent flash-decoding stream over chunks:
+//   * the first chunks of a warp are fixed (round-robin over the head's warps); the rest are
+//     drawn from a per-head counter with atomicAdd, so warps on SMs that get less memory
+//     bandwidth simply take fewer chunks and all warps of a head finish together.  The draw for
+//     the next chunk is issued one chunk ahead and its result is only read when that chunk is
+//     entered, so the round trip hides behind the loads already in flight;
+//   * lane 0 stages a tile (16 K rows + 16 V rows) into the warp's private shared-memory ring
+//     with tiled TMA loads (one tensor map views the whole arena as [rows][d]; 128-byte
 //     swizzle, no multicast) that complete on an mbarrier;
-//   * logits: S[16 x 16] = Q[16 x d] K^T with mma.sync m16n8k16 (bf16 in, fp32 out).  The rows
-//     of Q are the r <= 8 query heads of the KV head, zero-padded to 16; K fragments come from
-//     ldmatrix on the swizzled tile, so the bf16 data is never unpacked by ALU instructions;
-//   * one online softmax in base 2 runs over proximal and distant rows alike: at the boundary
-//     only the Q fragments (own query for proximal rows, the block's lowest-layer query for
-//     distant rows) and the tile coordinates change;
-//   * values: O[16 x d] += P[16 x 16] V[16 x d], P rounded to bf16 in the accumulator-to-A
-//     register layout, V fragments from ldmatrix.trans.
-// An earlier CUDA-core version of this kernel (packed fp32 FMAs on unpacked bf16) was bound by
-// instruction issue at half the memory rate; the tensor-core form needs about a tenth of the
-// instructions and leaves the kernel memory-bound.
-// Warps merge through shared memory; the CTA writes one fp32 partial (acc, max, sum) per
-// query head.  The log-sum-exp combine of the partials (the gate of Eq. 2 generalised from two
-// parts to n_splits parts) runs in the same launch: every CTA takes a ticket of its
-// (sequence, KV head) after publishing its partial, and the CTA that draws the last ticket
-// merges all of them and writes the bf16 output.  Nobody waits for anybody, so nothing can hang.
-// A stand-alone combine kernel is kept for callers that want the two-launch form.
+//   * when a tile lands the warp pulls all of its K and V fragments into registers with
+//     ldmatrix and refills the stage at once, so the memory pipeline never waits for the
+//     arithmetic;
+//   * logits: S[16 x 16] = Q[16 x d] K^T with mma.sync m16n8k16 (bf16 in, fp32 out); the rows of Q
+//     are the r <= 8 query heads of the KV head, zero-padded to 16.  One online softmax in base
+//     2 runs over proximal and distant tiles alike: proximal tiles use the layer's own query,
+//     distant tiles the stashed query of the block's lowest layer (Eq. 1 rows 1 and 3);
+//   * values: O^T[d x 8] += V^T[d x 16] P^T[16 x 8]: the channels are the M dimension, so no
+//     accumulator row is padding; the exponentials in the accumulator layout of S are exactly
+//     the B fragments, V^T fragments come from ldmatrix.trans.
+// Warps merge through shared memory; the CTA writes one fp32 partial (acc, max, sum) per query
+// head, takes a ticket of its (sequence, KV head), and the CTA that draws the last ticket merges
+// all partials (the gate of Eq. 2 generalised from two parts to n_splits parts): it pulls them
+// into shared memory with bulk async copies, so the merge costs one memory round trip instead of
+// one per split.  Nobody waits for anybody, so nothing can hang; every mbarrier wait is
+// bounded and a wait that gives up raises the cache's error flag.
 // The kernels are launched with programmatic stream serialization: everything above
-// griddepcontrol.wait (barrier setup) overlaps the tail of the previous kernel in the stream.
-// Every mbarrier wait is bounded; a wait that gives up raises the cache's error flag.
+// griddepcontrol.wait (barrier setup, policies) overlaps the tail of the previous kernel in the
+// stream.
 #include <cuda_bf16.h>
 
 #include "pod_common.h"
@@ -34,10 +39,7 @@ namespace pod {
 
 namespace {
 
-constexpr int NW = 4;            // warps per CTA
-constexpr int NSTAGE = 3;        // stages of each warp's ring
 constexpr int TOK = 16;          // tokens per tile (one mma k-step of P V)
-constexpr int CTAS_PER_SM = 2;
 constexpr uint32_t WAIT_LIMIT = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -89,15 +91,12 @@ __device__ __forceinline__ uint64_t policy_evict_last() {
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ float ld_cg(const float* p) {
-  float v;
-  asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
-  return v;
-}
-__device__ __forceinline__ float4 ld_cg4(const float* p) {
-  float4 v;
-  asm volatile("ld.global.cg.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
-  return v;
+__device__ __forceinline__ void fence_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+// Untiled bulk copy global -> shared; both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -125,22 +124,32 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+
 template <int D>
 struct Cfg {
+  static constexpr int NW = DECODE_WARPS;
+  static constexpr int NSTAGE = DECODE_STAGES;
   static constexpr int NSUB = D / 64;                 // 128-byte wide sub-tiles per row
   static constexpr int SUB_B = TOK * 128;             // bytes of one sub-tile (1024-byte multiple)
   static constexpr int TILE_B = NSUB * SUB_B;         // bytes of one K (or V) tile
   static constexpr int STAGE_B = 2 * TILE_B;
   static constexpr int WARP_B = NSTAGE * STAGE_B;
-  static constexpr int SMEM = NW * WARP_B + NW * NSTAGE * 8 + 1024;   // + slack to align to 1024
-  static_assert(NW * WARP_B >= 8 * MAX_SPLITS_CAP * 4, "combine weights must fit the rings");
+  static constexpr int RING_B = NW * WARP_B;
+  static constexpr int N_BARS = NW * NSTAGE + 1;      // one per stage, one for the combine
+  static constexpr int SMEM = RING_B + N_BARS * 8 + 1024;   // + slack to align to 1024
+  // the combine reuses the rings: split weights, (max, sum) pairs, then partial rows
+  static constexpr int CW_B = 8 * MAX_SPLITS_CAP * 4;
+  static constexpr int CML_B = 8 * MAX_SPLITS_CAP * 8;
+  static constexpr int CROWS = (RING_B - CW_B - CML_B) / (D * 4);   // partial rows per round
+  static_assert(CROWS >= 8, "the rings must hold a few partial rows for the combine");
   static_assert(WARP_B >= (8 * D + 16) * 4, "merge scratch must fit the warp's ring");
 };
 
 template <int D>
-__global__ void __launch_bounds__(NW * 32, CTAS_PER_SM)
+__global__ void __launch_bounds__(DECODE_WARPS * 32, DECODE_CTAS_PER_SM)
 pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeParams p) {
   using C = Cfg<D>;
+  constexpr int NW = C::NW, NSTAGE = C::NSTAGE;
   const Layout& y = p.y;
   const int r = y.H_q / y.H_kv;   // query heads per KV head (<= 8): rows of the Q operand
 
@@ -151,31 +160,45 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   unsigned char* wbuf = smem + warp * C::WARP_B;
   const uint32_t wbuf_s = smem_u32(wbuf);
-  const uint32_t bar0 = smem_u32(smem + NW * C::WARP_B) + warp * NSTAGE * 8;
+  const uint32_t bar0 = smem_u32(smem + C::RING_B) + warp * NSTAGE * 8;
+  const uint32_t cbar = smem_u32(smem + C::RING_B) + NW * NSTAGE * 8;
   if (lane == 0) {
     for (int s = 0; s < NSTAGE; ++s) mbar_init(bar0 + s * 8, 1);
+    if (warp == 0) mbar_init(cbar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
   }
-  // Everything below reads what earlier kernels of the stream wrote (lengths, cache rows, stash).
+  const int bv = b < SMALL_BATCH ? b : 0;
+  int n = p.v_len[bv];
+  int64_t cap_d = p.v_cap_d[bv];
+  int64_t seq_row = p.v_row_base[bv];
+  const uint64_t pol_stream = policy_evict_first();
+  const uint64_t pol_distk = p.keep_distk ? policy_evict_last() : pol_stream;
+
+  // Everything below reads what earlier kernels of the stream wrote (lengths, cache rows, stash,
+  // counters).
   pdl_wait();
   pdl_launch_dependents();
-
-  const int n = p.by_value ? p.v_len[b] : p.len[b];
-  const int64_t cap_d = p.by_value ? (int64_t)p.v_cap_d[b] : (int64_t)y.seq_cap_d[b];
-  const int64_t seq_row = p.by_value ? p.v_row_base[b] : y.seq_row_base[b];
+  if (!p.by_value) {
+    n = p.len[b];
+    cap_d = y.seq_cap_d[b];
+    seq_row = y.seq_row_base[b];
+  }
   const int nsplit = min(p.max_splits, (n + p.split_tokens - 1) / p.split_tokens);
   if (split >= nsplit) return;
 
-  // ---- token ranges ---------------------------------------------------------------------
-  const int n_p = min(n, y.S + y.W);
-  const int c0 = (int)((int64_t)n * split / nsplit), c1 = (int)((int64_t)n * (split + 1) / nsplit);
-  const int w0 = c0 + (int)((int64_t)(c1 - c0) * warp / NW);
-  const int w1 = c0 + (int)((int64_t)(c1 - c0) * (warp + 1) / NW);
-  const int pa0 = min(w0, n_p), pa1 = min(w1, n_p);              // proximal rows [pa0, pa1)
-  const int da0 = max(w0, n_p) - n_p, da1 = max(w1, n_p) - n_p;  // distant rows  [da0, da1)
-  const int ntp = (pa1 - pa0 + TOK - 1) / TOK, ntd = (da1 - da0 + TOK - 1) / TOK;
-  const int nt = ntp + ntd;
+  // ---- tiles and chunks of this (sequence, KV head) -----------------------------------------
+  const int n_p = min(n, y.S + y.W), n_d = n - n_p;
+  const int ntp = (n_p + TOK - 1) / TOK, ntd = (n_d + TOK - 1) / TOK;
+  const int ntiles = ntp + ntd;
+  const int tch = p.tiles_per_chunk;
+  const int nwh = nsplit * NW;                    // warps working on this head
+  const int gw = split * NW + warp;               // this warp's index among them
+  const int nchunks = (ntiles + tch - 1) / tch;
+  const int k_static = (nchunks / nwh) * p.static_eighths / 8;   // chunks per warp taken without a draw
+  const int dyn_base = k_static * nwh;            // first chunk id that is drawn
+  int* sched = p.sched + ((int64_t)b * y.H_kv + kvh) * SCHED_STRIDE;
 
   // arena rows of this (sequence, layer, head): tile coordinates of the tensor map
   const int rowKp = (int)(seq_row + prox_row(y, p.layer, 0, kvh));
@@ -183,20 +206,44 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int rowKd = (int)(seq_row + distk_row(y, p.block, kvh, cap_d));
   const int rowVd = (int)(seq_row + distv_row(y, p.layer, kvh, cap_d));
 
-  const uint64_t pol_stream = policy_evict_first();
-  const uint64_t pol_distk = p.keep_distk ? policy_evict_last() : pol_stream;
-
-  auto tile_rows = [&](int t) -> int {
-    return t < ntp ? min(TOK, pa1 - (pa0 + t * TOK)) : min(TOK, da1 - (da0 + (t - ntp) * TOK));
+  // ---- the warp's walk over its chunks (all values uniform across the warp) -----------------
+  unsigned drawn = 0;                             // lane 0: result of the draw issued one chunk ahead
+  if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+  int c_id, c_t = 0, c_j = 0;
+  bool walk_done = false;
+  if (k_static > 0) {
+    c_id = gw;
+  } else {
+    c_id = dyn_base + (int)__shfl_sync(0xffffffffu, drawn, 0);
+    if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+  }
+  auto next_tile = [&]() -> int {                 // virtual tile index, or -1 when the head is used up
+    if (walk_done) return -1;
+    if (c_t == tch) {
+      c_t = 0;
+      ++c_j;
+      if (c_j < k_static) {
+        c_id = gw + c_j * nwh;
+      } else {
+        c_id = dyn_base + (int)__shfl_sync(0xffffffffu, drawn, 0);
+        if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+      }
+    }
+    const int64_t vt = (int64_t)c_id * tch + c_t;
+    ++c_t;
+    if (vt >= ntiles) { walk_done = true; return -1; }
+    return (int)vt;
   };
-  auto issue = [&](int t) {   // lane 0 only.  Rows past the piece are other (finite) cache rows
-    const int stage = t % NSTAGE;   // or zero fill past the arena; their logits are masked.
-    const int yk = t < ntp ? rowKp + pa0 + t * TOK : rowKd + da0 + (t - ntp) * TOK;
-    const int yv = t < ntp ? rowVp + pa0 + t * TOK : rowVd + da0 + (t - ntp) * TOK;
+  // lane 0 only.  Rows past the segment are other (finite) cache rows, or zero fill past the
+  // arena; their logits are masked.  `dep` is zero; it carries a register dependency.
+  auto issue = [&](int vt, int stage, int dep) {
+    const bool dist = vt >= ntp;
+    const int yk = (dist ? rowKd + (vt - ntp) * TOK : rowKp + vt * TOK) + dep;
+    const int yv = dist ? rowVd + (vt - ntp) * TOK : rowVp + vt * TOK;
     const uint32_t bar = bar0 + stage * 8;
     const uint32_t dst = wbuf_s + stage * C::STAGE_B;
     mbar_expect_tx(bar, C::STAGE_B);
-    const uint64_t pol_k = t < ntp ? pol_stream : pol_distk;
+    const uint64_t pol_k = dist ? pol_distk : pol_stream;
 #pragma unroll
     for (int s = 0; s < C::NSUB; ++s) {
       tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yk, bar, pol_k);
@@ -204,8 +251,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     }
   };
 
-  if (lane == 0) {
-    for (int t = 0; t < NSTAGE && t < nt; ++t) issue(t);
+  int vt_q[NSTAGE];                               // tile held by each stage, -1 = none
+#pragma unroll
+  for (int s = 0; s < NSTAGE; ++s) {
+    vt_q[s] = next_tile();
+    if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, 0);
   }
 
   // a lowest layer saves its query for the other layers of the block
@@ -215,100 +265,139 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       *reinterpret_cast<uint4*>(p.stash + o) = *reinterpret_cast<const uint4*>(p.q + o);
     }
   }
-  __syncwarp();
 
   // ---- per-lane state -------------------------------------------------------------------
-  const int qrow = lane >> 2;          // query head (row of S and O) owned by this lane's quad
+  const int qrow = lane >> 2;          // query head (row of S) owned by this lane's quad
   const int qcol = (lane & 3) * 2;     // first of the two columns this lane holds in a fragment
-  uint32_t qa[D / 16][2];              // A fragments of Q: rows 0..7 only (rows 8..15 are zero)
-  float o[D / 8][4];                   // O accumulators; [.][2], [.][3] belong to the zero rows
-#pragma unroll
-  for (int c = 0; c < D / 8; ++c) { o[c][0] = o[c][1] = o[c][2] = o[c][3] = 0.f; }
-  float m_row = -INFINITY, l_row = 0.f;
-  bool failed = false;
-
-  auto load_q = [&](const uint16_t* qsrc) {
-    const uint16_t* base = qsrc + ((int64_t)b * y.H_q + kvh * r + qrow) * D + qcol;
+  uint32_t qp[D / 16][2], qd[D / 16][2];   // A fragments of Q (rows 0..7; rows 8..15 are zero):
+  {                                        // own query (proximal tiles), lowest layer's (distant)
+    const int64_t qo = ((int64_t)b * y.H_q + kvh * r + qrow) * D + qcol;
 #pragma unroll
     for (int kk = 0; kk < D / 16; ++kk) {
-      qa[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(base + kk * 16) : 0u;
-      qa[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(base + kk * 16 + 8) : 0u;
+      qp[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(p.q + qo + kk * 16) : 0u;
+      qp[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(p.q + qo + kk * 16 + 8) : 0u;
+      qd[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(p.q_low + qo + kk * 16) : 0u;
+      qd[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(p.q_low + qo + kk * 16 + 8) : 0u;
     }
-  };
+  }
+  // O^T accumulators: ot[cb][0], [1] = channel cb*16 + qrow of heads qcol, qcol + 1;
+  // ot[cb][2], [3] = channel cb*16 + 8 + qrow of the same heads
+  float ot[D / 16][4];
+#pragma unroll
+  for (int cb = 0; cb < D / 16; ++cb) { ot[cb][0] = ot[cb][1] = ot[cb][2] = ot[cb][3] = 0.f; }
+  float m_row = -INFINITY, l_row = 0.f;   // running max (log2 units) and sum of head qrow
+  bool failed = false;
+  uint32_t round = 0;                     // stage s holds its (round)-th tile: barrier parity round & 1
+  int fail_stage = 0;
 
   // ldmatrix lane addressing inside a [TOK][128 B] sub-tile with the 128-byte swizzle:
   // 16-byte chunk c of row t lives at t * 128 + ((c ^ (t & 7)) << 4).
   const int lm = lane >> 3, lr = lane & 7;
   // K (non-transposed): matrices (tokens 0-7, chunk 2kk), (0-7, 2kk+1), (8-15, 2kk), (8-15, 2kk+1)
   const int k_tok = (lm >> 1) * 8 + lr, k_chunk = lm & 1;
-  // V (transposed): matrices (tokens 0-7, chunk c), (8-15, c), (0-7, c+1), (8-15, c+1)
-  const int v_tok = (lm & 1) * 8 + lr, v_chunk = lm >> 1;
+  // V (transposed): matrices (tokens 0-7, chunk 2cb), (0-7, 2cb+1), (8-15, 2cb), (8-15, 2cb+1):
+  // the A fragments a0..a3 of V^T [16 channels x 16 tokens]
+  const int v_tok = (lm >> 1) * 8 + lr, v_chunk = lm & 1;
 
-  int t = 0;
-  for (; t < nt; ++t) {
-    if (t == 0 || t == ntp) load_q(t < ntp ? p.q : p.q_low);
-    const int stage = t % NSTAGE;
-    if (!__all_sync(0xffffffffu, mbar_wait(bar0 + stage * 8, (t / NSTAGE) & 1))) { failed = true; break; }
-    const int cnt = tile_rows(t);
-    const uint32_t ks = wbuf_s + stage * C::STAGE_B;
-    const uint32_t vs = ks + C::TILE_B;
+  for (bool more = true; more && !failed; ++round) {
+#pragma unroll
+    for (int s = 0; s < NSTAGE; ++s) {
+      if (!more || failed) continue;
+      const int vt = vt_q[s];
+      if (vt < 0) { more = false; continue; }
+      if (!__all_sync(0xffffffffu, mbar_wait(bar0 + s * 8, round & 1))) { failed = true; fail_stage = s; continue; }
+      const bool dist = vt >= ntp;
+      const int cnt = dist ? min(TOK, n_d - (vt - ntp) * TOK) : min(TOK, n_p - vt * TOK);
+      const uint32_t ks = wbuf_s + s * C::STAGE_B;
+      const uint32_t vs = ks + C::TILE_B;
 
-    // ---- S = Q K^T ------------------------------------------------------------------------
-    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+      // ---- the whole tile into registers, then hand the stage back --------------------------
+      uint32_t kf[D / 16][4], vf[D / 16][4];
 #pragma unroll
-    for (int kk = 0; kk < D / 16; ++kk) {
-      const int chunk = 2 * kk + k_chunk;          // 16-byte chunk of the row
-      uint32_t bfr[4];
-      ldsm4(ks + (chunk >> 3) * C::SUB_B + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), bfr);
-      mma16816(s0, qa[kk][0], 0u, qa[kk][1], 0u, bfr[0], bfr[1]);
-      mma16816(s1, qa[kk][0], 0u, qa[kk][1], 0u, bfr[2], bfr[3]);
-    }
-    // ---- online softmax (base 2) over this lane's row -----------------------------------------
-    float a00 = (qcol < cnt) ? s0[0] * p.scale_log2 : -INFINITY;
-    float a01 = (qcol + 1 < cnt) ? s0[1] * p.scale_log2 : -INFINITY;
-    float a10 = (qcol + 8 < cnt) ? s1[0] * p.scale_log2 : -INFINITY;
-    float a11 = (qcol + 9 < cnt) ? s1[1] * p.scale_log2 : -INFINITY;
-    float mx = fmaxf(fmaxf(a00, a01), fmaxf(a10, a11));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-    if (__any_sync(0xffffffffu, mx > m_row)) {
-      const float m_new = fmaxf(m_row, mx);
-      const float alpha = ex2(m_row - m_new);       // 0 on the first tile, 1 if unchanged
-      m_row = m_new;
-      l_row *= alpha;
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const int chunk = 2 * kk + k_chunk;          // 16-byte chunk of the row
+        ldsm4(ks + (chunk >> 3) * C::SUB_B + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), kf[kk]);
+      }
 #pragma unroll
-      for (int c = 0; c < D / 8; ++c) { o[c][0] *= alpha; o[c][1] *= alpha; }
-    }
-    a00 = ex2(a00 - m_row); a01 = ex2(a01 - m_row); a10 = ex2(a10 - m_row); a11 = ex2(a11 - m_row);
-    l_row += (a00 + a01) + (a10 + a11);
-    const uint32_t pa0 = pack_bf16(a00, a01), pa2 = pack_bf16(a10, a11);
-    // ---- O += P V ---------------------------------------------------------------------------
+      for (int cb = 0; cb < D / 16; ++cb) {
+        const int chunk = 2 * cb + v_chunk;
+        ldsm4_t(vs + (chunk >> 3) * C::SUB_B + v_tok * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), vf[cb]);
+      }
+      // The refill must not start before the last fragment load has returned (shared-memory
+      // loads of a warp return in order): its row coordinate depends on that load's result.
+      int dep;
+      asm volatile("and.b32 %0, %1, 0;" : "=r"(dep) : "r"(vf[D / 16 - 1][3]));
+      __syncwarp();
+      vt_q[s] = next_tile();
+      if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, dep);
+
+      // ---- S = Q K^T (two accumulation chains per token half) -------------------------------
+      float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+      float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int c = 0; c < D / 8; c += 2) {
-      const int chunk = c + v_chunk;
-      uint32_t bfr[4];
-      ldsm4_t(vs + (chunk >> 3) * C::SUB_B + v_tok * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), bfr);
-      mma16816(o[c], pa0, 0u, pa2, 0u, bfr[0], bfr[1]);
-      mma16816(o[c + 1], pa0, 0u, pa2, 0u, bfr[2], bfr[3]);
+      for (int kk = 0; kk < D / 16; kk += 2) {
+        const uint32_t a0 = dist ? qd[kk][0] : qp[kk][0], a2 = dist ? qd[kk][1] : qp[kk][1];
+        const uint32_t c0 = dist ? qd[kk + 1][0] : qp[kk + 1][0], c2 = dist ? qd[kk + 1][1] : qp[kk + 1][1];
+        mma16816(s0, a0, 0u, a2, 0u, kf[kk][0], kf[kk][1]);
+        mma16816(s1, a0, 0u, a2, 0u, kf[kk][2], kf[kk][3]);
+        mma16816(t0, c0, 0u, c2, 0u, kf[kk + 1][0], kf[kk + 1][1]);
+        mma16816(t1, c0, 0u, c2, 0u, kf[kk + 1][2], kf[kk + 1][3]);
+      }
+      // ---- online softmax (base 2) over this lane's row --------------------------------------
+      float a00 = (qcol < cnt) ? (s0[0] + t0[0]) * p.scale_log2 : -INFINITY;
+      float a01 = (qcol + 1 < cnt) ? (s0[1] + t0[1]) * p.scale_log2 : -INFINITY;
+      float a10 = (qcol + 8 < cnt) ? (s1[0] + t1[0]) * p.scale_log2 : -INFINITY;
+      float a11 = (qcol + 9 < cnt) ? (s1[1] + t1[1]) * p.scale_log2 : -INFINITY;
+      float mx = fmaxf(fmaxf(a00, a01), fmaxf(a10, a11));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      if (__any_sync(0xffffffffu, mx > m_row)) {
+        const float m_new = fmaxf(m_row, mx);
+        const float alpha = ex2(m_row - m_new);       // 0 on the first tile, 1 if unchanged
+        m_row = m_new;
+        l_row *= alpha;
+        // the accumulators of this lane belong to heads qcol and qcol + 1
+        const float al0 = __shfl_sync(0xffffffffu, alpha, qcol * 4);
+        const float al1 = __shfl_sync(0xffffffffu, alpha, qcol * 4 + 4);
+#pragma unroll
+        for (int cb = 0; cb < D / 16; ++cb) { ot[cb][0] *= al0; ot[cb][1] *= al1; ot[cb][2] *= al0; ot[cb][3] *= al1; }
+      }
+      a00 = ex2(a00 - m_row); a01 = ex2(a01 - m_row); a10 = ex2(a10 - m_row); a11 = ex2(a11 - m_row);
+      l_row += (a00 + a01) + (a10 + a11);
+      const uint32_t pb0 = pack_bf16(a00, a01), pb1 = pack_bf16(a10, a11);
+      // ---- O^T += V^T P^T ----------------------------------------------------------------------
+#pragma unroll
+      for (int cb = 0; cb < D / 16; ++cb) mma16816(ot[cb], vf[cb][0], vf[cb][1], vf[cb][2], vf[cb][3], pb0, pb1);
     }
-    __syncwarp();                          // all lanes are done reading this stage
-    if (lane == 0 && t + NSTAGE < nt) issue(t + NSTAGE);
   }
 
   if (failed) {
     if (lane == 0) atomicExch(p.err_flag, 1);
-    // drain the copies this warp still has in flight before its shared memory is reused
-    for (int u = t; u < nt && u < t + NSTAGE; ++u) mbar_wait(bar0 + (u % NSTAGE) * 8, (u / NSTAGE) & 1);
+    // `round` was advanced once after the failing pass.  Drain the copies this warp still has in
+    // flight before its shared memory is reused: stages before the failing one were refilled in
+    // that pass, the others still hold that pass's tile.
+    const uint32_t fr = round - 1;
+#pragma unroll
+    for (int s = 0; s < NSTAGE; ++s)
+      if (vt_q[s] >= 0) mbar_wait(bar0 + s * 8, (s < fail_stage ? fr + 1 : fr) & 1);
   }
 
   // ---- merge the warps of the CTA -------------------------------------------------------------
   l_row += __shfl_xor_sync(0xffffffffu, l_row, 1);
   l_row += __shfl_xor_sync(0xffffffffu, l_row, 2);
   __syncwarp();
-  float* mine = reinterpret_cast<float*>(wbuf);    // [8][D] acc, then [8] max, [8] sum
+  float* mine = reinterpret_cast<float*>(wbuf);    // [8 heads][D] acc, then [8] max, [8] sum
+  if (qcol < r) {
 #pragma unroll
-  for (int c = 0; c < D / 8; ++c)
-    *reinterpret_cast<float2*>(mine + qrow * D + c * 8 + qcol) = make_float2(o[c][0], o[c][1]);
+    for (int cb = 0; cb < D / 16; ++cb) {
+      mine[qcol * D + cb * 16 + qrow] = ot[cb][0];
+      mine[qcol * D + cb * 16 + 8 + qrow] = ot[cb][2];
+      if (qcol + 1 < r) {
+        mine[(qcol + 1) * D + cb * 16 + qrow] = ot[cb][1];
+        mine[(qcol + 1) * D + cb * 16 + 8 + qrow] = ot[cb][3];
+      }
+    }
+  }
   if ((lane & 3) == 0) { mine[8 * D + qrow] = m_row; mine[8 * D + 8 + qrow] = l_row; }
   __syncthreads();
 
@@ -331,74 +420,110 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     p.part_acc[ph * D + c] = a;
     if (c == 0) { p.part_ml[ph * 2] = M; p.part_ml[ph * 2 + 1] = l; }
   }
-  if (p.tickets == nullptr) return;      // two-launch form: a combine kernel follows
 
   // ---- ticket: the CTA that publishes the last partial of this (sequence, KV head) combines ----
   __shared__ int s_last;
+  __shared__ float s_inv[8];
   __threadfence();
+  fence_async_global();                  // the partials are read back through the async proxy
   __syncthreads();
   if (threadIdx.x == 0) {
-    int* tk = p.tickets + (int64_t)b * y.H_kv + kvh;
-    const int got = atomicAdd(tk, 1);
+    const int got = atomicAdd(sched + SCHED_TICKET, 1);
     s_last = (got == nsplit - 1);
-    if (s_last) *tk = 0;                 // ready for the next launch
+    if (s_last) { sched[SCHED_TICKET] = 0; sched[0] = 0; }   // ready for the next launch
   }
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  float* s_w = reinterpret_cast<float*>(smem);          // [8][MAX_SPLITS_CAP] split weights
-  for (int h = warp; h < r; h += NW) {
-    const int64_t ph = ((int64_t)b * y.H_q + kvh * r + h) * p.max_splits;
-    float mloc = -INFINITY;
-    for (int s = lane; s < nsplit; s += 32) mloc = fmaxf(mloc, ld_cg(p.part_ml + (ph + s) * 2));
+
+  float* s_w = reinterpret_cast<float*>(smem);                           // [8][MAX_SPLITS_CAP] split weights
+  float* s_ml = reinterpret_cast<float*>(smem + C::CW_B);                // [r][max_splits][2]
+  float* s_rows = reinterpret_cast<float*>(smem + C::CW_B + C::CML_B);   // partial rows of one round
+  const int64_t ph0 = ((int64_t)b * y.H_q + kvh * r) * p.max_splits;     // partial row of (head 0, split 0)
+  uint32_t cphase = 0;
+  if (threadIdx.x == 0) {
+    fence_async_global();
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    const uint32_t bytes = (uint32_t)p.max_splits * 8u;
+    mbar_expect_tx(cbar, bytes * r);
+    for (int h = 0; h < r; ++h)
+      bulk_load(smem_u32(s_ml + h * p.max_splits * 2), p.part_ml + (ph0 + (int64_t)h * p.max_splits) * 2, bytes, cbar);
+  }
+  bool cfail = !mbar_wait(cbar, cphase & 1);
+  ++cphase;
+  if (!cfail) {
+    for (int h = warp; h < r; h += NW) {
+      const float* ml = s_ml + h * p.max_splits * 2;
+      float mloc = -INFINITY;
+      for (int s = lane; s < nsplit; s += 32) mloc = fmaxf(mloc, ml[s * 2]);
 #pragma unroll
-    for (int o2 = 16; o2 >= 1; o2 >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o2));
-    float lloc = 0.f;
-    for (int s = lane; s < nsplit; s += 32) {
-      const float ms = ld_cg(p.part_ml + (ph + s) * 2);
-      const float wgt = (ms == -INFINITY) ? 0.f : ex2(ms - mloc);
-      s_w[h * MAX_SPLITS_CAP + s] = wgt;
-      lloc += ld_cg(p.part_ml + (ph + s) * 2 + 1) * wgt;
+      for (int o2 = 16; o2 >= 1; o2 >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o2));
+      float lloc = 0.f;
+      for (int s = lane; s < nsplit; s += 32) {
+        const float ms = ml[s * 2];
+        const float wgt = (ms == -INFINITY) ? 0.f : ex2(ms - mloc);
+        s_w[h * MAX_SPLITS_CAP + s] = wgt;
+        lloc += ml[s * 2 + 1] * wgt;
+      }
+#pragma unroll
+      for (int o2 = 16; o2 >= 1; o2 >>= 1) lloc += __shfl_xor_sync(0xffffffffu, lloc, o2);
+      if (lane == 0) s_inv[h] = lloc > 0.f ? 1.f / lloc : 0.f;
     }
+  }
+  __syncthreads();
+
+  // rows of the partial buffer, linearised as (head, split); rounds of up to CROWS rows
+  constexpr int CPL = D / 32;                 // channels per lane
+  constexpr int HPW = (8 + NW - 1) / NW;      // heads per warp
+  float acc[HPW][CPL];
 #pragma unroll
-    for (int o2 = 16; o2 >= 1; o2 >>= 1) lloc += __shfl_xor_sync(0xffffffffu, lloc, o2);
-    __syncwarp();
-    const float inv = lloc > 0.f ? 1.f / lloc : 0.f;
-    // each lane owns 4 consecutive channels (d = 128) or 2 (d = 64)
-    constexpr int CPL = D / 32;
-    float acc[CPL];
+  for (int i = 0; i < HPW; ++i)
 #pragma unroll
-    for (int j = 0; j < CPL; ++j) acc[j] = 0.f;
-    const float* src = p.part_acc + ph * D + lane * CPL;
-    int s = 0;
-    for (; s + 4 <= nsplit; s += 4) {
-      float v[4][CPL];
+    for (int j = 0; j < CPL; ++j) acc[i][j] = 0.f;
+  const int total_rows = r * nsplit;
+  for (int r0 = 0; r0 < total_rows && !cfail; r0 += C::CROWS) {
+    const int r1 = min(total_rows, r0 + C::CROWS);
+    if (threadIdx.x == 0) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_expect_tx(cbar, (uint32_t)(r1 - r0) * D * 4u);
+      for (int h = r0 / nsplit; h < r && h * nsplit < r1; ++h) {
+        const int a = max(r0, h * nsplit), e = min(r1, (h + 1) * nsplit);   // rows of head h in this round
+        bulk_load(smem_u32(s_rows + (int64_t)(a - r0) * D),
+                  p.part_acc + (ph0 + (int64_t)h * p.max_splits + (a - h * nsplit)) * D,
+                  (uint32_t)(e - a) * D * 4u, cbar);
+      }
+    }
+    cfail = !mbar_wait(cbar, cphase & 1);
+    ++cphase;
+    if (!cfail) {
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if constexpr (CPL == 4) {
-          const float4 x = ld_cg4(src + (int64_t)(s + u) * D);
-          v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
-        } else {
+      for (int i = 0; i < HPW; ++i) {
+        const int h = warp + i * NW;
+        if (h >= r) continue;
+        const int a = max(r0, h * nsplit), e = min(r1, (h + 1) * nsplit);
+        for (int row = a; row < e; ++row) {
+          const float wgt = s_w[h * MAX_SPLITS_CAP + (row - h * nsplit)];
+          const float* src = s_rows + (int64_t)(row - r0) * D + lane * CPL;
 #pragma unroll
-          for (int j = 0; j < CPL; ++j) v[u][j] = ld_cg(src + (int64_t)(s + u) * D + j);
+          for (int j = 0; j < CPL; ++j) acc[i][j] += src[j] * wgt;
         }
       }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const float wgt = s_w[h * MAX_SPLITS_CAP + s + u];
-#pragma unroll
-        for (int j = 0; j < CPL; ++j) acc[j] += v[u][j] * wgt;
-      }
     }
-    for (; s < nsplit; ++s) {
-      const float wgt = s_w[h * MAX_SPLITS_CAP + s];
+    __syncthreads();                          // the rows are overwritten by the next round
+  }
+  if (cfail) {
+    if (threadIdx.x == 0) atomicExch(p.err_flag, 1);
+    return;
+  }
 #pragma unroll
-      for (int j = 0; j < CPL; ++j) acc[j] += ld_cg(src + (int64_t)s * D + j) * wgt;
-    }
+  for (int i = 0; i < HPW; ++i) {
+    const int h = warp + i * NW;
+    if (h >= r) continue;
+    const float inv = s_inv[h];
     __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * y.H_q + kvh * r + h) * D + lane * CPL;
 #pragma unroll
     for (int j = 0; j < CPL; j += 2)
-      *reinterpret_cast<__nv_bfloat162*>(dst + j) = __floats2bfloat162_rn(acc[j] * inv, acc[j + 1] * inv);
+      *reinterpret_cast<__nv_bfloat162*>(dst + j) = __floats2bfloat162_rn(acc[i][j] * inv, acc[i][j + 1] * inv);
   }
 }
 
@@ -412,60 +537,12 @@ __global__ void pod_zero_empty_kernel(const DecodeParams p) {
   for (int i = threadIdx.x; i < per; i += blockDim.x) p.out[(int64_t)b * per + i] = 0;
 }
 
-// Merge of the split partials of one (sequence, query head): the gate of Eq. 2 generalised
-// from two parts to n_splits parts.  Block = D threads, grid (H_q, B).
-template <int D>
-__global__ void __launch_bounds__(D) pod_combine_kernel(const DecodeParams p) {
-  pdl_wait();
-  pdl_launch_dependents();
-  const int hq = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
-  const int n = p.len[b];
-  const int nsplit = min(p.max_splits, (n + p.split_tokens - 1) / p.split_tokens);
-  const int64_t ph = ((int64_t)b * p.y.H_q + hq) * p.max_splits;
-  __shared__ float s_w[MAX_SPLITS_CAP];     // weight of each split: 2^(m_s - M)
-  __shared__ float s_red[2][4];
-  // pass 1: every thread takes some splits' (max, sum); block-wide max
-  float mloc = -INFINITY;
-  for (int s = c; s < nsplit; s += D) mloc = fmaxf(mloc, p.part_ml[(ph + s) * 2]);
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o));
-  if ((c & 31) == 0) s_red[0][c >> 5] = mloc;
-  __syncthreads();
-  float M = s_red[0][0];
-  for (int w = 1; w < D / 32; ++w) M = fmaxf(M, s_red[0][w]);
-  float lloc = 0.f;
-  for (int s = c; s < nsplit; s += D) {
-    const float ms = p.part_ml[(ph + s) * 2];
-    const float wgt = (ms == -INFINITY) ? 0.f : ex2(ms - M);
-    s_w[s] = wgt;
-    lloc += p.part_ml[(ph + s) * 2 + 1] * wgt;
-  }
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) lloc += __shfl_xor_sync(0xffffffffu, lloc, o);
-  if ((c & 31) == 0) s_red[1][c >> 5] = lloc;
-  __syncthreads();
-  float l = 0.f;
-  for (int w = 0; w < D / 32; ++w) l += s_red[1][w];
-  // pass 2: channel c over the splits, loads independent of one another
-  float a = 0.f;
-  int s = 0;
-  for (; s + 4 <= nsplit; s += 4) {
-    const float v0 = p.part_acc[(ph + s) * D + c], v1 = p.part_acc[(ph + s + 1) * D + c];
-    const float v2 = p.part_acc[(ph + s + 2) * D + c], v3 = p.part_acc[(ph + s + 3) * D + c];
-    a += v0 * s_w[s] + v1 * s_w[s + 1] + v2 * s_w[s + 2] + v3 * s_w[s + 3];
-  }
-  for (; s < nsplit; ++s) a += p.part_acc[(ph + s) * D + c] * s_w[s];
-  const float out = (l > 0.f) ? a / l : 0.f;
-  reinterpret_cast<__nv_bfloat16*>(p.out)[((int64_t)b * p.y.H_q + hq) * D + c] = __float2bfloat16_rn(out);
-}
-
-cudaLaunchAttribute g_pdl_attr[1];
-cudaLaunchConfig_t pdl_config(dim3 grid, dim3 block, size_t smem, cudaStream_t s) {
-  g_pdl_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  g_pdl_attr[0].val.programmaticStreamSerializationAllowed = 1;
+cudaLaunchConfig_t pdl_config(cudaLaunchAttribute* attr, dim3 grid, dim3 block, size_t smem, cudaStream_t s) {
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
-  cfg.attrs = g_pdl_attr; cfg.numAttrs = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
   return cfg;
 }
 
@@ -479,7 +556,8 @@ int launch_decode_t(const CUtensorMap& tmap, const DecodeParams& p, int grid_spl
     if (e != cudaSuccess) return (int)e;
     configured = true;
   }
-  cudaLaunchConfig_t cfg = pdl_config(dim3(grid_splits, p.y.H_kv, p.y.B), dim3(NW * 32), C::SMEM, s);
+  cudaLaunchAttribute attr[1];
+  cudaLaunchConfig_t cfg = pdl_config(attr, dim3(grid_splits, p.y.H_kv, p.y.B), dim3(C::NW * 32), C::SMEM, s);
   return (int)cudaLaunchKernelEx(&cfg, pod_decode_splitk_kernel<D>, tmap, p);
 }
 
@@ -490,28 +568,25 @@ int resident_t() {
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
   if (e != cudaSuccess) return 0;
   int nb = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, pod_decode_splitk_kernel<D>, NW * 32, C::SMEM);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, pod_decode_splitk_kernel<D>, C::NW * 32, C::SMEM);
   return e == cudaSuccess ? nb : 0;
 }
 
 }  // namespace
 
 int decode_tile_tokens() { return TOK; }
+int decode_warps_per_cta() { return DECODE_WARPS; }
 
 int launch_decode(const CUtensorMap& tmap, const DecodeParams& p, int grid_splits, cudaStream_t s) {
+  if (p.tiles_per_chunk < 1 || p.static_eighths < 0 || p.static_eighths > 8 || (p.max_splits & 1)) return (int)cudaErrorInvalidValue;
   if (p.y.D == 128) return launch_decode_t<128>(tmap, p, grid_splits, s);
   if (p.y.D == 64) return launch_decode_t<64>(tmap, p, grid_splits, s);
   return (int)cudaErrorInvalidValue;
 }
 
-int launch_combine(const DecodeParams& p, cudaStream_t s) {
-  cudaLaunchConfig_t cfg = pdl_config(dim3(p.y.H_q, p.y.B), dim3(p.y.D), 0, s);
-  if (p.y.D == 128) return (int)cudaLaunchKernelEx(&cfg, pod_combine_kernel<128>, p);
-  return (int)cudaLaunchKernelEx(&cfg, pod_combine_kernel<64>, p);
-}
-
 int launch_zero_empty(const DecodeParams& p, cudaStream_t s) {
-  cudaLaunchConfig_t cfg = pdl_config(dim3(p.y.B), dim3(128), 0, s);
+  cudaLaunchAttribute attr[1];
+  cudaLaunchConfig_t cfg = pdl_config(attr, dim3(p.y.B), dim3(128), 0, s);
   return (int)cudaLaunchKernelEx(&cfg, pod_zero_empty_kernel, p);
 }
 

@@ -22,8 +22,9 @@ constexpr int STATIC_MAX_SPLITS = 64;
 constexpr int STATIC_MAX_DEVICES = 64;
 constexpr size_t OFF_PACC = 0;                                                         // fp32 [64][64][128]
 constexpr size_t OFF_PML = (size_t)STATIC_MAX_Q_HEADS * STATIC_MAX_SPLITS * 128 * 4;   // fp32 [64][64][2]
-constexpr size_t OFF_TICKETS = OFF_PML + (size_t)STATIC_MAX_Q_HEADS * STATIC_MAX_SPLITS * 2 * 4;   // int32 [64]
-constexpr size_t OFF_ERR = OFF_TICKETS + 256;
+constexpr size_t SCHED_BYTES = (size_t)STATIC_MAX_Q_HEADS * SCHED_STRIDE * 4;          // int32 [64 KV heads][32]
+constexpr size_t OFF_SCHED = OFF_PML + (size_t)STATIC_MAX_Q_HEADS * STATIC_MAX_SPLITS * 2 * 4;
+constexpr size_t OFF_ERR = OFF_SCHED + SCHED_BYTES;
 constexpr size_t STATIC_BYTES = OFF_ERR + 256;
 static_assert(STATIC_BYTES == POD_STATIC_SCRATCH_BYTES, "header and library disagree on the scratch size");
 
@@ -121,15 +122,20 @@ extern "C" int pod_dense_decode_attn_static(const void* kv_device, int capacity,
   p.part_ml = reinterpret_cast<float*>(su->scratch + OFF_PML);
   p.out = static_cast<uint16_t*>(out_device);
   p.err_flag = reinterpret_cast<int32_t*>(su->scratch + OFF_ERR);
-  p.tickets = reinterpret_cast<int32_t*>(su->scratch + OFF_TICKETS);
+  p.sched = reinterpret_cast<int32_t*>(su->scratch + OFF_SCHED);
   p.layer = 0; p.block = 0; p.split_tokens = split_tokens; p.max_splits = STATIC_MAX_SPLITS;
+  p.tiles_per_chunk = split_tokens / (decode_tile_tokens() * decode_warps_per_cta() * 16);
+  if (p.tiles_per_chunk < 1) p.tiles_per_chunk = 1;
+  if (p.tiles_per_chunk > 16) p.tiles_per_chunk = 16;
+  p.static_eighths = 5;
   p.scale_log2 = (sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim)) * 1.4426950408889634f;
   p.keep_distk = 0;
   p.by_value = 1;
   p.v_len[0] = n_tokens; p.v_cap_d[0] = 0; p.v_row_base[0] = 0;
 
-  // The array keeps whatever the previous call left: the tickets must start at zero.
-  if (cudaMemsetAsync(su->scratch + OFF_TICKETS, 0, 512, stream) != cudaSuccess) return POD_ERR_CUDA;
+  // The array keeps whatever the previous call left: the chunk counters, the tickets and the
+  // error flag must start at zero.
+  if (cudaMemsetAsync(su->scratch + OFF_SCHED, 0, SCHED_BYTES + 256, stream) != cudaSuccess) return POD_ERR_CUDA;
   const int e = launch_decode(tmap, p, grid_splits, stream);
   return e == 0 ? POD_OK : POD_ERR_CUDA;
 }
