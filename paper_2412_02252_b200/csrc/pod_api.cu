@@ -340,7 +340,7 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* str
     // A warp sees about split_tokens / (tile tokens x warps) tiles; it should make a dozen draws.
     int tch = plan.split_tokens / (decode_tile_tokens() * decode_warps_per_cta() * 16);
     if (c->force_chunk_tiles > 0) tch = c->force_chunk_tiles;
-    p.tiles_per_chunk = tch < 1 ? 1 : (tch > 16 ? 16 : tch);
+    p.tiles_per_chunk = tch < 1 ? 1 : (tch > 256 ? 256 : tch);
     p.static_eighths = c->static_eighths;
   }
   p.scale_log2 = c->scale * 1.4426950408889634f;

@@ -1,6 +1,7 @@
 // Split-K decode attention over the PoD layout with the log-sum-exp combine in the same launch.
 //
-// Grid (split, KV head, sequence); the CTAs of one (sequence, KV head) share that head's tokens.
+// Grid (KV head, split, sequence): consecutive CTAs belong to different heads, so every head's
+// CTAs are spread over all SMs.  The CTAs of one (sequence, KV head) share that head's tokens.
 // The tokens are cut into tiles of 16 in "virtual" order -- proximal rows first (sink, then
 // ring slots), distant rows after -- and tiles into chunks of a few tiles.  Each warp is an
 // independent flash-decoding stream over chunks:
@@ -98,6 +99,24 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
+__device__ __forceinline__ float lds_f32(uint32_t a) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ float2 lds_f32x2(uint32_t a) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ float4 lds_f32x4(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t a, float v) {
+  asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -135,13 +154,12 @@ struct Cfg {
   static constexpr int STAGE_B = 2 * TILE_B;
   static constexpr int WARP_B = NSTAGE * STAGE_B;
   static constexpr int RING_B = NW * WARP_B;
-  static constexpr int N_BARS = NW * NSTAGE + 1;      // one per stage, one for the combine
+  static constexpr int N_BARS = NW * NSTAGE + NW;     // one per stage, one per warp for the combine
   static constexpr int SMEM = RING_B + N_BARS * 8 + 1024;   // + slack to align to 1024
-  // the combine reuses the rings: split weights, (max, sum) pairs, then partial rows
-  static constexpr int CW_B = 8 * MAX_SPLITS_CAP * 4;
-  static constexpr int CML_B = 8 * MAX_SPLITS_CAP * 8;
-  static constexpr int CROWS = (RING_B - CW_B - CML_B) / (D * 4);   // partial rows per round
-  static_assert(CROWS >= 8, "the rings must hold a few partial rows for the combine");
+  // the combine reuses each warp's ring: (max, sum) pairs, split weights, then partial rows
+  static constexpr int CML_OFF = 0, CW_OFF = MAX_SPLITS_CAP * 8, CROW_OFF = CW_OFF + MAX_SPLITS_CAP * 4;
+  static constexpr int CROWS = (WARP_B - CROW_OFF) / (D * 4);   // partial rows per round
+  static_assert(CROWS >= 8, "a warp's ring must hold a few partial rows for the combine");
   static_assert(WARP_B >= (8 * D + 16) * 4, "merge scratch must fit the warp's ring");
 };
 
@@ -153,7 +171,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const Layout& y = p.y;
   const int r = y.H_q / y.H_kv;   // query heads per KV head (<= 8): rows of the Q operand
 
-  const int b = blockIdx.z, kvh = blockIdx.y, split = blockIdx.x;
+  const int b = blockIdx.z, kvh = blockIdx.x, split = blockIdx.y;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);   // swizzle atoms are 1024 B
@@ -161,10 +179,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   unsigned char* wbuf = smem + warp * C::WARP_B;
   const uint32_t wbuf_s = smem_u32(wbuf);
   const uint32_t bar0 = smem_u32(smem + C::RING_B) + warp * NSTAGE * 8;
-  const uint32_t cbar = smem_u32(smem + C::RING_B) + NW * NSTAGE * 8;
+  const uint32_t cbar = smem_u32(smem + C::RING_B) + (NW * NSTAGE + warp) * 8;   // this warp's combine barrier
   if (lane == 0) {
     for (int s = 0; s < NSTAGE; ++s) mbar_init(bar0 + s * 8, 1);
-    if (warp == 0) mbar_init(cbar, 1);
+    mbar_init(cbar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap)) : "memory");
@@ -422,109 +440,101 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   }
 
   // ---- ticket: the CTA that publishes the last partial of this (sequence, KV head) combines ----
+  // The barrier orders every thread's partial stores before thread 0's release at GPU scope
+  // (cumulative), and the winner's acquire orders them before its reads.
   __shared__ int s_last;
-  __shared__ float s_inv[8];
-  __threadfence();
   fence_async_global();                  // the partials are read back through the async proxy
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int got = atomicAdd(sched + SCHED_TICKET, 1);
+    int got;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(got) : "l"(sched + SCHED_TICKET) : "memory");
     s_last = (got == nsplit - 1);
     if (s_last) { sched[SCHED_TICKET] = 0; sched[0] = 0; }   // ready for the next launch
   }
   __syncthreads();
   if (!s_last) return;
-  __threadfence();
 
-  float* s_w = reinterpret_cast<float*>(smem);                           // [8][MAX_SPLITS_CAP] split weights
-  float* s_ml = reinterpret_cast<float*>(smem + C::CW_B);                // [r][max_splits][2]
-  float* s_rows = reinterpret_cast<float*>(smem + C::CW_B + C::CML_B);   // partial rows of one round
+  // ---- combine: every warp merges the partials of its own query heads, on its own -----------
+  // The (max, sum) pairs and the partial rows of a head come into the warp's ring with bulk
+  // copies (one memory round trip); rounds of CROWS rows if a head has more splits than fit.
+  constexpr int CPL = D / 32;                 // channels per lane
+  const uint32_t w_ml = wbuf_s + C::CML_OFF, w_w = wbuf_s + C::CW_OFF, w_rows = wbuf_s + C::CROW_OFF;
   const int64_t ph0 = ((int64_t)b * y.H_q + kvh * r) * p.max_splits;     // partial row of (head 0, split 0)
   uint32_t cphase = 0;
-  if (threadIdx.x == 0) {
-    fence_async_global();
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    const uint32_t bytes = (uint32_t)p.max_splits * 8u;
-    mbar_expect_tx(cbar, bytes * r);
-    for (int h = 0; h < r; ++h)
-      bulk_load(smem_u32(s_ml + h * p.max_splits * 2), p.part_ml + (ph0 + (int64_t)h * p.max_splits) * 2, bytes, cbar);
-  }
-  bool cfail = !mbar_wait(cbar, cphase & 1);
-  ++cphase;
-  if (!cfail) {
-    for (int h = warp; h < r; h += NW) {
-      const float* ml = s_ml + h * p.max_splits * 2;
-      float mloc = -INFINITY;
-      for (int s = lane; s < nsplit; s += 32) mloc = fmaxf(mloc, ml[s * 2]);
+  bool cfail = false;
+  for (int h = warp; h < r && !cfail; h += NW) {
+    const int64_t ph = ph0 + (int64_t)h * p.max_splits;
+    float acc[CPL];
 #pragma unroll
-      for (int o2 = 16; o2 >= 1; o2 >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o2));
-      float lloc = 0.f;
-      for (int s = lane; s < nsplit; s += 32) {
-        const float ms = ml[s * 2];
-        const float wgt = (ms == -INFINITY) ? 0.f : ex2(ms - mloc);
-        s_w[h * MAX_SPLITS_CAP + s] = wgt;
-        lloc += ml[s * 2 + 1] * wgt;
+    for (int j = 0; j < CPL; ++j) acc[j] = 0.f;
+    float inv = 0.f;
+    for (int r0 = 0; r0 < nsplit; r0 += C::CROWS) {
+      const int r1 = min(nsplit, r0 + C::CROWS);
+      if (lane == 0) {
+        fence_async_global();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const uint32_t ml_bytes = (uint32_t)p.max_splits * 8u;
+        mbar_expect_tx(cbar, (uint32_t)(r1 - r0) * D * 4u + (r0 == 0 ? ml_bytes : 0u));
+        if (r0 == 0) bulk_load(w_ml, p.part_ml + ph * 2, ml_bytes, cbar);
+        bulk_load(w_rows, p.part_acc + (ph + r0) * D, (uint32_t)(r1 - r0) * D * 4u, cbar);
       }
+      if (!__all_sync(0xffffffffu, mbar_wait(cbar, cphase & 1))) { cfail = true; break; }
+      ++cphase;
+      if (r0 == 0) {                          // weights 2^(m_s - M) of the splits and 1 / sum, once per head
+        float2 ml[MAX_SPLITS_CAP / 32];
+        float mloc = -INFINITY;
 #pragma unroll
-      for (int o2 = 16; o2 >= 1; o2 >>= 1) lloc += __shfl_xor_sync(0xffffffffu, lloc, o2);
-      if (lane == 0) s_inv[h] = lloc > 0.f ? 1.f / lloc : 0.f;
-    }
-  }
-  __syncthreads();
-
-  // rows of the partial buffer, linearised as (head, split); rounds of up to CROWS rows
-  constexpr int CPL = D / 32;                 // channels per lane
-  constexpr int HPW = (8 + NW - 1) / NW;      // heads per warp
-  float acc[HPW][CPL];
-#pragma unroll
-  for (int i = 0; i < HPW; ++i)
-#pragma unroll
-    for (int j = 0; j < CPL; ++j) acc[i][j] = 0.f;
-  const int total_rows = r * nsplit;
-  for (int r0 = 0; r0 < total_rows && !cfail; r0 += C::CROWS) {
-    const int r1 = min(total_rows, r0 + C::CROWS);
-    if (threadIdx.x == 0) {
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_expect_tx(cbar, (uint32_t)(r1 - r0) * D * 4u);
-      for (int h = r0 / nsplit; h < r && h * nsplit < r1; ++h) {
-        const int a = max(r0, h * nsplit), e = min(r1, (h + 1) * nsplit);   // rows of head h in this round
-        bulk_load(smem_u32(s_rows + (int64_t)(a - r0) * D),
-                  p.part_acc + (ph0 + (int64_t)h * p.max_splits + (a - h * nsplit)) * D,
-                  (uint32_t)(e - a) * D * 4u, cbar);
-      }
-    }
-    cfail = !mbar_wait(cbar, cphase & 1);
-    ++cphase;
-    if (!cfail) {
-#pragma unroll
-      for (int i = 0; i < HPW; ++i) {
-        const int h = warp + i * NW;
-        if (h >= r) continue;
-        const int a = max(r0, h * nsplit), e = min(r1, (h + 1) * nsplit);
-        for (int row = a; row < e; ++row) {
-          const float wgt = s_w[h * MAX_SPLITS_CAP + (row - h * nsplit)];
-          const float* src = s_rows + (int64_t)(row - r0) * D + lane * CPL;
-#pragma unroll
-          for (int j = 0; j < CPL; ++j) acc[i][j] += src[j] * wgt;
+        for (int k = 0; k < MAX_SPLITS_CAP / 32; ++k) {
+          const int sp = lane + 32 * k;
+          ml[k] = sp < nsplit ? lds_f32x2(w_ml + sp * 8) : make_float2(-INFINITY, 0.f);
+          mloc = fmaxf(mloc, ml[k].x);
         }
-      }
-    }
-    __syncthreads();                          // the rows are overwritten by the next round
-  }
-  if (cfail) {
-    if (threadIdx.x == 0) atomicExch(p.err_flag, 1);
-    return;
-  }
 #pragma unroll
-  for (int i = 0; i < HPW; ++i) {
-    const int h = warp + i * NW;
-    if (h >= r) continue;
-    const float inv = s_inv[h];
+        for (int o2 = 16; o2 >= 1; o2 >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o2));
+        float lloc = 0.f;
+#pragma unroll
+        for (int k = 0; k < MAX_SPLITS_CAP / 32; ++k) {
+          const int sp = lane + 32 * k;
+          const float wgt = (ml[k].x == -INFINITY) ? 0.f : ex2(ml[k].x - mloc);
+          if (sp < nsplit) sts_f32(w_w + sp * 4, wgt);
+          lloc += ml[k].y * wgt;
+        }
+#pragma unroll
+        for (int o2 = 16; o2 >= 1; o2 >>= 1) lloc += __shfl_xor_sync(0xffffffffu, lloc, o2);
+        inv = lloc > 0.f ? 1.f / lloc : 0.f;
+        __syncwarp();
+      }
+      // eight rows per trip, the last trip padded with weight 0 on a valid row
+      for (int row = r0; row < r1; row += 8) {
+        float v[8][CPL], wg[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const bool in = row + u < r1;
+          const int rr = in ? row + u : r0;
+          wg[u] = in ? lds_f32(w_w + rr * 4) : 0.f;
+          const uint32_t src = w_rows + (uint32_t)(rr - r0) * (D * 4) + lane * (CPL * 4);
+          if constexpr (CPL == 4) {
+            const float4 x = lds_f32x4(src);
+            v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
+          } else {
+            const float2 x = lds_f32x2(src);
+            v[u][0] = x.x; v[u][1] = x.y;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+#pragma unroll
+          for (int j = 0; j < CPL; ++j) acc[j] += v[u][j] * wg[u];
+      }
+      __syncwarp();                           // the rows are overwritten by the next round
+    }
+    if (cfail) break;
     __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * y.H_q + kvh * r + h) * D + lane * CPL;
 #pragma unroll
     for (int j = 0; j < CPL; j += 2)
-      *reinterpret_cast<__nv_bfloat162*>(dst + j) = __floats2bfloat162_rn(acc[i][j] * inv, acc[i][j + 1] * inv);
+      *reinterpret_cast<__nv_bfloat162*>(dst + j) = __floats2bfloat162_rn(acc[j] * inv, acc[j + 1] * inv);
   }
+  if (cfail && lane == 0) atomicExch(p.err_flag, 1);
 }
 
 // Outputs of sequences that hold no token are zero (no split CTA exists to write them).
@@ -557,7 +567,7 @@ int launch_decode_t(const CUtensorMap& tmap, const DecodeParams& p, int grid_spl
     configured = true;
   }
   cudaLaunchAttribute attr[1];
-  cudaLaunchConfig_t cfg = pdl_config(attr, dim3(grid_splits, p.y.H_kv, p.y.B), dim3(C::NW * 32), C::SMEM, s);
+  cudaLaunchConfig_t cfg = pdl_config(attr, dim3(p.y.H_kv, grid_splits, p.y.B), dim3(C::NW * 32), C::SMEM, s);
   return (int)cudaLaunchKernelEx(&cfg, pod_decode_splitk_kernel<D>, tmap, p);
 }
 
