@@ -120,6 +120,20 @@ int pod_cache_write(pod_cache* c, int layer, int seq, const void* k_device,
 int pod_decode_attn(pod_cache* c, int layer, const void* q_device, void* out_device,
                     void* cuda_stream);
 
+/* pod_cache_write(layer, seq = -1, k, v, 1) followed by pod_decode_attn(layer, q, out), as one
+ * kernel launch: the decode step of Section 2.2 as a layer runs it -- append the current token's
+ * K/V, then attend over all tokens up to and including it (Eq. 1 ranges end at n) -- with the
+ * cache update of Fig. 2 (right) applied by the same kernel: the new rows go to the sink or to
+ * their ring slot, the slot's previous occupant moves to the distant stores (value always, key
+ * from the block's lowest layer only).  Results (output and cache contents) are those of the
+ * two separate calls; only the summation order of the softmax differs.
+ *   k_device, v_device: device bf16 [B][H_kv][d], one new token per sequence.
+ *   q_device, out_device: device bf16 [B][H_q][d].
+ * Errors: INVALID, CAPACITY (a sequence is full; nothing changed), ORDER (as pod_decode_attn,
+ * judged at the lengths after the append), CUDA. */
+int pod_append_decode_attn(pod_cache* c, int layer, const void* k_device, const void* v_device,
+                           const void* q_device, void* out_device, void* cuda_stream);
+
 /* Byte accounting (host integers).  Live bytes of a sequence of length n (at the layer with
  * the most tokens): row * H_kv * (L * (2 n_p + n_d) + ceil(L / G) * n_d), n_p = min(n, n_s+n_r),
  * n_d = n - n_p; the saving against dense is (n_d / n) (1 - ceil(L/G)/L) / 2 -- only keys

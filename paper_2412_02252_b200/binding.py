@@ -44,6 +44,7 @@ def _load() -> ctypes.CDLL:
         "pod_cache_destroy": (c_int, [c_void_p]),
         "pod_cache_write": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_void_p]),
         "pod_decode_attn": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
+        "pod_append_decode_attn": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
         "pod_cache_bytes": (c_int64, [c_void_p, c_int]),
         "pod_cache_seq_len": (c_int, [c_void_p, c_int, c_int]),
         "pod_cache_reset": (c_int, [c_void_p, c_int]),
@@ -63,7 +64,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_destroy", "pod_cache_write",
-           "pod_decode_attn", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
+           "pod_decode_attn", "pod_append_decode_attn", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
            "pod_cache_read_region", "pod_cache_device_status", "pod_cache_last_cuda_error",
            "pod_cache_last_launch", "pod_strerror", "pod_dense_decode_attn_static"]
 
@@ -135,6 +136,10 @@ class PodCache:
 
     def decode_attn(self, layer: int, q, out, stream: int = 0) -> int:
         return _check(lib.pod_decode_attn(self._h, layer, _ptr(q), _ptr(out), stream), "pod_decode_attn")
+
+    def append_decode_attn(self, layer: int, k, v, q, out, stream: int = 0) -> int:
+        return _check(lib.pod_append_decode_attn(self._h, layer, _ptr(k), _ptr(v), _ptr(q), _ptr(out), stream),
+                      "pod_append_decode_attn")
 
     def bytes(self, which: int) -> int:
         return lib.pod_cache_bytes(self._h, which)

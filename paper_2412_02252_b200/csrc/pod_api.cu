@@ -68,7 +68,7 @@ bool carve(const pod_config& c, const int32_t* cap, Carve* out) {
   if (rows >= ((int64_t)1 << 31)) return false;   // tile coordinates are 32-bit row indices
   out->total_rows = rows;
   size_t off = align_up((size_t)(rows * row_bytes));
-  out->off_len = off;      off = align_up(off + (size_t)c.n_layers * c.batch * 4);
+  out->off_len = off;      off = align_up(off + (size_t)2 * c.n_layers * c.batch * 4);   // two copies, see len_cur
   out->off_rowbase = off;  off = align_up(off + (size_t)c.batch * 8);
   out->off_capd = off;     off = align_up(off + (size_t)c.batch * 4);
   out->off_stash = off;    off = align_up(off + (size_t)n_blocks * c.batch * c.n_q_heads * row_bytes);
@@ -105,7 +105,14 @@ struct pod_cache {
   // planner memo
   int64_t memo_sum = -1; int32_t memo_max = -1; DecodePlan memo_plan{};
 
-  int32_t* d_len(int layer) const { return reinterpret_cast<int32_t*>(arena + cv.off_len) + (size_t)layer * cfg.batch; }
+  // Device lengths are kept twice.  A launch that appends and attends at once reads one copy and
+  // writes the other (its CTAs start at different times, so nobody may change what they read);
+  // len_cur[layer] says which copy is current.
+  std::vector<uint8_t> len_cur;        // [L]
+  int32_t* d_len_copy(int layer, int which) const {
+    return reinterpret_cast<int32_t*>(arena + cv.off_len) + ((size_t)which * cfg.n_layers + layer) * cfg.batch;
+  }
+  int32_t* d_len(int layer) const { return d_len_copy(layer, len_cur[layer]); }
   int32_t& h_len(int layer, int b) { return len[(size_t)layer * cfg.batch + b]; }
   int32_t h_len(int layer, int b) const { return len[(size_t)layer * cfg.batch + b]; }
 };
@@ -208,6 +215,7 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
   if (!carve(*cfg, seq_capacity, &c->cv)) { delete c; return POD_ERR_INVALID; }
   c->cap.assign(seq_capacity, seq_capacity + cfg->batch);
   c->len.assign((size_t)cfg->n_layers * cfg->batch, 0);
+  c->len_cur.assign((size_t)cfg->n_layers, 0);
   c->stash_len.assign((size_t)c->cv.n_blocks * cfg->batch, -1);
   c->scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)cfg->head_dim);
   c->dry = cfg->device < 0;
@@ -301,20 +309,33 @@ int pod_cache_write(pod_cache* c, int layer, int seq, const void* k, const void*
   return c->dry ? POD_DRY_RUN : POD_OK;
 }
 
-int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* stream) {
+// pod_decode_attn (k_new == nullptr) and pod_append_decode_attn (k_new, v_new: one new token per
+// sequence, appended by the same launch that attends).
+static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v_new, const void* q, void* out,
+                       void* stream) {
   if (!c || !q || !out) return POD_ERR_INVALID;
+  const bool fused = k_new != nullptr;
+  if (fused && (!v_new || ((uintptr_t)k_new % 16) != 0 || ((uintptr_t)v_new % 16) != 0)) return POD_ERR_INVALID;
   const pod_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return POD_ERR_INVALID;
   if (((uintptr_t)q % 16) != 0 || ((uintptr_t)out % 16) != 0) return POD_ERR_INVALID;
   const int low = layer - layer % g.group_size, block = layer / g.group_size;
   const bool lowest = (low == layer);
   int32_t* sl = &c->stash_len[(size_t)block * g.batch];
+  const int add = fused ? 1 : 0;
+  if (fused)
+    for (int b = 0; b < g.batch; ++b)
+      if ((int64_t)c->h_len(layer, b) + 1 > c->cap[b]) return POD_ERR_CAPACITY;
   if (!lowest) {
     for (int b = 0; b < g.batch; ++b) {
-      const int32_t n = c->h_len(layer, b);
+      const int32_t n = c->h_len(layer, b) + add;
       if (n != c->h_len(low, b)) return POD_ERR_ORDER;       // block must hold equal lengths
       if (n > 0 && sl[b] != n) return POD_ERR_ORDER;         // lowest layer's q not stashed at this step
     }
+  }
+  if (fused) {                          // from here on the host lengths are the new ones
+    for (int b = 0; b < g.batch; ++b) c->h_len(layer, b) += 1;
+    c->memo_sum = -1;
   }
   if (c->dry) {
     if (lowest) for (int b = 0; b < g.batch; ++b) sl[b] = c->h_len(layer, b);
@@ -325,6 +346,9 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* str
   p.y = c->y;
   p.arena = reinterpret_cast<const uint16_t*>(c->arena);
   p.len = c->d_len(layer);
+  p.new_k = static_cast<const uint16_t*>(k_new);
+  p.new_v = static_cast<const uint16_t*>(v_new);
+  p.len_out = fused ? c->d_len_copy(layer, c->len_cur[layer] ^ 1) : nullptr;
   p.q = static_cast<const uint16_t*>(q);
   uint16_t* stash = reinterpret_cast<uint16_t*>(c->arena + c->cv.off_stash) + (size_t)block * g.batch * g.n_q_heads * g.head_dim;
   p.q_low = lowest ? p.q : stash;
@@ -367,8 +391,12 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* str
   int kernels = 0;
   if (plan.n_ctas > 0) {
     const int e = launch_decode(c->tmap, p, plan.grid_splits, s);
-    if (e != 0) return cuda_fail(c, (cudaError_t)e);
+    if (e != 0) {
+      if (fused) { for (int b = 0; b < g.batch; ++b) c->h_len(layer, b) -= 1; c->memo_sum = -1; }
+      return cuda_fail(c, (cudaError_t)e);
+    }
     ++kernels;
+    if (fused) c->len_cur[layer] ^= 1;
   }
   {
     bool any_empty = false;
@@ -382,6 +410,16 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* str
   if (lowest) for (int b = 0; b < g.batch; ++b) sl[b] = c->h_len(layer, b);
   c->last_split_tokens = plan.split_tokens; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;
   return POD_OK;
+}
+
+int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* stream) {
+  return decode_impl(c, layer, nullptr, nullptr, q, out, stream);
+}
+
+int pod_append_decode_attn(pod_cache* c, int layer, const void* k, const void* v, const void* q, void* out,
+                           void* stream) {
+  if (!k || !v) return POD_ERR_INVALID;
+  return decode_impl(c, layer, k, v, q, out, stream);
 }
 
 int64_t pod_cache_bytes(const pod_cache* c, int which) {
@@ -424,6 +462,8 @@ int pod_cache_reset(pod_cache* c, int seq) {
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e == cudaSuccess)
     e = cudaMemcpy(c->arena + c->cv.off_len, c->len.data(), c->len.size() * 4, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(c->arena + c->cv.off_len + c->len.size() * 4, c->len.data(), c->len.size() * 4, cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return cuda_fail(c, e);
   return POD_OK;
 }

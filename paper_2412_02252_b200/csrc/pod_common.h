@@ -71,6 +71,12 @@ struct DecodeParams {
   Layout y;
   const uint16_t* arena;
   const int32_t* len;      // device lengths of this layer, [B]
+  // Append fused into the launch: one new token per sequence, k/v [B][H_kv][D]; nullptr = the
+  // cache already holds the token.  len then holds the lengths before the append and the kernel
+  // writes the new ones to len_out (a different array: CTAs read len at different times).
+  const uint16_t* new_k;
+  const uint16_t* new_v;
+  int32_t* len_out;
   const uint16_t* q;       // [B][H_q][D] queries of this layer
   const uint16_t* q_low;   // [B][H_q][D] queries of the block's lowest layer (== q if lowest)
   uint16_t* stash;         // where a lowest layer saves q for its block, else nullptr

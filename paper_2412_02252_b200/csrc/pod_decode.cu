@@ -198,8 +198,9 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // counters).
   pdl_wait();
   pdl_launch_dependents();
+  const bool fused = p.new_k != nullptr;      // this launch also appends one token per sequence
   if (!p.by_value) {
-    n = p.len[b];
+    n = p.len[b] + (fused ? 1 : 0);
     cap_d = y.seq_cap_d[b];
     seq_row = y.seq_row_base[b];
   }
@@ -269,6 +270,22 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     }
   };
 
+  // Rows that change in a fused launch are masked in the streamed tiles and added by one warp
+  // from registers: the new token's proximal row, and the distant row of the token it pushes
+  // out of the recent window.
+  int tA = -1, cA = 0, tB = -1, cB = 0, rA = -1, rB = -1;
+  if (fused) {
+    const int pos = n - 1;
+    if (pos < y.S) {
+      rA = pos;
+    } else {
+      rA = y.S + (pos - y.S) % y.W;
+      if (pos - y.W >= y.S) rB = pos - y.W - y.S;
+    }
+    tA = rA / TOK; cA = rA % TOK;
+    if (rB >= 0) { tB = ntp + rB / TOK; cB = rB % TOK; }
+  }
+
   int vt_q[NSTAGE];                               // tile held by each stage, -1 = none
 #pragma unroll
   for (int s = 0; s < NSTAGE; ++s) {
@@ -308,6 +325,66 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   uint32_t round = 0;                     // stage s holds its (round)-th tile: barrier parity round & 1
   int fail_stage = 0;
 
+  // ---- fused append: warp 0 of the head's first CTA moves the rows and adds their terms ------
+  if (fused && split == 0 && warp == 0) {
+    __shared__ __align__(16) uint16_t s_sp[4][128];     // new K, new V, displaced K, displaced V
+    constexpr int LPR = D / 8;                          // lanes per row, 16 bytes each
+    uint16_t* arena_w = const_cast<uint16_t*>(p.arena);
+    const bool lowest = (p.layer % y.G) == 0;
+    if (lane < 2 * LPR) {
+      const bool isv = lane >= LPR;
+      const int sub = lane % LPR;
+      const uint4 nw = *reinterpret_cast<const uint4*>((isv ? p.new_v : p.new_k) + ((int64_t)b * y.H_kv + kvh) * D + sub * 8);
+      uint4* slot = reinterpret_cast<uint4*>(arena_w + ((int64_t)(isv ? rowVp : rowKp) + rA) * D + sub * 8);
+      if (rB >= 0) {
+        // The slot's occupant leaves the window: its value row moves to the layer's distant values,
+        // its key row to the block's key store only from the lowest layer (other layers drop theirs
+        // and score the token with the block's key, written by the lowest layer's launch).
+        const uint4 old = *slot;
+        uint4* dst = reinterpret_cast<uint4*>(arena_w + ((int64_t)(isv ? rowVd : rowKd) + rB) * D + sub * 8);
+        uint4 use = old;
+        if (isv || lowest) *dst = old; else use = *dst;
+        *reinterpret_cast<uint4*>(&s_sp[isv ? 3 : 2][sub * 8]) = use;
+      }
+      *slot = nw;
+      *reinterpret_cast<uint4*>(&s_sp[isv ? 1 : 0][sub * 8]) = nw;
+    }
+    if (kvh == 0 && lane == 0) p.len_out[b] = n;
+    __syncwarp();
+    // one token: logit of head qrow from this lane's Q fragments (quad-reduced), then the same
+    // online-softmax update as a tile, in fp32
+    auto add_token = [&](const uint16_t* krow, const uint16_t* vrow, const uint32_t (&qf)[D / 16][2]) {
+      float dot = 0.f;
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const float2 q0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&qf[kk][0]));
+        const float2 q1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&qf[kk][1]));
+        const float2 k0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(krow + kk * 16 + qcol));
+        const float2 k1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(krow + kk * 16 + 8 + qcol));
+        dot += q0.x * k0.x + q0.y * k0.y + q1.x * k1.x + q1.y * k1.y;
+      }
+      dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+      dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+      const float a = dot * p.scale_log2;
+      const float m_new = fmaxf(m_row, a);
+      const float alpha = ex2(m_row - m_new);
+      const float pr = ex2(a - m_new);
+      m_row = m_new;
+      l_row = l_row * alpha + ((lane & 3) == 0 ? pr : 0.f);   // l_row holds per-lane partial sums
+      const float al0 = __shfl_sync(0xffffffffu, alpha, qcol * 4), al1 = __shfl_sync(0xffffffffu, alpha, qcol * 4 + 4);
+      const float p0 = __shfl_sync(0xffffffffu, pr, qcol * 4), p1 = __shfl_sync(0xffffffffu, pr, qcol * 4 + 4);
+#pragma unroll
+      for (int cb = 0; cb < D / 16; ++cb) {
+        const float v0 = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(vrow + cb * 16 + qrow));
+        const float v1 = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(vrow + cb * 16 + 8 + qrow));
+        ot[cb][0] = ot[cb][0] * al0 + p0 * v0; ot[cb][1] = ot[cb][1] * al1 + p1 * v0;
+        ot[cb][2] = ot[cb][2] * al0 + p0 * v1; ot[cb][3] = ot[cb][3] * al1 + p1 * v1;
+      }
+    };
+    add_token(s_sp[0], s_sp[1], qp);                    // the new token is proximal: own query
+    if (rB >= 0) add_token(s_sp[2], s_sp[3], qd);       // the displaced token is distant: block's query
+  }
+
   // ldmatrix lane addressing inside a [TOK][128 B] sub-tile with the 128-byte swizzle:
   // 16-byte chunk c of row t lives at t * 128 + ((c ^ (t & 7)) << 4).
   const int lm = lane >> 3, lr = lane & 7;
@@ -326,6 +403,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       if (!__all_sync(0xffffffffu, mbar_wait(bar0 + s * 8, round & 1))) { failed = true; fail_stage = s; continue; }
       const bool dist = vt >= ntp;
       const int cnt = dist ? min(TOK, n_d - (vt - ntp) * TOK) : min(TOK, n_p - vt * TOK);
+      const int mcol = vt == tA ? cA : (vt == tB ? cB : -1);    // column handled outside the stream
       const uint32_t ks = wbuf_s + s * C::STAGE_B;
       const uint32_t vs = ks + C::TILE_B;
 
@@ -362,10 +440,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
         mma16816(t1, c0, 0u, c2, 0u, kf[kk + 1][2], kf[kk + 1][3]);
       }
       // ---- online softmax (base 2) over this lane's row --------------------------------------
-      float a00 = (qcol < cnt) ? (s0[0] + t0[0]) * p.scale_log2 : -INFINITY;
-      float a01 = (qcol + 1 < cnt) ? (s0[1] + t0[1]) * p.scale_log2 : -INFINITY;
-      float a10 = (qcol + 8 < cnt) ? (s1[0] + t1[0]) * p.scale_log2 : -INFINITY;
-      float a11 = (qcol + 9 < cnt) ? (s1[1] + t1[1]) * p.scale_log2 : -INFINITY;
+      float a00 = (qcol < cnt && qcol != mcol) ? (s0[0] + t0[0]) * p.scale_log2 : -INFINITY;
+      float a01 = (qcol + 1 < cnt && qcol + 1 != mcol) ? (s0[1] + t0[1]) * p.scale_log2 : -INFINITY;
+      float a10 = (qcol + 8 < cnt && qcol + 8 != mcol) ? (s1[0] + t1[0]) * p.scale_log2 : -INFINITY;
+      float a11 = (qcol + 9 < cnt && qcol + 9 != mcol) ? (s1[1] + t1[1]) * p.scale_log2 : -INFINITY;
       float mx = fmaxf(fmaxf(a00, a01), fmaxf(a10, a11));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
@@ -380,7 +458,9 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
 #pragma unroll
         for (int cb = 0; cb < D / 16; ++cb) { ot[cb][0] *= al0; ot[cb][1] *= al1; ot[cb][2] *= al0; ot[cb][3] *= al1; }
       }
-      a00 = ex2(a00 - m_row); a01 = ex2(a01 - m_row); a10 = ex2(a10 - m_row); a11 = ex2(a11 - m_row);
+      // a tile whose only valid column is handled outside the stream leaves the maximum at -inf
+      const float m_use = (m_row == -INFINITY) ? 0.f : m_row;
+      a00 = ex2(a00 - m_use); a01 = ex2(a01 - m_use); a10 = ex2(a10 - m_use); a11 = ex2(a11 - m_use);
       l_row += (a00 + a01) + (a10 + a11);
       const uint32_t pb0 = pack_bf16(a00, a01), pb1 = pack_bf16(a10, a11);
       // ---- O^T += V^T P^T ----------------------------------------------------------------------

@@ -156,6 +156,34 @@ def test_decode_order_rules():
         assert e.value.status == B.POD_ERR_INVALID
 
 
+def test_fused_append_decode_order_and_capacity_rules():
+    """The one-launch form obeys the rules of write + decode, judged at the lengths after the append."""
+    cfg = _cfg(batch=2)
+    c = B.PodCache(cfg, [12, 40])
+    p = _fake_ptr()
+    for l in range(4):
+        for b in range(2):
+            c.write(l, b, p, p, 10)
+    with pytest.raises(B.PodError) as e:      # block's lowest layer has not run this step
+        c.append_decode_attn(1, p, p, p, p)
+    assert e.value.status == B.POD_ERR_ORDER
+    assert c.seq_len(0, 1) == 10              # a refused call changes nothing
+    assert c.append_decode_attn(0, p, p, p, p) == B.POD_DRY_RUN
+    assert c.seq_len(0, 0) == 11 and c.seq_len(1, 0) == 11
+    assert c.append_decode_attn(1, p, p, p, p) == B.POD_DRY_RUN
+    assert c.decode_attn(1, p, p) == B.POD_DRY_RUN          # same lengths, same stash: allowed again
+    assert c.append_decode_attn(0, p, p, p, p) == B.POD_DRY_RUN
+    with pytest.raises(B.PodError) as e:      # sequence 0 is full at 12
+        c.append_decode_attn(0, p, p, p, p)
+    assert e.value.status == B.POD_ERR_CAPACITY
+    assert c.seq_len(0, 0) == 12 and c.seq_len(1, 0) == 12
+    for args in [(0, 0, p, p, p), (0, p, 0, p, p), (0, p, p, 0, p), (0, p, p, p, 0), (9, p, p, p, p),
+                 (0, p + 2, p, p, p)]:
+        with pytest.raises(B.PodError) as e:
+            c.append_decode_attn(*args)
+        assert e.value.status == B.POD_ERR_INVALID
+
+
 def test_dense_configuration_needs_no_order():
     cfg = _cfg(group_size=1)
     c = B.PodCache(cfg, [64])
@@ -179,4 +207,5 @@ def test_null_handles():
     assert B.lib.pod_cache_seq_len(None, 0, 0) == B.POD_ERR_INVALID
     assert B.lib.pod_cache_reset(None, 0) == B.POD_ERR_INVALID
     assert B.lib.pod_decode_attn(None, 0, None, None, None) == B.POD_ERR_INVALID
+    assert B.lib.pod_append_decode_attn(None, 0, None, None, None, None, None) == B.POD_ERR_INVALID
     assert B.lib.pod_cache_write(None, 0, 0, None, None, 1, None) == B.POD_ERR_INVALID

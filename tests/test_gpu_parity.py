@@ -158,6 +158,55 @@ def test_decode_steps_with_window_rollover():
     assert cache.device_status() == B.POD_OK
 
 
+@pytest.mark.parametrize("d,G,lens0", [(128, 2, [30, 75, 9, 0, 3]), (64, 3, [19, 20, 21, 150]),
+                                       (128, 2, [5 * i for i in range(10)])])
+def test_fused_append_decode_steps(d, G, lens0):
+    """pod_append_decode_attn over many steps (first tokens, sink fill, ring fill, ring wraps, small
+    and large batches): outputs against the oracle, cache contents bit for bit against the
+    oracle's layout, which is maintained by plain appends."""
+    S, W = 4, 16
+    case = Case(seed=15, L=4, G=G, Hq=8, Hkv=2, d=d, S=S, W=W, lens=lens0, caps=[n + 40 for n in lens0])
+    cache = case.make_cache()
+    case.prefill(cache)
+    ocs = [_oracle_cache(case, b) for b in range(case.B)]
+    for b, oc in enumerate(ocs):
+        for l in range(case.L):
+            if lens0[b]:
+                oc.write(l, synth.bf16_bits(case.kv(synth.TAG_K, l, b, 0, lens0[b], "cpu")),
+                         synth.bf16_bits(case.kv(synth.TAG_V, l, b, 0, lens0[b], "cpu")))
+    stream = torch.cuda.current_stream().cuda_stream
+    for step in range(1, 40):
+        lens = [n + step for n in lens0]
+        outs = torch.empty(case.L, case.B, case.Hq, case.d, dtype=torch.bfloat16, device="cuda")
+        for l in range(case.L):
+            k = torch.stack([case.kv(synth.TAG_K, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            v = torch.stack([case.kv(synth.TAG_V, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            cache.append_decode_attn(l, k, v, case.q(l, step, "cuda"), outs[l], stream)
+            kb, vb = synth.bf16_bits(k), synth.bf16_bits(v)
+            for b, oc in enumerate(ocs):
+                oc.append(l, kb[b], vb[b])
+        torch.cuda.synchronize()
+        assert [cache.seq_len(b, 0) for b in range(case.B)] == lens
+        if step in (1, 2, 3, 4, 5, 16, 17, 20, 21, 22, 37, 39):
+            _check_all_heads(case, outs, step=step, lens=lens)
+            _compare_layout(case, cache, ocs)
+    assert cache.device_status() == B.POD_OK
+    # the two-call form continues from the state the fused form left (device lengths included)
+    step = 40
+    lens = [n + step for n in lens0]
+    outs = torch.empty(case.L, case.B, case.Hq, case.d, dtype=torch.bfloat16, device="cuda")
+    for l in range(case.L):
+        k = torch.stack([case.kv(synth.TAG_K, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+        v = torch.stack([case.kv(synth.TAG_V, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+        cache.write(l, -1, k, v, 1, stream)
+        cache.decode_attn(l, case.q(l, step, "cuda"), outs[l], stream)
+    torch.cuda.synchronize()
+    _check_all_heads(case, outs, step=step, lens=lens)
+    with pytest.raises(B.PodError) as e:
+        cache.append_decode_attn(0, k, v, case.q(0, 0, "cuda"), outs[0], stream)
+    assert e.value.status == B.POD_ERR_CAPACITY
+
+
 def test_custom_scale():
     case = Case(seed=6, L=2, G=2, Hq=4, Hkv=1, d=64, S=2, W=6, lens=[50], scale=0.31)
     cache = case.make_cache()
