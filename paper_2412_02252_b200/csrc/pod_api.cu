@@ -370,15 +370,13 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
   p.scale_log2 = c->scale * 1.4426950408889634f;
   {
     // Shared distant keys are read again by the next layer of the block within the same step.
-    // If the batch's key store of one block fits the L2 budget, ask L2 to keep those lines.
+    // Ask L2 to keep the first tiles of every head's key store, as many as the budget holds
+    // (all of them when the batch's store of one block is small enough).
     const int last_of_block = (low + g.group_size - 1 < g.n_layers - 1) ? low + g.group_size - 1 : g.n_layers - 1;
-    int64_t distk_bytes = 0;
-    const int64_t SW = (int64_t)g.n_sink + g.n_recent;
-    for (int b = 0; b < g.batch; ++b) {
-      const int64_t n = c->h_len(layer, b);
-      distk_bytes += (n > SW ? n - SW : 0) * g.n_kv_heads * g.head_dim * 2;
-    }
-    p.keep_distk = (layer < last_of_block && distk_bytes <= c->l2_keep_budget) ? 1 : 0;
+    const int64_t tile_bytes = (int64_t)decode_tile_tokens() * g.head_dim * 2;
+    const int64_t per_tile_index = (int64_t)g.batch * g.n_kv_heads * tile_bytes;   // one tile of every head
+    const int64_t keep = c->l2_keep_budget / per_tile_index;
+    p.keep_dist_tiles = layer < last_of_block ? (int32_t)(keep > 0x3fffffff ? 0x3fffffff : keep) : 0;
   }
   p.by_value = g.batch <= SMALL_BATCH ? 1 : 0;
   for (int b = 0; b < SMALL_BATCH; ++b) {

@@ -91,7 +91,8 @@ struct DecodeParams {
   float scale_log2;        // sm_scale * log2(e)
   // Small batches carry the per-sequence lengths and row offsets by value (the host mirrors the
   // device lengths exactly), which takes two dependent global loads off every CTA's start-up.
-  int32_t keep_distk;      // 1: later layers of the block re-read the distant keys this step: keep them in L2
+  int32_t keep_dist_tiles; // distant key tiles below this index are loaded with an L2 evict_last hint: later
+                           // layers of the block read them again in the same step
   int32_t by_value;        // 1: use the arrays below instead of len / seq_row_base / seq_cap_d
   int32_t v_len[SMALL_BATCH];
   int32_t v_cap_d[SMALL_BATCH];

@@ -192,7 +192,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   int64_t cap_d = p.v_cap_d[bv];
   int64_t seq_row = p.v_row_base[bv];
   const uint64_t pol_stream = policy_evict_first();
-  const uint64_t pol_distk = p.keep_distk ? policy_evict_last() : pol_stream;
+  const uint64_t pol_keep = policy_evict_last();
 
   // Everything below reads what earlier kernels of the stream wrote (lengths, cache rows, stash,
   // counters).
@@ -262,7 +262,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     const uint32_t bar = bar0 + stage * 8;
     const uint32_t dst = wbuf_s + stage * C::STAGE_B;
     mbar_expect_tx(bar, C::STAGE_B);
-    const uint64_t pol_k = dist ? pol_distk : pol_stream;
+    const uint64_t pol_k = (dist && vt - ntp < p.keep_dist_tiles) ? pol_keep : pol_stream;
 #pragma unroll
     for (int s = 0; s < C::NSUB; ++s) {
       tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yk, bar, pol_k);
