@@ -64,6 +64,11 @@ bool carve(const pod_config& c, const int32_t* cap, Carve* out) {
     out->seq_row_base[b] = rows;
     out->seq_cap_d[b] = (int32_t)cap_d;
     rows += (int64_t)c.n_layers * 2 * c.n_kv_heads * SW + ((int64_t)c.n_layers + n_blocks) * c.n_kv_heads * cap_d;
+    {                                  // shared distant logits (blocks of several layers only)
+      Layout y{};
+      y.H_q = c.n_q_heads; y.H_kv = c.n_kv_heads; y.D = c.head_dim; y.G = c.group_size;
+      rows += score_rows_per_seq(y, cap_d);
+    }
   }
   if (rows >= ((int64_t)1 << 31)) return false;   // tile coordinates are 32-bit row indices
   out->total_rows = rows;
@@ -93,7 +98,8 @@ struct pod_cache {
   bool dry = false;
   int last_cuda = 0;
   int sm_count = 148, resident = 2;
-  int64_t l2_keep_budget = 0;          // bytes of shared keys worth pinning in L2 (from the L2 size)
+  int score_block = -1;                // block whose distant logits the score store holds, -1 = none
+  std::vector<int32_t> score_len;      // [B] lengths at which they were stored
   int force_split_tokens = 0;          // POD_SPLIT_TOKENS > 0 overrides the planner
   int force_chunk_tiles = 0;           // POD_CHUNK_TILES > 0 overrides the tiles per draw
   int static_eighths = 5;              // POD_STATIC_EIGHTHS: share of a warp's chunks assigned without a draw
@@ -216,6 +222,7 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
   c->cap.assign(seq_capacity, seq_capacity + cfg->batch);
   c->len.assign((size_t)cfg->n_layers * cfg->batch, 0);
   c->len_cur.assign((size_t)cfg->n_layers, 0);
+  c->score_len.assign((size_t)cfg->batch, -1);
   c->stash_len.assign((size_t)c->cv.n_blocks * cfg->batch, -1);
   c->scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)cfg->head_dim);
   c->dry = cfg->device < 0;
@@ -257,9 +264,6 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
     return POD_ERR_CUDA;
   }
   c->sm_count = sm; c->resident = res;
-  int l2 = 0;
-  if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, cfg->device) == cudaSuccess) c->l2_keep_budget = (int64_t)l2 * 3 / 4;
-  if (const char* kb = getenv("POD_L2_KEEP_MB")) c->l2_keep_budget = (int64_t)atoi(kb) << 20;
   if (const char* ct = getenv("POD_CHUNK_TILES")) c->force_chunk_tiles = atoi(ct);
   if (const char* se = getenv("POD_STATIC_EIGHTHS")) {
     const int v = atoi(se);
@@ -368,15 +372,18 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     p.static_eighths = c->static_eighths;
   }
   p.scale_log2 = c->scale * 1.4426950408889634f;
-  {
-    // Shared distant keys are read again by the next layer of the block within the same step.
-    // Ask L2 to keep the first tiles of every head's key store, as many as the budget holds
-    // (all of them when the batch's store of one block is small enough).
-    const int last_of_block = (low + g.group_size - 1 < g.n_layers - 1) ? low + g.group_size - 1 : g.n_layers - 1;
-    const int64_t tile_bytes = (int64_t)decode_tile_tokens() * g.head_dim * 2;
-    const int64_t per_tile_index = (int64_t)g.batch * g.n_kv_heads * tile_bytes;   // one tile of every head
-    const int64_t keep = c->l2_keep_budget / per_tile_index;
-    p.keep_dist_tiles = layer < last_of_block ? (int32_t)(keep > 0x3fffffff ? 0x3fffffff : keep) : 0;
+  // Shared distant logits: a lowest layer of a block of several layers stores them; another
+  // layer reads them if they are the ones of its block at exactly these lengths, else it falls
+  // back to scoring the block's keys itself.
+  p.score_mode = 0;
+  if (g.group_size > 1) {
+    if (lowest) {
+      p.score_mode = 1;
+    } else if (c->score_block == block) {
+      bool same = true;
+      for (int b = 0; b < g.batch; ++b) same = same && c->score_len[b] == c->h_len(layer, b);
+      if (same) p.score_mode = 2;
+    }
   }
   p.by_value = g.batch <= SMALL_BATCH ? 1 : 0;
   for (int b = 0; b < SMALL_BATCH; ++b) {
@@ -406,6 +413,10 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     }
   }
   if (lowest) for (int b = 0; b < g.batch; ++b) sl[b] = c->h_len(layer, b);
+  if (p.score_mode == 1) {
+    c->score_block = block;
+    for (int b = 0; b < g.batch; ++b) c->score_len[b] = c->h_len(layer, b);
+  }
   c->last_split_tokens = plan.split_tokens; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;
   return POD_OK;
 }
@@ -455,6 +466,7 @@ int pod_cache_reset(pod_cache* c, int seq) {
   for (int blk = 0; blk < c->cv.n_blocks; ++blk)
     for (int b = b0; b < b1; ++b) c->stash_len[(size_t)blk * g.batch + b] = -1;
   c->memo_sum = -1;
+  c->score_block = -1;
   if (c->dry) return POD_DRY_RUN;
   cudaError_t e = cudaSetDevice(g.device);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();

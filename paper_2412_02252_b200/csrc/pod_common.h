@@ -36,6 +36,10 @@ constexpr int SCHED_TICKET = 16;      // [0] = chunk counter, [SCHED_TICKET] = f
 //   prox  [L][2 (K, V)][H_kv][n_s + n_r]     rows [0, n_s) = sink, row n_s + slot = ring slot
 //   distV [L][H_kv][cap_d[b]]                 index p - n_s
 //   distK [n_blocks][H_kv][cap_d[b]]          index p - n_s, key of the block's lowest layer
+//   guard [16]                                only when G > 1: rows that stay zero
+//   score [H_kv][score_rows_per_head]         only when G > 1: the distant logits of the block being
+//                                             decoded (fp32, log2 units), one group of 16 tokens x r
+//                                             query heads = r * 64 bytes in mma fragment order
 // with cap_d[b] = max(0, capacity[b] - n_s - n_r).  Sink and ring of one (layer, head) are
 // adjacent so that the proximal tokens of a head are one contiguous stream (the softmax does
 // not care about token order, so ring slots are read in slot order).
@@ -56,6 +60,26 @@ __host__ __device__ inline int64_t distv_row(const Layout& y, int layer, int hea
 }
 __host__ __device__ inline int64_t distk_row(const Layout& y, int block, int head, int64_t cap_d) {
   return dist_base_row(y) + (((int64_t)y.L + block) * y.H_kv + head) * cap_d;
+}
+
+// Bytes of one 16-token group of shared distant logits (r query heads), and rows one head's
+// groups take (a row is D bf16).
+__host__ __device__ inline int score_group_bytes(const Layout& y) { return (y.H_q / y.H_kv) * 64; }
+__host__ __device__ inline int64_t score_rows_per_head(const Layout& y, int64_t cap_d) {
+  if (y.G <= 1) return 0;
+  const int64_t bytes = ((cap_d + 15) / 16) * score_group_bytes(y);
+  return (bytes + y.D * 2 - 1) / (y.D * 2);
+}
+// Tiles of the decode kernel may extend up to 15 rows past a head's rows; everything they can
+// reach must be finite bf16.  The logits are fp32 (and may be -inf), so a guard of zero rows
+// separates them from the key and value rows before them.
+constexpr int SCORE_GUARD_ROWS = 16;
+__host__ __device__ inline int64_t score_rows_per_seq(const Layout& y, int64_t cap_d) {
+  return y.G <= 1 ? 0 : SCORE_GUARD_ROWS + y.H_kv * score_rows_per_head(y, cap_d);
+}
+__host__ __device__ inline int64_t score_row(const Layout& y, int head, int64_t cap_d) {
+  return dist_base_row(y) + ((int64_t)y.L + y.n_blocks) * y.H_kv * cap_d + SCORE_GUARD_ROWS +
+         head * score_rows_per_head(y, cap_d);
 }
 
 struct WriteParams {
@@ -91,8 +115,10 @@ struct DecodeParams {
   float scale_log2;        // sm_scale * log2(e)
   // Small batches carry the per-sequence lengths and row offsets by value (the host mirrors the
   // device lengths exactly), which takes two dependent global loads off every CTA's start-up.
-  int32_t keep_dist_tiles; // distant key tiles below this index are loaded with an L2 evict_last hint: later
-                           // layers of the block read them again in the same step
+  // Shared distant logits (Section 2.2: a block shares the attention scores of its lowest layer):
+  // 1 = this launch is a lowest layer and stores them, 2 = this launch reads them instead of the
+  // block's keys, 0 = neither (dense, or the stored logits belong to other lengths).
+  int32_t score_mode;
   int32_t by_value;        // 1: use the arrays below instead of len / seq_row_base / seq_cap_d
   int32_t v_len[SMALL_BATCH];
   int32_t v_cap_d[SMALL_BATCH];

@@ -77,17 +77,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tma
       ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar), "l"(policy)
       : "memory");
 }
-// L2 eviction policies.  Rows that are read once per decode step stream through with
-// evict_first; the block's shared distant keys are kept with evict_last while later layers of
-// the block will read them again in the same step.
+// L2 eviction policy: cache rows are read once per decode step and stream through with evict_first.
 __device__ __forceinline__ uint64_t policy_evict_first() {
   uint64_t p;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ uint64_t policy_evict_last() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
   return p;
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -192,7 +185,6 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   int64_t cap_d = p.v_cap_d[bv];
   int64_t seq_row = p.v_row_base[bv];
   const uint64_t pol_stream = policy_evict_first();
-  const uint64_t pol_keep = policy_evict_last();
 
   // Everything below reads what earlier kernels of the stream wrote (lengths, cache rows, stash,
   // counters).
@@ -224,6 +216,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int rowVp = (int)(seq_row + prox_row(y, p.layer, 1, kvh));
   const int rowKd = (int)(seq_row + distk_row(y, p.block, kvh, cap_d));
   const int rowVd = (int)(seq_row + distv_row(y, p.layer, kvh, cap_d));
+  // shared distant logits of this head: groups of 16 tokens x r heads, fp32, fragment order
+  const int sc_group_b = score_group_bytes(y);
+  unsigned char* sc_base = reinterpret_cast<unsigned char*>(const_cast<uint16_t*>(p.arena)) +
+                           (seq_row + score_row(y, kvh, cap_d)) * (int64_t)(D * 2);
+  const bool sc_write = p.score_mode == 1, sc_read = p.score_mode == 2;
 
   // ---- the warp's walk over its chunks (all values uniform across the warp) -----------------
   unsigned drawn = 0;                             // lane 0: result of the draw issued one chunk ahead
@@ -261,11 +258,17 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     const int yv = dist ? rowVd + (vt - ntp) * TOK : rowVp + vt * TOK;
     const uint32_t bar = bar0 + stage * 8;
     const uint32_t dst = wbuf_s + stage * C::STAGE_B;
+    if (dist && sc_read) {            // the block's logits stand in for the key rows
+      mbar_expect_tx(bar, C::TILE_B + sc_group_b);
+      bulk_load(dst, sc_base + (int64_t)(vt - ntp + dep) * sc_group_b, sc_group_b, bar);
+#pragma unroll
+      for (int s = 0; s < C::NSUB; ++s) tma_load_2d(dst + C::TILE_B + s * C::SUB_B, &tmap, s * 64, yv, bar, pol_stream);
+      return;
+    }
     mbar_expect_tx(bar, C::STAGE_B);
-    const uint64_t pol_k = (dist && vt - ntp < p.keep_dist_tiles) ? pol_keep : pol_stream;
 #pragma unroll
     for (int s = 0; s < C::NSUB; ++s) {
-      tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yk, bar, pol_k);
+      tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yk, bar, pol_stream);
       tma_load_2d(dst + C::TILE_B + s * C::SUB_B, &tmap, s * 64, yv, bar, pol_stream);
     }
   };
@@ -353,7 +356,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     __syncwarp();
     // one token: logit of head qrow from this lane's Q fragments (quad-reduced), then the same
     // online-softmax update as a tile, in fp32
-    auto add_token = [&](const uint16_t* krow, const uint16_t* vrow, const uint32_t (&qf)[D / 16][2]) {
+    auto add_token = [&](const uint16_t* krow, const uint16_t* vrow, const uint32_t (&qf)[D / 16][2], float* logit_dst) {
       float dot = 0.f;
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
@@ -366,6 +369,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       dot += __shfl_xor_sync(0xffffffffu, dot, 1);
       dot += __shfl_xor_sync(0xffffffffu, dot, 2);
       const float a = dot * p.scale_log2;
+      if (logit_dst != nullptr && (lane & 3) == 0 && qrow < r) *logit_dst = a;
       const float m_new = fmaxf(m_row, a);
       const float alpha = ex2(m_row - m_new);
       const float pr = ex2(a - m_new);
@@ -381,8 +385,12 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
         ot[cb][2] = ot[cb][2] * al0 + p0 * v1; ot[cb][3] = ot[cb][3] * al1 + p1 * v1;
       }
     };
-    add_token(s_sp[0], s_sp[1], qp);                    // the new token is proximal: own query
-    if (rB >= 0) add_token(s_sp[2], s_sp[3], qd);       // the displaced token is distant: block's query
+    add_token(s_sp[0], s_sp[1], qp, nullptr);           // the new token is proximal: own query
+    if (rB >= 0) {                                      // the displaced token is distant: block's query
+      float* slot = reinterpret_cast<float*>(sc_base + (int64_t)(rB / TOK) * sc_group_b + (qrow * 4 + ((cB & 7) >> 1)) * 16) +
+                    ((cB >> 3) * 2 + (cB & 1));
+      add_token(s_sp[2], s_sp[3], qd, sc_write ? slot : nullptr);
+    }
   }
 
   // ldmatrix lane addressing inside a [TOK][128 B] sub-tile with the 128-byte swizzle:
@@ -408,11 +416,17 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       const uint32_t vs = ks + C::TILE_B;
 
       // ---- the whole tile into registers, then hand the stage back --------------------------
+      const bool from_scores = dist && sc_read;
       uint32_t kf[D / 16][4], vf[D / 16][4];
+      float4 sc = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (from_scores) {
+        if (qrow < r) sc = lds_f32x4(ks + (qrow * 4 + (lane & 3)) * 16);
+      } else {
 #pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-        const int chunk = 2 * kk + k_chunk;          // 16-byte chunk of the row
-        ldsm4(ks + (chunk >> 3) * C::SUB_B + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), kf[kk]);
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const int chunk = 2 * kk + k_chunk;          // 16-byte chunk of the row
+          ldsm4(ks + (chunk >> 3) * C::SUB_B + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), kf[kk]);
+        }
       }
 #pragma unroll
       for (int cb = 0; cb < D / 16; ++cb) {
@@ -427,23 +441,41 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       vt_q[s] = next_tile();
       if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, dep);
 
-      // ---- S = Q K^T (two accumulation chains per token half) -------------------------------
-      float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-      float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};
+      // ---- S = Q K^T (two accumulation chains per token half), or the block's stored logits ----
+      float l00, l01, l10, l11;                        // logits in log2 units: tokens qcol, +1, +8, +9
+      if (from_scores) {
+        l00 = sc.x; l01 = sc.y; l10 = sc.z; l11 = sc.w;
+      } else {
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int kk = 0; kk < D / 16; kk += 2) {
-        const uint32_t a0 = dist ? qd[kk][0] : qp[kk][0], a2 = dist ? qd[kk][1] : qp[kk][1];
-        const uint32_t c0 = dist ? qd[kk + 1][0] : qp[kk + 1][0], c2 = dist ? qd[kk + 1][1] : qp[kk + 1][1];
-        mma16816(s0, a0, 0u, a2, 0u, kf[kk][0], kf[kk][1]);
-        mma16816(s1, a0, 0u, a2, 0u, kf[kk][2], kf[kk][3]);
-        mma16816(t0, c0, 0u, c2, 0u, kf[kk + 1][0], kf[kk + 1][1]);
-        mma16816(t1, c0, 0u, c2, 0u, kf[kk + 1][2], kf[kk + 1][3]);
+        for (int kk = 0; kk < D / 16; kk += 2) {
+          const uint32_t a0 = dist ? qd[kk][0] : qp[kk][0], a2 = dist ? qd[kk][1] : qp[kk][1];
+          const uint32_t c0 = dist ? qd[kk + 1][0] : qp[kk + 1][0], c2 = dist ? qd[kk + 1][1] : qp[kk + 1][1];
+          mma16816(s0, a0, 0u, a2, 0u, kf[kk][0], kf[kk][1]);
+          mma16816(s1, a0, 0u, a2, 0u, kf[kk][2], kf[kk][3]);
+          mma16816(t0, c0, 0u, c2, 0u, kf[kk + 1][0], kf[kk + 1][1]);
+          mma16816(t1, c0, 0u, c2, 0u, kf[kk + 1][2], kf[kk + 1][3]);
+        }
+        l00 = (s0[0] + t0[0]) * p.scale_log2; l01 = (s0[1] + t0[1]) * p.scale_log2;
+        l10 = (s1[0] + t1[0]) * p.scale_log2; l11 = (s1[1] + t1[1]) * p.scale_log2;
       }
       // ---- online softmax (base 2) over this lane's row --------------------------------------
-      float a00 = (qcol < cnt && qcol != mcol) ? (s0[0] + t0[0]) * p.scale_log2 : -INFINITY;
-      float a01 = (qcol + 1 < cnt && qcol + 1 != mcol) ? (s0[1] + t0[1]) * p.scale_log2 : -INFINITY;
-      float a10 = (qcol + 8 < cnt && qcol + 8 != mcol) ? (s1[0] + t1[0]) * p.scale_log2 : -INFINITY;
-      float a11 = (qcol + 9 < cnt && qcol + 9 != mcol) ? (s1[1] + t1[1]) * p.scale_log2 : -INFINITY;
+      float a00 = (qcol < cnt && qcol != mcol) ? l00 : -INFINITY;
+      float a01 = (qcol + 1 < cnt && qcol + 1 != mcol) ? l01 : -INFINITY;
+      float a10 = (qcol + 8 < cnt && qcol + 8 != mcol) ? l10 : -INFINITY;
+      float a11 = (qcol + 9 < cnt && qcol + 9 != mcol) ? l11 : -INFINITY;
+      if (dist && sc_write && qrow < r) {            // the other layers of the block reuse these logits
+        float* dst = reinterpret_cast<float*>(sc_base + (int64_t)(vt - ntp) * sc_group_b + (qrow * 4 + (lane & 3)) * 16);
+        if (mcol < 0) {
+          *reinterpret_cast<float4*>(dst) = make_float4(a00, a01, a10, a11);
+        } else {                                       // the column of the displaced token is written by warp 0
+          if (qcol != mcol) dst[0] = a00;
+          if (qcol + 1 != mcol) dst[1] = a01;
+          if (qcol + 8 != mcol) dst[2] = a10;
+          if (qcol + 9 != mcol) dst[3] = a11;
+        }
+      }
       float mx = fmaxf(fmaxf(a00, a01), fmaxf(a10, a11));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));

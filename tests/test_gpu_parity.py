@@ -207,6 +207,35 @@ def test_fused_append_decode_steps(d, G, lens0):
     assert e.value.status == B.POD_ERR_CAPACITY
 
 
+def test_shared_logits_fallback_and_mixed_calls():
+    """Layers other than a block's lowest reuse the lowest layer's distant logits when the stored
+    ones are theirs, and score the block's keys themselves when another block has been decoded in
+    between; one-launch and two-call forms may be mixed inside a block.  All against the oracle."""
+    lens0 = [90, 41]
+    case = Case(seed=16, L=4, G=2, Hq=8, Hkv=2, d=128, S=4, W=16, lens=lens0, caps=[n + 8 for n in lens0])
+    cache = case.make_cache()
+    case.prefill(cache)
+    stream = torch.cuda.current_stream().cuda_stream
+    outs = torch.empty(case.L, case.B, case.Hq, case.d, dtype=torch.bfloat16, device="cuda")
+    for l in (0, 2, 1, 3, 1):                 # layer 1 after block 1's lowest layer: fallback; layer 3, then 1 again
+        cache.decode_attn(l, case.q(l, 0, "cuda"), outs[l], stream)
+    torch.cuda.synchronize()
+    _check_all_heads(case, outs, step=0)
+    for step, fused_layers in ((1, (0, 2)), (2, (1, 3)), (3, (0, 1, 2, 3)), (4, ())):
+        lens = [n + step for n in lens0]
+        for l in range(case.L):
+            k = torch.stack([case.kv(synth.TAG_K, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            v = torch.stack([case.kv(synth.TAG_V, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            if l in fused_layers:
+                cache.append_decode_attn(l, k, v, case.q(l, step, "cuda"), outs[l], stream)
+            else:
+                cache.write(l, -1, k, v, 1, stream)
+                cache.decode_attn(l, case.q(l, step, "cuda"), outs[l], stream)
+        torch.cuda.synchronize()
+        _check_all_heads(case, outs, step=step, lens=lens)
+    assert cache.device_status() == B.POD_OK
+
+
 def test_custom_scale():
     case = Case(seed=6, L=2, G=2, Hq=4, Hkv=1, d=64, S=2, W=6, lens=[50], scale=0.31)
     cache = case.make_cache()
