@@ -36,7 +36,7 @@ constexpr int SCHED_TICKET = 16;      // [0] = chunk counter, [SCHED_TICKET] = f
 //   prox  [L][2 (K, V)][H_kv][n_s + n_r]     rows [0, n_s) = sink, row n_s + slot = ring slot
 //   distV [L][H_kv][cap_d[b]]                 index p - n_s
 //   distK [n_blocks][H_kv][cap_d[b]]          index p - n_s, key of the block's lowest layer
-//   guard [16]                                only when G > 1: rows that stay zero
+//   guard [32]                                only when G > 1: rows that stay zero
 //   score [H_kv][score_rows_per_head]         only when G > 1: the distant logits of the block being
 //                                             decoded (fp32, log2 units), one group of 16 tokens x r
 //                                             query heads = r * 64 bytes in mma fragment order
@@ -67,13 +67,13 @@ __host__ __device__ inline int64_t distk_row(const Layout& y, int block, int hea
 __host__ __device__ inline int score_group_bytes(const Layout& y) { return (y.H_q / y.H_kv) * 64; }
 __host__ __device__ inline int64_t score_rows_per_head(const Layout& y, int64_t cap_d) {
   if (y.G <= 1) return 0;
-  const int64_t bytes = ((cap_d + 15) / 16) * score_group_bytes(y);
+  const int64_t bytes = 2 * ((cap_d + 31) / 32) * score_group_bytes(y);   // read two groups at a time
   return (bytes + y.D * 2 - 1) / (y.D * 2);
 }
-// Tiles of the decode kernel may extend up to 15 rows past a head's rows; everything they can
+// Tiles of the decode kernel may extend up to 31 rows past a head's rows; everything they can
 // reach must be finite bf16.  The logits are fp32 (and may be -inf), so a guard of zero rows
 // separates them from the key and value rows before them.
-constexpr int SCORE_GUARD_ROWS = 16;
+constexpr int SCORE_GUARD_ROWS = 32;
 __host__ __device__ inline int64_t score_rows_per_seq(const Layout& y, int64_t cap_d) {
   return y.G <= 1 ? 0 : SCORE_GUARD_ROWS + y.H_kv * score_rows_per_head(y, cap_d);
 }

@@ -147,8 +147,10 @@ struct Cfg {
   static constexpr int STAGE_B = 2 * TILE_B;
   static constexpr int WARP_B = NSTAGE * STAGE_B;
   static constexpr int RING_B = NW * WARP_B;
+  static constexpr int SC_SLOT_B = 1024;              // per stage: logits of 32 tokens x up to 8 heads, fp32
+  static constexpr int SC_B = NW * NSTAGE * SC_SLOT_B;
   static constexpr int N_BARS = NW * NSTAGE + NW;     // one per stage, one per warp for the combine
-  static constexpr int SMEM = RING_B + N_BARS * 8 + 1024;   // + slack to align to 1024
+  static constexpr int SMEM = RING_B + SC_B + N_BARS * 8 + 1024;   // + slack to align to 1024
   // the combine reuses each warp's ring: (max, sum) pairs, split weights, then partial rows
   static constexpr int CML_OFF = 0, CW_OFF = MAX_SPLITS_CAP * 8, CROW_OFF = CW_OFF + MAX_SPLITS_CAP * 4;
   static constexpr int CROWS = (WARP_B - CROW_OFF) / (D * 4);   // partial rows per round
@@ -171,8 +173,9 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   unsigned char* wbuf = smem + warp * C::WARP_B;
   const uint32_t wbuf_s = smem_u32(wbuf);
-  const uint32_t bar0 = smem_u32(smem + C::RING_B) + warp * NSTAGE * 8;
-  const uint32_t cbar = smem_u32(smem + C::RING_B) + (NW * NSTAGE + warp) * 8;   // this warp's combine barrier
+  const uint32_t sc0 = smem_u32(smem + C::RING_B) + warp * NSTAGE * C::SC_SLOT_B;   // this warp's logit slots
+  const uint32_t bar0 = smem_u32(smem + C::RING_B + C::SC_B) + warp * NSTAGE * 8;
+  const uint32_t cbar = smem_u32(smem + C::RING_B + C::SC_B) + (NW * NSTAGE + warp) * 8;   // this warp's combine barrier
   if (lane == 0) {
     for (int s = 0; s < NSTAGE; ++s) mbar_init(bar0 + s * 8, 1);
     mbar_init(cbar, 1);
@@ -201,7 +204,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
 
   // ---- tiles and chunks of this (sequence, KV head) -----------------------------------------
   const int n_p = min(n, y.S + y.W), n_d = n - n_p;
-  const int ntp = (n_p + TOK - 1) / TOK, ntd = (n_d + TOK - 1) / TOK;
+  // A layer that reads the block's stored logits needs no key rows: its distant tiles hold 32
+  // value rows (both halves of a stage), so the bytes in flight per stage stay the same.
+  const bool sc_write = p.score_mode == 1, sc_read = p.score_mode == 2;
+  const int DT = sc_read ? 2 * TOK : TOK;         // tokens per distant tile
+  const int ntp = (n_p + TOK - 1) / TOK, ntd = (n_d + DT - 1) / DT;
   const int ntiles = ntp + ntd;
   const int tch = p.tiles_per_chunk;
   const int nwh = nsplit * NW;                    // warps working on this head
@@ -220,7 +227,6 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int sc_group_b = score_group_bytes(y);
   unsigned char* sc_base = reinterpret_cast<unsigned char*>(const_cast<uint16_t*>(p.arena)) +
                            (seq_row + score_row(y, kvh, cap_d)) * (int64_t)(D * 2);
-  const bool sc_write = p.score_mode == 1, sc_read = p.score_mode == 2;
 
   // ---- the warp's walk over its chunks (all values uniform across the warp) -----------------
   unsigned drawn = 0;                             // lane 0: result of the draw issued one chunk ahead
@@ -254,17 +260,21 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // arena; their logits are masked.  `dep` is zero; it carries a register dependency.
   auto issue = [&](int vt, int stage, int dep) {
     const bool dist = vt >= ntp;
-    const int yk = (dist ? rowKd + (vt - ntp) * TOK : rowKp + vt * TOK) + dep;
-    const int yv = dist ? rowVd + (vt - ntp) * TOK : rowVp + vt * TOK;
     const uint32_t bar = bar0 + stage * 8;
     const uint32_t dst = wbuf_s + stage * C::STAGE_B;
-    if (dist && sc_read) {            // the block's logits stand in for the key rows
-      mbar_expect_tx(bar, C::TILE_B + sc_group_b);
-      bulk_load(dst, sc_base + (int64_t)(vt - ntp + dep) * sc_group_b, sc_group_b, bar);
+    if (dist && sc_read) {            // 32 value rows + their logits; no key rows
+      const int yv0 = rowVd + (vt - ntp) * DT + dep;
+      mbar_expect_tx(bar, C::STAGE_B + 2 * sc_group_b);
+      bulk_load(sc0 + stage * C::SC_SLOT_B, sc_base + (int64_t)(vt - ntp) * 2 * sc_group_b, 2 * sc_group_b, bar);
 #pragma unroll
-      for (int s = 0; s < C::NSUB; ++s) tma_load_2d(dst + C::TILE_B + s * C::SUB_B, &tmap, s * 64, yv, bar, pol_stream);
+      for (int s = 0; s < C::NSUB; ++s) {
+        tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yv0, bar, pol_stream);
+        tma_load_2d(dst + C::TILE_B + s * C::SUB_B, &tmap, s * 64, yv0 + TOK, bar, pol_stream);
+      }
       return;
     }
+    const int yk = (dist ? rowKd + (vt - ntp) * TOK : rowKp + vt * TOK) + dep;
+    const int yv = dist ? rowVd + (vt - ntp) * TOK : rowVp + vt * TOK;
     mbar_expect_tx(bar, C::STAGE_B);
 #pragma unroll
     for (int s = 0; s < C::NSUB; ++s) {
@@ -286,7 +296,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       if (pos - y.W >= y.S) rB = pos - y.W - y.S;
     }
     tA = rA / TOK; cA = rA % TOK;
-    if (rB >= 0) { tB = ntp + rB / TOK; cB = rB % TOK; }
+    if (rB >= 0) { tB = ntp + rB / DT; cB = rB % DT; }
   }
 
   int vt_q[NSTAGE];                               // tile held by each stage, -1 = none
@@ -410,94 +420,111 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       if (vt < 0) { more = false; continue; }
       if (!__all_sync(0xffffffffu, mbar_wait(bar0 + s * 8, round & 1))) { failed = true; fail_stage = s; continue; }
       const bool dist = vt >= ntp;
-      const int cnt = dist ? min(TOK, n_d - (vt - ntp) * TOK) : min(TOK, n_p - vt * TOK);
-      const int mcol = vt == tA ? cA : (vt == tB ? cB : -1);    // column handled outside the stream
+      const bool from_scores = dist && sc_read;
+      const int rem = dist ? n_d - (vt - ntp) * DT : n_p - vt * TOK;      // valid rows from the tile's start
+      const int mtile = vt == tA ? cA : (vt == tB ? cB : -1);             // row handled outside the stream
       const uint32_t ks = wbuf_s + s * C::STAGE_B;
       const uint32_t vs = ks + C::TILE_B;
 
       // ---- the whole tile into registers, then hand the stage back --------------------------
-      const bool from_scores = dist && sc_read;
-      uint32_t kf[D / 16][4], vf[D / 16][4];
-      float4 sc = make_float4(0.f, 0.f, 0.f, 0.f);
+      // fa: key fragments, or (reading stored logits) value fragments of rows 0-15;
+      // fb: value fragments (of rows 16-31 when reading stored logits)
+      uint32_t fa[D / 16][4], fb[D / 16][4];
+      float4 sca = make_float4(0.f, 0.f, 0.f, 0.f), scb = sca;
       if (from_scores) {
-        if (qrow < r) sc = lds_f32x4(ks + (qrow * 4 + (lane & 3)) * 16);
+        if (qrow < r) {
+          sca = lds_f32x4(sc0 + s * C::SC_SLOT_B + (qrow * 4 + (lane & 3)) * 16);
+          scb = lds_f32x4(sc0 + s * C::SC_SLOT_B + sc_group_b + (qrow * 4 + (lane & 3)) * 16);
+        }
+#pragma unroll
+        for (int cb = 0; cb < D / 16; ++cb) {
+          const int chunk = 2 * cb + v_chunk;
+          ldsm4_t(ks + (chunk >> 3) * C::SUB_B + v_tok * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), fa[cb]);
+        }
       } else {
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const int chunk = 2 * kk + k_chunk;          // 16-byte chunk of the row
-          ldsm4(ks + (chunk >> 3) * C::SUB_B + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), kf[kk]);
+          ldsm4(ks + (chunk >> 3) * C::SUB_B + k_tok * 128 + (((chunk & 7) ^ (k_tok & 7)) << 4), fa[kk]);
         }
       }
 #pragma unroll
       for (int cb = 0; cb < D / 16; ++cb) {
         const int chunk = 2 * cb + v_chunk;
-        ldsm4_t(vs + (chunk >> 3) * C::SUB_B + v_tok * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), vf[cb]);
+        ldsm4_t(vs + (chunk >> 3) * C::SUB_B + v_tok * 128 + (((chunk & 7) ^ (v_tok & 7)) << 4), fb[cb]);
       }
       // The refill must not start before the last fragment load has returned (shared-memory
       // loads of a warp return in order): its row coordinate depends on that load's result.
       int dep;
-      asm volatile("and.b32 %0, %1, 0;" : "=r"(dep) : "r"(vf[D / 16 - 1][3]));
+      asm volatile("and.b32 %0, %1, 0;" : "=r"(dep) : "r"(fb[D / 16 - 1][3]));
       __syncwarp();
       vt_q[s] = next_tile();
       if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, dep);
 
-      // ---- S = Q K^T (two accumulation chains per token half), or the block's stored logits ----
-      float l00, l01, l10, l11;                        // logits in log2 units: tokens qcol, +1, +8, +9
+      // one online-softmax step (base 2) over 16 tokens: logits l (log2 units; tokens qcol, +1,
+      // +8, +9 of head qrow), `cnt` valid tokens, token `mcol` left out, value fragments vf
+      auto softmax_pv = [&](float l00, float l01, float l10, float l11, int cnt, int mcol, const uint32_t (&vf)[D / 16][4],
+                            float* store) {
+        float a00 = (qcol < cnt && qcol != mcol) ? l00 : -INFINITY;
+        float a01 = (qcol + 1 < cnt && qcol + 1 != mcol) ? l01 : -INFINITY;
+        float a10 = (qcol + 8 < cnt && qcol + 8 != mcol) ? l10 : -INFINITY;
+        float a11 = (qcol + 9 < cnt && qcol + 9 != mcol) ? l11 : -INFINITY;
+        if (store != nullptr) {                        // the other layers of the block reuse these logits
+          if (mcol < 0) {
+            *reinterpret_cast<float4*>(store) = make_float4(a00, a01, a10, a11);
+          } else {                                     // the displaced token's column is written by warp 0
+            if (qcol != mcol) store[0] = a00;
+            if (qcol + 1 != mcol) store[1] = a01;
+            if (qcol + 8 != mcol) store[2] = a10;
+            if (qcol + 9 != mcol) store[3] = a11;
+          }
+        }
+        float mx = fmaxf(fmaxf(a00, a01), fmaxf(a10, a11));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        if (__any_sync(0xffffffffu, mx > m_row)) {
+          const float m_new = fmaxf(m_row, mx);
+          const float alpha = ex2(m_row - m_new);     // 0 on the first tile, 1 if unchanged
+          m_row = m_new;
+          l_row *= alpha;
+          // the accumulators of this lane belong to heads qcol and qcol + 1
+          const float al0 = __shfl_sync(0xffffffffu, alpha, qcol * 4);
+          const float al1 = __shfl_sync(0xffffffffu, alpha, qcol * 4 + 4);
+#pragma unroll
+          for (int cb = 0; cb < D / 16; ++cb) { ot[cb][0] *= al0; ot[cb][1] *= al1; ot[cb][2] *= al0; ot[cb][3] *= al1; }
+        }
+        // a tile whose only valid column is handled outside the stream leaves the maximum at -inf
+        const float m_use = (m_row == -INFINITY) ? 0.f : m_row;
+        a00 = ex2(a00 - m_use); a01 = ex2(a01 - m_use); a10 = ex2(a10 - m_use); a11 = ex2(a11 - m_use);
+        l_row += (a00 + a01) + (a10 + a11);
+        const uint32_t pb0 = pack_bf16(a00, a01), pb1 = pack_bf16(a10, a11);
+        // O^T += V^T P^T
+#pragma unroll
+        for (int cb = 0; cb < D / 16; ++cb) mma16816(ot[cb], vf[cb][0], vf[cb][1], vf[cb][2], vf[cb][3], pb0, pb1);
+      };
+
       if (from_scores) {
-        l00 = sc.x; l01 = sc.y; l10 = sc.z; l11 = sc.w;
+        softmax_pv(sca.x, sca.y, sca.z, sca.w, min(TOK, rem), mtile, fa, nullptr);
+        if (rem > TOK) softmax_pv(scb.x, scb.y, scb.z, scb.w, min(TOK, rem - TOK), mtile - TOK, fb, nullptr);
       } else {
+        // S = Q K^T, two accumulation chains per token half
         float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
         float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int kk = 0; kk < D / 16; kk += 2) {
           const uint32_t a0 = dist ? qd[kk][0] : qp[kk][0], a2 = dist ? qd[kk][1] : qp[kk][1];
           const uint32_t c0 = dist ? qd[kk + 1][0] : qp[kk + 1][0], c2 = dist ? qd[kk + 1][1] : qp[kk + 1][1];
-          mma16816(s0, a0, 0u, a2, 0u, kf[kk][0], kf[kk][1]);
-          mma16816(s1, a0, 0u, a2, 0u, kf[kk][2], kf[kk][3]);
-          mma16816(t0, c0, 0u, c2, 0u, kf[kk + 1][0], kf[kk + 1][1]);
-          mma16816(t1, c0, 0u, c2, 0u, kf[kk + 1][2], kf[kk + 1][3]);
+          mma16816(s0, a0, 0u, a2, 0u, fa[kk][0], fa[kk][1]);
+          mma16816(s1, a0, 0u, a2, 0u, fa[kk][2], fa[kk][3]);
+          mma16816(t0, c0, 0u, c2, 0u, fa[kk + 1][0], fa[kk + 1][1]);
+          mma16816(t1, c0, 0u, c2, 0u, fa[kk + 1][2], fa[kk + 1][3]);
         }
-        l00 = (s0[0] + t0[0]) * p.scale_log2; l01 = (s0[1] + t0[1]) * p.scale_log2;
-        l10 = (s1[0] + t1[0]) * p.scale_log2; l11 = (s1[1] + t1[1]) * p.scale_log2;
+        float* store = nullptr;
+        if (dist && sc_write && qrow < r)
+          store = reinterpret_cast<float*>(sc_base + (int64_t)(vt - ntp) * sc_group_b + (qrow * 4 + (lane & 3)) * 16);
+        softmax_pv((s0[0] + t0[0]) * p.scale_log2, (s0[1] + t0[1]) * p.scale_log2, (s1[0] + t1[0]) * p.scale_log2,
+                   (s1[1] + t1[1]) * p.scale_log2, min(TOK, rem), mtile, fb, store);
       }
-      // ---- online softmax (base 2) over this lane's row --------------------------------------
-      float a00 = (qcol < cnt && qcol != mcol) ? l00 : -INFINITY;
-      float a01 = (qcol + 1 < cnt && qcol + 1 != mcol) ? l01 : -INFINITY;
-      float a10 = (qcol + 8 < cnt && qcol + 8 != mcol) ? l10 : -INFINITY;
-      float a11 = (qcol + 9 < cnt && qcol + 9 != mcol) ? l11 : -INFINITY;
-      if (dist && sc_write && qrow < r) {            // the other layers of the block reuse these logits
-        float* dst = reinterpret_cast<float*>(sc_base + (int64_t)(vt - ntp) * sc_group_b + (qrow * 4 + (lane & 3)) * 16);
-        if (mcol < 0) {
-          *reinterpret_cast<float4*>(dst) = make_float4(a00, a01, a10, a11);
-        } else {                                       // the column of the displaced token is written by warp 0
-          if (qcol != mcol) dst[0] = a00;
-          if (qcol + 1 != mcol) dst[1] = a01;
-          if (qcol + 8 != mcol) dst[2] = a10;
-          if (qcol + 9 != mcol) dst[3] = a11;
-        }
-      }
-      float mx = fmaxf(fmaxf(a00, a01), fmaxf(a10, a11));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      if (__any_sync(0xffffffffu, mx > m_row)) {
-        const float m_new = fmaxf(m_row, mx);
-        const float alpha = ex2(m_row - m_new);       // 0 on the first tile, 1 if unchanged
-        m_row = m_new;
-        l_row *= alpha;
-        // the accumulators of this lane belong to heads qcol and qcol + 1
-        const float al0 = __shfl_sync(0xffffffffu, alpha, qcol * 4);
-        const float al1 = __shfl_sync(0xffffffffu, alpha, qcol * 4 + 4);
-#pragma unroll
-        for (int cb = 0; cb < D / 16; ++cb) { ot[cb][0] *= al0; ot[cb][1] *= al1; ot[cb][2] *= al0; ot[cb][3] *= al1; }
-      }
-      // a tile whose only valid column is handled outside the stream leaves the maximum at -inf
-      const float m_use = (m_row == -INFINITY) ? 0.f : m_row;
-      a00 = ex2(a00 - m_use); a01 = ex2(a01 - m_use); a10 = ex2(a10 - m_use); a11 = ex2(a11 - m_use);
-      l_row += (a00 + a01) + (a10 + a11);
-      const uint32_t pb0 = pack_bf16(a00, a01), pb1 = pack_bf16(a10, a11);
-      // ---- O^T += V^T P^T ----------------------------------------------------------------------
-#pragma unroll
-      for (int cb = 0; cb < D / 16; ++cb) mma16816(ot[cb], vf[cb][0], vf[cb][1], vf[cb][2], vf[cb][3], pb0, pb1);
     }
   }
 
