@@ -98,6 +98,7 @@ struct pod_cache {
   bool dry = false;
   int last_cuda = 0;
   int sm_count = 148, resident = 2;
+  int last_decode_layer = -1;          // layer of the previous launch on this cache if it was a decode launch, else -1
   int score_block = -1;                // block whose distant logits the score store holds, -1 = none
   std::vector<int32_t> score_len;      // [B] lengths at which they were stored
   int force_split_tokens = 0;          // POD_SPLIT_TOKENS > 0 overrides the planner
@@ -310,6 +311,7 @@ int pod_cache_write(pod_cache* c, int layer, int seq, const void* k, const void*
   }
   for (int b = b0; b < b1; ++b) c->h_len(layer, b) += n_tokens;
   c->memo_sum = -1;
+  c->last_decode_layer = -1;
   return c->dry ? POD_DRY_RUN : POD_OK;
 }
 
@@ -385,6 +387,10 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
       if (same) p.score_mode = 2;
     }
   }
+  // A launch that appends and attends streams only rows written before this step (the new token's
+  // and the displaced token's rows are handled apart); the one launch that may still be running is
+  // the previous one on this cache, which touches other rows if it was a decode of another layer.
+  p.early_ok = (fused && c->last_decode_layer >= 0 && c->last_decode_layer != layer) ? 1 : 0;
   p.by_value = g.batch <= SMALL_BATCH ? 1 : 0;
   for (int b = 0; b < SMALL_BATCH; ++b) {
     const bool in = p.by_value && b < g.batch;
@@ -417,6 +423,7 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     c->score_block = block;
     for (int b = 0; b < g.batch; ++b) c->score_len[b] = c->h_len(layer, b);
   }
+  c->last_decode_layer = layer;
   c->last_split_tokens = plan.split_tokens; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;
   return POD_OK;
 }
@@ -467,6 +474,7 @@ int pod_cache_reset(pod_cache* c, int seq) {
     for (int b = b0; b < b1; ++b) c->stash_len[(size_t)blk * g.batch + b] = -1;
   c->memo_sum = -1;
   c->score_block = -1;
+  c->last_decode_layer = -1;
   if (c->dry) return POD_DRY_RUN;
   cudaError_t e = cudaSetDevice(g.device);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();

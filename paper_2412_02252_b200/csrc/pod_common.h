@@ -119,6 +119,9 @@ struct DecodeParams {
   // 1 = this launch is a lowest layer and stores them, 2 = this launch reads them instead of the
   // block's keys, 0 = neither (dense, or the stored logits belong to other lengths).
   int32_t score_mode;
+  int32_t early_ok;        // 1: no unfinished launch writes cache rows this launch streams (the two rows a
+                           //    fused launch changes itself aside): tiles may be requested before the
+                           //    wait for the previous kernel of the stream
   int32_t by_value;        // 1: use the arrays below instead of len / seq_row_base / seq_cap_d
   int32_t v_len[SMALL_BATCH];
   int32_t v_cap_d[SMALL_BATCH];

@@ -189,10 +189,17 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   int64_t seq_row = p.v_row_base[bv];
   const uint64_t pol_stream = policy_evict_first();
 
-  // Everything below reads what earlier kernels of the stream wrote (lengths, cache rows, stash,
-  // counters).
-  pdl_wait();
-  pdl_launch_dependents();
+  // The wait for the previous kernel of the stream comes before anything that kernel may have
+  // written is read: stash, counters, logits, the new token.  The cache rows and this layer's
+  // lengths are older when the host says so (early_ok: the previous launch on this cache was a decode
+  // launch of another layer); then the first tiles are requested before the wait, so that the
+  // memory latency of the start-up overlaps the previous kernel's tail.
+  bool waited = false;
+  if (!p.early_ok) {
+    pdl_wait();
+    pdl_launch_dependents();
+    waited = true;
+  }
   const bool fused = p.new_k != nullptr;      // this launch also appends one token per sequence
   if (!p.by_value) {
     n = p.len[b] + (fused ? 1 : 0);
@@ -229,8 +236,13 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
                            (seq_row + score_row(y, kvh, cap_d)) * (int64_t)(D * 2);
 
   // ---- the warp's walk over its chunks (all values uniform across the warp) -----------------
+  if (!waited && k_static * tch < NSTAGE) {       // the first tiles need draws: no early start
+    pdl_wait();
+    pdl_launch_dependents();
+    waited = true;
+  }
   unsigned drawn = 0;                             // lane 0: result of the draw issued one chunk ahead
-  if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+  if (waited && lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
   int c_id, c_t = 0, c_j = 0;
   bool walk_done = false;
   if (k_static > 0) {
@@ -258,14 +270,17 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   };
   // lane 0 only.  Rows past the segment are other (finite) cache rows, or zero fill past the
   // arena; their logits are masked.  `dep` is zero; it carries a register dependency.
-  auto issue = [&](int vt, int stage, int dep) {
+  // part 0: the whole tile; 1: all but the stored logits (before the wait); 2: the logits alone
+  auto issue = [&](int vt, int stage, int dep, int part) {
     const bool dist = vt >= ntp;
     const uint32_t bar = bar0 + stage * 8;
     const uint32_t dst = wbuf_s + stage * C::STAGE_B;
     if (dist && sc_read) {            // 32 value rows + their logits; no key rows
       const int yv0 = rowVd + (vt - ntp) * DT + dep;
-      mbar_expect_tx(bar, C::STAGE_B + 2 * sc_group_b);
-      bulk_load(sc0 + stage * C::SC_SLOT_B, sc_base + (int64_t)(vt - ntp) * 2 * sc_group_b, 2 * sc_group_b, bar);
+      if (part != 2) mbar_expect_tx(bar, C::STAGE_B + 2 * sc_group_b);
+      if (part != 1)
+        bulk_load(sc0 + stage * C::SC_SLOT_B, sc_base + (int64_t)(vt - ntp) * 2 * sc_group_b, 2 * sc_group_b, bar);
+      if (part == 2) return;
 #pragma unroll
       for (int s = 0; s < C::NSUB; ++s) {
         tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yv0, bar, pol_stream);
@@ -273,6 +288,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       }
       return;
     }
+    if (part == 2) return;
     const int yk = (dist ? rowKd + (vt - ntp) * TOK : rowKp + vt * TOK) + dep;
     const int yv = dist ? rowVd + (vt - ntp) * TOK : rowVp + vt * TOK;
     mbar_expect_tx(bar, C::STAGE_B);
@@ -303,7 +319,17 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
 #pragma unroll
   for (int s = 0; s < NSTAGE; ++s) {
     vt_q[s] = next_tile();
-    if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, 0);
+    if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, 0, waited ? 0 : 1);
+  }
+  if (!waited) {
+    pdl_wait();
+    pdl_launch_dependents();
+    if (lane == 0) {
+#pragma unroll
+      for (int s = 0; s < NSTAGE; ++s)
+        if (vt_q[s] >= 0) issue(vt_q[s], s, 0, 2);
+      drawn = (unsigned)atomicAdd(sched, 1);
+    }
   }
 
   // a lowest layer saves its query for the other layers of the block
@@ -459,7 +485,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       asm volatile("and.b32 %0, %1, 0;" : "=r"(dep) : "r"(fb[D / 16 - 1][3]));
       __syncwarp();
       vt_q[s] = next_tile();
-      if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, dep);
+      if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, dep, 0);
 
       // one online-softmax step (base 2) over 16 tokens: logits l (log2 units; tokens qcol, +1,
       // +8, +9 of head qrow), `cnt` valid tokens, token `mcol` left out, value fragments vf

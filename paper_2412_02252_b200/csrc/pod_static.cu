@@ -130,6 +130,7 @@ extern "C" int pod_dense_decode_attn_static(const void* kv_device, int capacity,
   p.static_eighths = 5;
   p.scale_log2 = (sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim)) * 1.4426950408889634f;
   p.score_mode = 0;
+  p.early_ok = 0;
   p.by_value = 1;
   p.v_len[0] = n_tokens; p.v_cap_d[0] = 0; p.v_row_base[0] = 0;
 
