@@ -301,7 +301,19 @@ def run_ours(args):
     us_layer = agg["us_per_layer_step"]
     hbm_peak, peak_kind = _peaks()
     n_avg = n + args.warmup + args.steps / 2.0
-    alg_bytes = Bn * 2 * n_avg * Hkv * d * 2              # K row-set + V row-set of every token
+    row = d * 2
+    n_p = min(n_avg, S + W)
+    n_d = n_avg - n_p
+    # Algorithmic bytes of one launch.  A block's lowest layer (every layer when G = 1) reads one key
+    # and one value row-set per token and, when the block has more layers, stores the distant logits
+    # (4 bytes per query head and distant token); the other layers read the value row-sets, the
+    # proximal key row-sets and those logits.
+    logit_bytes = n_d * Hq * 4 if G > 1 else 0
+    bytes_low = Bn * (2 * n_avg * Hkv * row + logit_bytes)
+    bytes_other = Bn * (n_avg * Hkv * row + n_p * Hkv * row + logit_bytes)
+    n_low = (L + G - 1) // G
+    alg_bytes = (n_low * bytes_low + (L - n_low) * bytes_other) / L
+    dense_bytes = Bn * 2 * n_avg * Hkv * row              # what a per-layer K+V cache would read
     # the timed region holds nothing but launches of the one kernel: its average duration
     per_us = ms * 1e3 / n_launch
     achieved = alg_bytes / (per_us * 1e-6) / 1e9
@@ -314,6 +326,7 @@ def run_ours(args):
         "config": {"workload": args.workload, "batch_per_gpu": Bn, "context": n_now, "layers": L,
                    "group_size": G, "q_heads": Hq, "kv_heads": Hkv, "head_dim": d, "n_sink": S,
                    "n_recent": W, "l2": "inputs larger than L2 (a step reads %.1f GiB)" % (L * alg_bytes / 2**30),
+                   "launches_per_step": "%d lowest-layer + %d other" % (n_low, L - n_low),
                    "split_tokens": geo["split_tokens"], "ctas": geo["n_ctas"]},
         "decode_tokens_per_s": round(agg["decode_tokens_per_s"], 1),
         "hbm_gbs_step": round(L * alg_bytes / (ms * 1e-3 / args.steps) / 1e9, 1),
@@ -321,7 +334,11 @@ def run_ours(args):
                      "frac": round(achieved / hbm_peak, 4), "traffic": traffic, "peak_kind": peak_kind,
                      "kernel": "pod_decode_splitk_kernel (append + split-K + combine in one launch)",
                      "us_per_launch": round(per_us, 3),
-                     "algorithmic_bytes_per_call": int(alg_bytes), "frac_of_8TBs": round(achieved / 8000.0, 4)},
+                     "algorithmic_bytes_per_launch": int(alg_bytes),
+                     "algorithmic_bytes_lowest_layer_launch": int(bytes_low),
+                     "algorithmic_bytes_other_layer_launch": int(bytes_other),
+                     "frac_of_8TBs": round(achieved / 8000.0, 4),
+                     "dense_equivalent_gbs": round(dense_bytes / (per_us * 1e-6) / 1e9, 1)},
         "e2e": {"value": round(e2e_ms * 1e3 / (e2e_steps * L * world), 3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": n_launch,
