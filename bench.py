@@ -249,18 +249,19 @@ def run_ours(args):
     dk, dv, dq = torch.empty_like(ks[0]), torch.empty_like(vs[0]), torch.empty_like(qs[0])
     hout = torch.empty(L, Bn, Hq, d, dtype=torch.bfloat16).pin_memory()
 
-    dkl, dvl, dql = [dk[l] for l in range(L)], [dv[l] for l in range(L)], [dq[l] for l in range(L)]
-    hkl = [[hk[i, l] for l in range(L)] for i in range(n_in)]
-    hvl = [[hv[i, l] for l in range(L)] for i in range(n_in)]
-    hql = [[hq[i, l] for l in range(L)] for i in range(n_in)]
+    dkp = [dk[l].data_ptr() for l in range(L)]
+    dvp = [dv[l].data_ptr() for l in range(L)]
+    dqp = [dq[l].data_ptr() for l in range(L)]
 
     def e2e_step(s):
+        """One step through the public call with host buffers: the step's k, v, q of every layer go up
+        in three copies from pinned memory, one launch per layer, the outputs come back."""
         i = s % n_in
+        dk.copy_(hk[i], non_blocking=True)
+        dv.copy_(hv[i], non_blocking=True)
+        dq.copy_(hq[i], non_blocking=True)
         for l in range(L):
-            dkl[l].copy_(hkl[i][l], non_blocking=True)
-            dvl[l].copy_(hvl[i][l], non_blocking=True)
-            dql[l].copy_(hql[i][l], non_blocking=True)
-            cache.append_decode_attn(l, dkl[l], dvl[l], dql[l], op[l], stream)
+            cache.append_decode_attn(l, dkp[l], dvp[l], dqp[l], op[l], stream)
         hout.copy_(outs, non_blocking=True)
         torch.cuda.current_stream().synchronize()      # the caller needs the outputs on the host
 
@@ -435,7 +436,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3-8b-32k", choices=sorted(WORKLOADS))

@@ -80,7 +80,9 @@ typedef struct {
 
 /* Bytes of device memory a cache with these per-sequence capacities (tokens, [batch]) needs:
  * the regions of every sequence at capacity plus library scratch (device lengths, the
- * per-block query stash, split-K partials).  Returns 0 on invalid arguments.  Host only. */
+ * per-block query stash, split-K partials and, when group_size > 1, the distant logits a block's
+ * lowest layer leaves for the block's other layers: 4 bytes per query head and distant token).
+ * Returns 0 on invalid arguments.  Host only. */
 size_t pod_cache_required_bytes(const pod_config* cfg, const int32_t* seq_capacity);
 
 /* Creates a cache.  arena: device memory of at least pod_cache_required_bytes, 256-byte

@@ -23,15 +23,24 @@
 //   * values: O^T[d x 8] += V^T[d x 16] P^T[16 x 8]: the channels are the M dimension, so no
 //     accumulator row is padding; the exponentials in the accumulator layout of S are exactly
 //     the B fragments, V^T fragments come from ldmatrix.trans.
+//   * shared distant scores (Section 2.2: the layers of a block share the attention scores of the
+//     lowest layer): a lowest layer of a block with several layers stores its distant logits as it
+//     computes them; the other layers read them (r * 64 bytes per 16 tokens) in place of the key
+//     rows and skip Q K^T.  Their distant tiles hold 32 value rows, so a stage carries the same
+//     bytes either way.
+// A launch may also do the append of the step's token (pod_append_decode_attn): warp 0 of a head's
+// first CTA copies the new rows in, moves the displaced rows to the distant stores and adds the
+// terms of those two tokens from registers, while every streaming warp masks those two rows.
 // Warps merge through shared memory; the CTA writes one fp32 partial (acc, max, sum) per query
 // head, takes a ticket of its (sequence, KV head), and the CTA that draws the last ticket merges
-// all partials (the gate of Eq. 2 generalised from two parts to n_splits parts): it pulls them
-// into shared memory with bulk async copies, so the merge costs one memory round trip instead of
-// one per split.  Nobody waits for anybody, so nothing can hang; every mbarrier wait is
-// bounded and a wait that gives up raises the cache's error flag.
+// all partials (the gate of Eq. 2 generalised from two parts to n_splits parts): each of its warps
+// pulls one query head's partials into shared memory with bulk async copies, so the merge costs
+// one memory round trip instead of one per split.  Nobody waits for anybody, so nothing can hang;
+// every mbarrier wait is bounded and a wait that gives up raises the cache's error flag.
 // The kernels are launched with programmatic stream serialization: everything above
-// griddepcontrol.wait (barrier setup, policies) overlaps the tail of the previous kernel in the
-// stream.
+// griddepcontrol.wait overlaps the tail of the previous kernel in the stream -- barrier setup
+// always, and the requests for the first tiles when the host knows that no unfinished launch
+// writes the rows they read.
 #include <cuda_bf16.h>
 
 #include "pod_common.h"

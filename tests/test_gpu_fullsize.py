@@ -75,7 +75,8 @@ def test_config3_batch16_32k():
 
 def test_config5_ragged_serving_mix():
     """32 sequences of 4096..65536 tokens (seeded), G = 2, S = 16, W = 2048: prefill of every full
-    sequence, then 16 decode steps (append one token per sequence and layer, decode every layer)."""
+    sequence, then 16 decode steps (append one token per sequence and layer, decode every layer),
+    alternating between the one-launch form and the two-call form."""
     if _free_gb() < 140:
         pytest.skip("needs 140 GiB of free device memory")
     seed, steps = 5, 16
@@ -93,10 +94,13 @@ def test_config5_ragged_serving_mix():
         for l in range(case.L):
             k = torch.stack([case.kv(synth.TAG_K, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
             v = torch.stack([case.kv(synth.TAG_V, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
-            cache.write(l, -1, k, v, 1, stream)
-            cache.decode_attn(l, case.q(l, step, "cuda"), outs[l], stream)
+            if step % 2:                       # odd steps as one launch per layer, even steps as two calls
+                cache.append_decode_attn(l, k, v, case.q(l, step, "cuda"), outs[l], stream)
+            else:
+                cache.write(l, -1, k, v, 1, stream)
+                cache.decode_attn(l, case.q(l, step, "cuda"), outs[l], stream)
         torch.cuda.synchronize()
-        if step in (1, 9, steps):
+        if step in (1, 8, 9, steps):
             triples = [(short, 0, 0), (short, 1, 3), (long_, 30, 8), (long_, 31, 8)]
             triples += [(int(rng.integers(32)), int(rng.integers(32)), int(rng.integers(32))) for _ in range(4)]
             _sample_check(case, outs, triples, step=step, lens=lens)
