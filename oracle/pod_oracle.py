@@ -18,6 +18,13 @@ sum to one; pure-Python brute force; hand-worked rational example; planted-key c
 shared-score invariance; incremental layout == layout built from the history; byte counts
 against the closed form and the paper's own saving arithmetic.
 
+Blocks are per head (Section 2.1, Algorithm 1: every head gets its own partition of the
+layers into runs of consecutive similar layers).  A partition is carried as a "lowest map"
+low[l][h] = lowest layer of the block that holds layer l for KV head h; ``group_size`` is the
+special case in which every head uses runs of G layers.  greedy_layer_blocks is Algorithm 1.
+Pins of these: hand-worked grouping example, the algorithm's defining properties checked by
+brute force, uniform maps == group_size, per-head independence, byte counts by enumeration.
+
 Readings of points the paper leaves open are listed next to the code that takes them.
 """
 from __future__ import annotations
@@ -39,6 +46,67 @@ def bits_to_f64(bits: np.ndarray) -> np.ndarray:
 def lowest_layer(layer: int, group_size: int) -> int:
     """Blocks are runs of ``group_size`` consecutive layers (0-based); the last may be short."""
     return layer - layer % group_size
+
+
+def uniform_lowest_map(n_layers: int, n_kv_heads: int, group_size: int) -> np.ndarray:
+    """low[l][h] for blocks of ``group_size`` consecutive layers, the same for every head."""
+    return np.array([[lowest_layer(l, group_size)] * n_kv_heads for l in range(n_layers)], dtype=np.int64)
+
+
+def check_lowest_map(low) -> np.ndarray:
+    """A lowest map describes, per head, a partition of the layers into runs of consecutive
+    layers: low[0][h] = 0 and low[l][h] is either l (a new block starts) or low[l-1][h]."""
+    low = np.asarray(low, dtype=np.int64)
+    L, H = low.shape
+    for h in range(H):
+        for l in range(L):
+            ok = low[l, h] == l or (l > 0 and low[l, h] == low[l - 1, h])
+            if not ok:
+                raise ValueError(f"not a partition into consecutive runs at layer {l}, head {h}")
+    return low
+
+
+def greedy_layer_blocks(sim, threshold=0.5):
+    """Algorithm 1 (Section 2.1): bottom-up greedy grouping of consecutive similar layers, per head.
+
+    sim: [H][L][L], sim[h][a][b] = similarity of layers a and b for head h (1 = identical).
+    For each head the first layer opens a block; every next layer joins the current (last)
+    block if it is similar (>= threshold) to ALL layers already in it, else it opens a new one.
+    Returns, per head, the list of blocks, each a list of 0-based layers.
+    """
+    sim = np.asarray(sim, dtype=np.float64)
+    H, L, _ = sim.shape
+    head_wise_layer_blocks = []
+    for h in range(H):
+        current_head_layer_blocks = [[0]]
+        for l in range(1, L):
+            current_block = current_head_layer_blocks[-1]
+            if all(sim[h, l, lh] >= threshold for lh in current_block):
+                current_block.append(l)
+            else:
+                current_head_layer_blocks.append([l])
+        head_wise_layer_blocks.append(current_head_layer_blocks)
+    return head_wise_layer_blocks
+
+
+def lowest_map_from_blocks(head_wise_layer_blocks, n_layers: int) -> np.ndarray:
+    """low[l][h] from the per-head block lists of greedy_layer_blocks."""
+    H = len(head_wise_layer_blocks)
+    low = np.full((n_layers, H), -1, dtype=np.int64)
+    for h, blocks in enumerate(head_wise_layer_blocks):
+        for block in blocks:
+            for l in block:
+                low[l, h] = block[0]
+    return check_lowest_map(low)
+
+
+def _resolve_map(n_layers, n_kv_heads, group_size, lowest):
+    if lowest is not None:
+        low = check_lowest_map(lowest)
+        if low.shape != (n_layers, n_kv_heads):
+            raise ValueError("lowest map must be [n_layers][n_kv_heads]")
+        return low
+    return uniform_lowest_map(n_layers, n_kv_heads, group_size)
 
 
 def is_proximal(p: int, n: int, n_s: int, n_r: int) -> bool:
@@ -107,24 +175,26 @@ def _softmax(a):
 # --------------------------------------------------------------------------------------
 # all heads of one layer, full history
 # --------------------------------------------------------------------------------------
-def pod_decode_layer(q, K, V, layer, *, group_size, n_s, n_r, scale=None, form="joint"):
+def pod_decode_layer(q, K, V, layer, *, group_size=None, lowest=None, n_s, n_r, scale=None, form="joint"):
     """One layer's decode attention for one sequence from the uncompressed history.
 
-    q: [L][H_q][d] queries of every layer at this step (only rows ``layer`` and its block's
-    lowest layer are read); K, V: [L][n][H_kv][d].  Query head h reads KV head h // r,
+    q: [L][H_q][d] queries of every layer at this step (only rows ``layer`` and its blocks'
+    lowest layers are read); K, V: [L][n][H_kv][d].  Blocks: ``group_size`` (runs of G layers for
+    every head) or ``lowest`` (a per-head lowest map [L][H_kv]).  Query head h reads KV head h // r,
     r = H_q / H_kv (grouped-query attention).  Returns o [H_q][d] (float64).
     An empty history (n == 0) gives zeros (convention of this build; the paper is silent).
     """
     L, n, H_kv, d = K.shape
     H_q = q.shape[1]
     r = H_q // H_kv
-    a = lowest_layer(layer, group_size)
+    low = _resolve_map(L, H_kv, group_size, lowest)
     out = np.zeros((H_q, d))
     if n == 0:
         return out
     fn = pod_attention_joint if form == "joint" else pod_attention_gate
     for h in range(H_q):
         kv = h // r
+        a = int(low[layer, kv])                 # lowest layer of this head's block
         out[h], _ = fn(q[layer, h], q[a, h], K[layer, :, kv], K[a, :, kv], V[layer, :, kv],
                        n_s, n_r, scale)
     return out
@@ -149,12 +219,17 @@ class PodCacheOracle:
     only when l is the lowest layer of its block and is discarded otherwise.
     """
 
-    def __init__(self, n_layers, n_kv_heads, head_dim, group_size, n_s, n_r, capacity):
+    def __init__(self, n_layers, n_kv_heads, head_dim, group_size, n_s, n_r, capacity, lowest=None):
         self.L, self.H, self.d = n_layers, n_kv_heads, head_dim
         self.G, self.S, self.W = group_size, n_s, n_r
         self.cap = capacity
         self.cap_d = max(0, capacity - n_s - n_r)
-        self.n_blocks = (n_layers + group_size - 1) // group_size
+        self.low = _resolve_map(n_layers, n_kv_heads, group_size, lowest)
+        # blocks of a head in layer order; block_of[l][h] = index of (l, h)'s block in that list
+        self.blocks = [sorted(set(int(x) for x in self.low[:, h])) for h in range(n_kv_heads)]
+        self.block_of = np.array([[self.blocks[h].index(int(self.low[l, h])) for h in range(n_kv_heads)]
+                                  for l in range(n_layers)])
+        self.n_blocks = max(len(b) for b in self.blocks)      # most blocks any head has
         z = lambda *s: np.zeros(s, dtype=np.uint16)
         self.sinkK = z(self.L, self.H, n_s, head_dim)
         self.sinkV = z(self.L, self.H, n_s, head_dim)
@@ -179,8 +254,9 @@ class PodCacheOracle:
             old = p - W
             if old >= S:                                   # leaves the recent window
                 self.distV[layer, :, old - S] = self.ringV[layer, :, slot]
-                if layer % self.G == 0:                    # keys survive once per block
-                    self.distK[layer // self.G, :, old - S] = self.ringK[layer, :, slot]
+                for h in range(self.H):
+                    if self.low[layer, h] == layer:        # keys survive once per block
+                        self.distK[self.block_of[layer, h], h, old - S] = self.ringK[layer, h, slot]
             self.ringK[layer, :, slot] = k_row
             self.ringV[layer, :, slot] = v_row
         self.len[layer] = p + 1
@@ -194,7 +270,9 @@ class PodCacheOracle:
     def valid_rows(self, region, index, head):
         """Valid rows of a region for one head, in region order, as uint16 [count][d],
         together with the first region index they start at."""
-        n = self.len[index * self.G if region == "distK" else index]
+        if region == "distK" and index >= len(self.blocks[head]):
+            return self.distK[index, head, :0], 0          # this head has fewer blocks
+        n = self.len[self.blocks[head][index] if region == "distK" else index]
         S, W = self.S, self.W
         n_d = max(0, n - S - W)
         if region in ("sinkK", "sinkV"):
@@ -208,8 +286,8 @@ class PodCacheOracle:
     def attend(self, layer, q, q_low, scale=None):
         """Decode attention of ``layer`` computed from the regions.
 
-        q: [H_q][d] float64 queries of this layer; q_low: [H_q][d] queries of the block's
-        lowest layer at the same step.  Token order inside the softmax is sink, ring slots,
+        q: [H_q][d] float64 queries of this layer; q_low: [H_q][d], row h = the query of head h
+        at the lowest layer of that head's block at the same step.  Token order inside the softmax is sink, ring slots,
         distant; the softmax does not depend on it.  Returns o [H_q][d] float64.
         """
         S, W, G = self.S, self.W, self.G
@@ -220,9 +298,9 @@ class PodCacheOracle:
         out = np.zeros((H_q, self.d))
         if n == 0:
             return out
-        g = layer // G
-        if self.len[g * G] != n:
-            raise ValueError("layers of a block must hold the same number of tokens")
+        for kv in range(self.H):
+            if self.len[int(self.low[layer, kv])] != n:
+                raise ValueError("layers of a block must hold the same number of tokens")
         n_sink, n_ring, n_d = min(n, S), min(W, max(0, n - S)), max(0, n - S - W)
         for h in range(H_q):
             kv = h // r
@@ -230,7 +308,7 @@ class PodCacheOracle:
                                              self.ringK[layer, kv, :n_ring]]))
             Vp = bits_to_f64(np.concatenate([self.sinkV[layer, kv, :n_sink],
                                              self.ringV[layer, kv, :n_ring]]))
-            Kd = bits_to_f64(self.distK[g, kv, :n_d])
+            Kd = bits_to_f64(self.distK[self.block_of[layer, kv], kv, :n_d])
             Vd = bits_to_f64(self.distV[layer, kv, :n_d])
             a = np.concatenate([(Kp @ q[h]) * scale, (Kd @ q_low[h]) * scale])
             e = np.exp(a - a.max())
@@ -239,11 +317,11 @@ class PodCacheOracle:
         return out
 
 
-def layout_from_history(K_bits, V_bits, *, group_size, n_s, n_r, capacity):
+def layout_from_history(K_bits, V_bits, *, group_size=None, lowest=None, n_s, n_r, capacity):
     """The regions as a function of the full history, written out directly (no appends):
     K_bits, V_bits uint16 [L][n][H_kv][d].  Used to check the incremental update rule."""
     L, n, H, d = K_bits.shape
-    c = PodCacheOracle(L, H, d, group_size, n_s, n_r, capacity)
+    c = PodCacheOracle(L, H, d, group_size, n_s, n_r, capacity, lowest=lowest)
     for l in range(L):
         for p in range(n):
             kr, vr = K_bits[l, p], V_bits[l, p]
@@ -254,8 +332,9 @@ def layout_from_history(K_bits, V_bits, *, group_size, n_s, n_r, capacity):
                 c.ringK[l, :, s], c.ringV[l, :, s] = kr, vr
             else:
                 c.distV[l, :, p - n_s] = vr
-                if l % group_size == 0:
-                    c.distK[l // group_size, :, p - n_s] = kr
+                for h in range(H):
+                    if c.low[l, h] == l:
+                        c.distK[c.block_of[l, h], h, p - n_s] = kr[h]
         c.len[l] = n
     return c
 
@@ -263,7 +342,7 @@ def layout_from_history(K_bits, V_bits, *, group_size, n_s, n_r, capacity):
 # --------------------------------------------------------------------------------------
 # byte accounting
 # --------------------------------------------------------------------------------------
-def pod_cache_bytes(lens, *, n_layers, n_kv_heads, head_dim, group_size, n_s, n_r,
+def pod_cache_bytes(lens, *, n_layers, n_kv_heads, head_dim, group_size=None, lowest=None, n_s, n_r,
                     elem_bytes=2):
     """(live PoD bytes, dense-equivalent bytes) for sequences of the given lengths.
 
@@ -271,19 +350,25 @@ def pod_cache_bytes(lens, *, n_layers, n_kv_heads, head_dim, group_size, n_s, n_
     once per block (abstract; Section 2.2).  Dense keeps K and V of all tokens in all layers.
     """
     row = head_dim * elem_bytes
-    n_blocks = (n_layers + group_size - 1) // group_size
+    low = _resolve_map(n_layers, n_kv_heads, group_size, lowest)
+    # (layer, head) pairs that are the lowest layer of their block keep their distant keys
+    n_key_stores = int(sum(low[l, h] == l for l in range(n_layers) for h in range(n_kv_heads)))
     live = dense = 0
     for n in lens:
         n_p = min(n, n_s + n_r)
         n_d = n - n_p
-        live += n_kv_heads * row * (n_layers * (2 * n_p + n_d) + n_blocks * n_d)
+        live += row * (n_kv_heads * n_layers * (2 * n_p + n_d) + n_key_stores * n_d)
         dense += n_kv_heads * row * n_layers * 2 * n
     return live, dense
 
 
-def pod_saving_closed_form(n, *, n_layers, group_size, n_s, n_r):
+def pod_saving_closed_form(n, *, n_layers, group_size=None, n_s, n_r, shared_fraction=None):
     """Fraction of dense KV bytes saved at length n: half of the bytes are keys, a fraction
-    n_d/n of them belongs to distant tokens, and of those only one layer per block remains."""
+    n_d/n of them belongs to distant tokens, and of those only one layer per block remains.
+    ``shared_fraction``: fraction of (layer, head) pairs that are not the lowest layer of their
+    block, for head-wise blocks; with ``group_size`` it is 1 - ceil(L/G)/L."""
     n_d = max(0, n - n_s - n_r)
-    n_blocks = (n_layers + group_size - 1) // group_size
-    return (n_d / n) * (1.0 - n_blocks / n_layers) / 2.0
+    if shared_fraction is None:
+        n_blocks = (n_layers + group_size - 1) // group_size
+        shared_fraction = 1.0 - n_blocks / n_layers
+    return (n_d / n) * shared_fraction / 2.0
