@@ -60,7 +60,7 @@ extern "C" {
 #define POD_REGION_SINK_V 1
 #define POD_REGION_RING_K 2 /* [layer][kv_head][n_r][d]            slot (p - n_s) % n_r  */
 #define POD_REGION_RING_V 3
-#define POD_REGION_DIST_K 4 /* [block][kv_head][capacity-n_s-n_r][d] index p - n_s, key of the block's lowest layer */
+#define POD_REGION_DIST_K 4 /* [block of that head][kv_head][capacity-n_s-n_r][d] index p - n_s, key of the block's lowest layer */
 #define POD_REGION_DIST_V 5 /* [layer][kv_head][capacity-n_s-n_r][d] index p - n_s       */
 
 typedef struct pod_cache pod_cache; /* opaque: host bookkeeping + device arena */
@@ -93,6 +93,33 @@ size_t pod_cache_required_bytes(const pod_config* cfg, const int32_t* seq_capaci
  * multiple of 128 bytes.  Errors: INVALID, ARENA, CUDA. */
 int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity,
                      void* arena_device, size_t arena_bytes, pod_cache** out);
+
+/* Head-wise blocks (Section 2.1, "Layer Grouping Strategy" and Algorithm 1: every head gets its own
+ * partition of the layers into blocks of consecutive similar layers).  lowest_layer is a host
+ * array [n_layers][n_kv_heads]: lowest_layer[l][h] = lowest layer of the block that holds layer l
+ * for KV head h (all query heads of a KV head follow it).  It must describe runs of consecutive
+ * layers: lowest_layer[0][h] = 0 and lowest_layer[l][h] is l or lowest_layer[l-1][h].
+ * cfg->group_size is ignored by these two calls; everything else is as in pod_cache_required_bytes
+ * and pod_cache_create, which are the special case lowest_layer[l][h] = l - l % group_size.
+ * With head-wise blocks a layer may be the lowest of the block for some heads and not for others:
+ * pod_decode_attn then needs, for every head whose block started lower, that lower layer decoded
+ * at the same lengths before (POD_ERR_ORDER otherwise), exactly as for uniform blocks.
+ * For POD_REGION_DIST_K the index passed to pod_cache_read_region counts the blocks of that head. */
+size_t pod_cache_required_bytes_blocks(const pod_config* cfg, const int32_t* seq_capacity,
+                                       const int32_t* lowest_layer);
+int pod_cache_create_blocks(const pod_config* cfg, const int32_t* seq_capacity,
+                            const int32_t* lowest_layer, void* arena_device, size_t arena_bytes,
+                            pod_cache** out);
+
+/* Greedy layer grouping (Algorithm 1), on the host: sim is [n_heads][n_layers][n_layers] with
+ * sim[h][a][b] the similarity of the attention of layers a and b for head h (Section 2.1: 1 =
+ * identical).  For each head, layer 0 opens a block; every next layer joins the current block if
+ * its similarity to EVERY layer already in that block is >= threshold (the paper uses 0.5), else
+ * it opens a new block.  Writes lowest_layer [n_layers][n_heads], ready for
+ * pod_cache_create_blocks.  Computing sim (Section 2.1, from attention maps of a trained model) is
+ * outside this library.  Errors: INVALID. */
+int pod_greedy_layer_blocks(const float* sim, int n_heads, int n_layers, float threshold,
+                            int32_t* lowest_layer);
 
 /* Frees host state (and the arena if the library allocated it).  Synchronises the device. */
 int pod_cache_destroy(pod_cache* c);

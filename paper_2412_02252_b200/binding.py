@@ -41,6 +41,9 @@ def _load() -> ctypes.CDLL:
     sig = {
         "pod_cache_required_bytes": (c_size_t, [P(pod_config), P(c_int32)]),
         "pod_cache_create": (c_int, [P(pod_config), P(c_int32), c_void_p, c_size_t, P(c_void_p)]),
+        "pod_cache_required_bytes_blocks": (c_size_t, [P(pod_config), P(c_int32), P(c_int32)]),
+        "pod_cache_create_blocks": (c_int, [P(pod_config), P(c_int32), P(c_int32), c_void_p, c_size_t, P(c_void_p)]),
+        "pod_greedy_layer_blocks": (c_int, [P(c_float), c_int, c_int, c_float, P(c_int32)]),
         "pod_cache_destroy": (c_int, [c_void_p]),
         "pod_cache_write": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_void_p]),
         "pod_decode_attn": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
@@ -63,7 +66,8 @@ def _load() -> ctypes.CDLL:
 
 
 lib = _load()
-EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_destroy", "pod_cache_write",
+EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_required_bytes_blocks",
+           "pod_cache_create_blocks", "pod_greedy_layer_blocks", "pod_cache_destroy", "pod_cache_write",
            "pod_decode_attn", "pod_append_decode_attn", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
            "pod_cache_read_region", "pod_cache_device_status", "pod_cache_last_cuda_error",
            "pod_cache_last_launch", "pod_strerror", "pod_dense_decode_attn_static"]
@@ -102,21 +106,46 @@ def _caps(cfg: pod_config, seq_capacity):
     return (c_int32 * cfg.batch)(*caps)
 
 
-def pod_cache_required_bytes(cfg: pod_config, seq_capacity) -> int:
-    return lib.pod_cache_required_bytes(ctypes.byref(cfg), _caps(cfg, seq_capacity))
+def _lowest(cfg: pod_config, lowest_layer):
+    """[n_layers][n_kv_heads] nested sequence (or array) -> flat c_int32 array."""
+    flat = [int(x) for row in lowest_layer for x in row]
+    if len(flat) != cfg.n_layers * cfg.n_kv_heads:
+        raise ValueError("lowest_layer must be [n_layers][n_kv_heads]")
+    return (c_int32 * len(flat))(*flat)
+
+
+def pod_cache_required_bytes(cfg: pod_config, seq_capacity, lowest_layer=None) -> int:
+    if lowest_layer is None:
+        return lib.pod_cache_required_bytes(ctypes.byref(cfg), _caps(cfg, seq_capacity))
+    return lib.pod_cache_required_bytes_blocks(ctypes.byref(cfg), _caps(cfg, seq_capacity), _lowest(cfg, lowest_layer))
+
+
+def pod_greedy_layer_blocks(sim, threshold: float = 0.5):
+    """sim: nested sequence / array [n_heads][n_layers][n_layers]; returns lowest_layer as a list
+    [n_layers][n_heads] of ints."""
+    H, L = len(sim), len(sim[0])
+    flat = (c_float * (H * L * L))(*[float(x) for a in sim for row in a for x in row])
+    out = (c_int32 * (L * H))()
+    _check(lib.pod_greedy_layer_blocks(flat, H, L, threshold, out), "pod_greedy_layer_blocks")
+    return [[out[l * H + h] for h in range(H)] for l in range(L)]
 
 
 class PodCache:
     """Owner of one ``pod_cache*``; methods carry the C names without the prefix."""
 
-    def __init__(self, cfg: pod_config, seq_capacity, arena=None):
+    def __init__(self, cfg: pod_config, seq_capacity, arena=None, lowest_layer=None):
         self.cfg = cfg
         self._arena = arena                       # keeps the caller's tensor alive
         handle = c_void_p()
         nbytes = 0 if arena is None else arena.numel() * arena.element_size()
-        st = lib.pod_cache_create(ctypes.byref(cfg), _caps(cfg, seq_capacity), _ptr(arena), nbytes,
-                                  ctypes.byref(handle))
-        _check(st, "pod_cache_create")
+        if lowest_layer is None:
+            st = lib.pod_cache_create(ctypes.byref(cfg), _caps(cfg, seq_capacity), _ptr(arena), nbytes,
+                                      ctypes.byref(handle))
+            _check(st, "pod_cache_create")
+        else:
+            st = lib.pod_cache_create_blocks(ctypes.byref(cfg), _caps(cfg, seq_capacity), _lowest(cfg, lowest_layer),
+                                             _ptr(arena), nbytes, ctypes.byref(handle))
+            _check(st, "pod_cache_create_blocks")
         self._h = handle
 
     def destroy(self):

@@ -41,18 +41,53 @@ int max_splits_for(const pod_config& c) {
   return (per + 1) & ~1;   // even: the combine's bulk copies move 16-byte multiples
 }
 
+// Per-head partition of the layers into blocks of consecutive layers (Section 2.1, Algorithm 1).
+struct BlockMap {
+  std::vector<int32_t> low;        // [L][H_kv] lowest layer of the block of (layer, head)
+  std::vector<int32_t> slot;       // [L][H_kv] key-store index of that block; a head's stores are adjacent
+  std::vector<int32_t> head_base;  // [H_kv + 1] first key store of each head
+  int n_slots = 0;
+  bool shared = false;             // some block has more than one layer
+};
+
+// low[l][h] must be l (a block starts) or low[l-1][h] (the block goes on); low[0][h] = 0.
+bool build_block_map(const pod_config& c, const int32_t* lowest, BlockMap* m) {
+  const int L = c.n_layers, H = c.n_kv_heads;
+  m->low.resize((size_t)L * H);
+  m->slot.resize((size_t)L * H);
+  m->head_base.assign((size_t)H + 1, 0);
+  m->shared = false;
+  for (int l = 0; l < L; ++l)
+    for (int h = 0; h < H; ++h) {
+      const int v = lowest ? lowest[(size_t)l * H + h] : l - l % c.group_size;
+      const bool ok = v == l || (l > 0 && v == m->low[(size_t)(l - 1) * H + h]);
+      if (!ok) return false;
+      m->low[(size_t)l * H + h] = v;
+      if (v != l) m->shared = true;
+    }
+  int next = 0;
+  for (int h = 0; h < H; ++h) {
+    m->head_base[h] = next;
+    for (int l = 0; l < L; ++l) {
+      if (m->low[(size_t)l * H + h] == l) ++next;
+      m->slot[(size_t)l * H + h] = next - 1;
+    }
+  }
+  m->head_base[H] = next;
+  m->n_slots = next;
+  return true;
+}
+
 struct Carve {
   std::vector<int64_t> seq_row_base;   // rows
   std::vector<int32_t> seq_cap_d;
-  size_t off_len, off_rowbase, off_capd, off_stash, off_pacc, off_pml, off_err, off_sched, total;
+  size_t off_len, off_rowbase, off_capd, off_low, off_slot, off_stash, off_pacc, off_pml, off_err, off_sched, total;
   int64_t total_rows;
-  int n_blocks, max_splits;
+  int max_splits;
 };
 
-bool carve(const pod_config& c, const int32_t* cap, Carve* out) {
+bool carve(const pod_config& c, const BlockMap& m, const int32_t* cap, Carve* out) {
   const int64_t row_bytes = (int64_t)c.head_dim * 2;
-  const int n_blocks = (c.n_layers + c.group_size - 1) / c.group_size;
-  out->n_blocks = n_blocks;
   out->max_splits = max_splits_for(c);
   out->seq_row_base.resize(c.batch);
   out->seq_cap_d.resize(c.batch);
@@ -63,10 +98,10 @@ bool carve(const pod_config& c, const int32_t* cap, Carve* out) {
     const int64_t cap_d = cap[b] > SW ? cap[b] - SW : 0;
     out->seq_row_base[b] = rows;
     out->seq_cap_d[b] = (int32_t)cap_d;
-    rows += (int64_t)c.n_layers * 2 * c.n_kv_heads * SW + ((int64_t)c.n_layers + n_blocks) * c.n_kv_heads * cap_d;
-    {                                  // shared distant logits (blocks of several layers only)
+    rows += (int64_t)c.n_layers * 2 * c.n_kv_heads * SW + ((int64_t)c.n_layers * c.n_kv_heads + m.n_slots) * cap_d;
+    {                                  // shared distant logits (only when some block has several layers)
       Layout y{};
-      y.H_q = c.n_q_heads; y.H_kv = c.n_kv_heads; y.D = c.head_dim; y.G = c.group_size;
+      y.H_q = c.n_q_heads; y.H_kv = c.n_kv_heads; y.D = c.head_dim; y.shared = m.shared ? 1 : 0;
       rows += score_rows_per_seq(y, cap_d);
     }
   }
@@ -76,7 +111,9 @@ bool carve(const pod_config& c, const int32_t* cap, Carve* out) {
   out->off_len = off;      off = align_up(off + (size_t)2 * c.n_layers * c.batch * 4);   // two copies, see len_cur
   out->off_rowbase = off;  off = align_up(off + (size_t)c.batch * 8);
   out->off_capd = off;     off = align_up(off + (size_t)c.batch * 4);
-  out->off_stash = off;    off = align_up(off + (size_t)n_blocks * c.batch * c.n_q_heads * row_bytes);
+  out->off_low = off;      off = align_up(off + (size_t)c.n_layers * c.n_kv_heads * 4);
+  out->off_slot = off;     off = align_up(off + (size_t)c.n_layers * c.n_kv_heads * 4);
+  out->off_stash = off;    off = align_up(off + (size_t)m.n_slots * c.batch * (c.n_q_heads / c.n_kv_heads) * row_bytes);
   out->off_pacc = off;     off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * c.head_dim * 4);
   out->off_pml = off;      off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * 2 * 4);
   out->off_err = off;      off = align_up(off + 4);
@@ -91,7 +128,8 @@ struct pod_cache {
   pod_config cfg;
   std::vector<int32_t> cap;            // [B]
   std::vector<int32_t> len;            // host mirror [L][B]
-  std::vector<int32_t> stash_len;      // [n_blocks][B]: lengths at which the block's q was stashed, -1 = none
+  std::vector<int32_t> stash_len;      // [n_slots][B]: lengths at which a block's q was stashed, -1 = none
+  BlockMap bm;
   Carve cv;
   unsigned char* arena = nullptr;
   bool owns_arena = false;
@@ -99,8 +137,8 @@ struct pod_cache {
   int last_cuda = 0;
   int sm_count = 148, resident = 2;
   int last_decode_layer = -1;          // layer of the previous launch on this cache if it was a decode launch, else -1
-  int score_block = -1;                // block whose distant logits the score store holds, -1 = none
-  std::vector<int32_t> score_len;      // [B] lengths at which they were stored
+  std::vector<int32_t> score_low;      // [H_kv] lowest layer whose distant logits the head's score store holds, -1 = none
+  std::vector<int32_t> score_len;      // [H_kv][B] lengths at which they were stored
   int force_split_tokens = 0;          // POD_SPLIT_TOKENS > 0 overrides the planner
   int force_chunk_tiles = 0;           // POD_CHUNK_TILES > 0 overrides the tiles per draw
   int static_eighths = 5;              // POD_STATIC_EIGHTHS: share of a warp's chunks assigned without a draw
@@ -122,6 +160,8 @@ struct pod_cache {
   int32_t* d_len(int layer) const { return d_len_copy(layer, len_cur[layer]); }
   int32_t& h_len(int layer, int b) { return len[(size_t)layer * cfg.batch + b]; }
   int32_t h_len(int layer, int b) const { return len[(size_t)layer * cfg.batch + b]; }
+  int low_of(int layer, int head) const { return bm.low[(size_t)layer * cfg.n_kv_heads + head]; }
+  int slot_of(int layer, int head) const { return bm.slot[(size_t)layer * cfg.n_kv_heads + head]; }
 };
 
 namespace {
@@ -204,33 +244,44 @@ const char* pod_strerror(int status) {
   }
 }
 
-size_t pod_cache_required_bytes(const pod_config* cfg, const int32_t* seq_capacity) {
+static size_t required_bytes_impl(const pod_config* cfg, const int32_t* seq_capacity, const int32_t* lowest) {
   if (!config_ok(cfg) || !seq_capacity) return 0;
+  BlockMap bm;
   Carve cv;
-  if (!carve(*cfg, seq_capacity, &cv)) return 0;
+  if (!build_block_map(*cfg, lowest, &bm) || !carve(*cfg, bm, seq_capacity, &cv)) return 0;
   return cv.total;
 }
 
-int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* arena_device,
-                     size_t arena_bytes, pod_cache** out) {
+size_t pod_cache_required_bytes(const pod_config* cfg, const int32_t* seq_capacity) {
+  return required_bytes_impl(cfg, seq_capacity, nullptr);
+}
+
+size_t pod_cache_required_bytes_blocks(const pod_config* cfg, const int32_t* seq_capacity,
+                                       const int32_t* lowest_layer) {
+  return lowest_layer ? required_bytes_impl(cfg, seq_capacity, lowest_layer) : 0;
+}
+
+static int create_impl(const pod_config* cfg, const int32_t* seq_capacity, const int32_t* lowest,
+                       void* arena_device, size_t arena_bytes, pod_cache** out) {
   if (!out) return POD_ERR_INVALID;
   *out = nullptr;
   if (!config_ok(cfg) || !seq_capacity) return POD_ERR_INVALID;
   pod_cache* c = new (std::nothrow) pod_cache();
   if (!c) return POD_ERR_INVALID;
   c->cfg = *cfg;
-  if (!carve(*cfg, seq_capacity, &c->cv)) { delete c; return POD_ERR_INVALID; }
+  if (!build_block_map(*cfg, lowest, &c->bm) || !carve(*cfg, c->bm, seq_capacity, &c->cv)) { delete c; return POD_ERR_INVALID; }
   c->cap.assign(seq_capacity, seq_capacity + cfg->batch);
   c->len.assign((size_t)cfg->n_layers * cfg->batch, 0);
   c->len_cur.assign((size_t)cfg->n_layers, 0);
-  c->score_len.assign((size_t)cfg->batch, -1);
-  c->stash_len.assign((size_t)c->cv.n_blocks * cfg->batch, -1);
+  c->score_low.assign((size_t)cfg->n_kv_heads, -1);
+  c->score_len.assign((size_t)cfg->n_kv_heads * cfg->batch, -1);
+  c->stash_len.assign((size_t)c->bm.n_slots * cfg->batch, -1);
   c->scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)cfg->head_dim);
   c->dry = cfg->device < 0;
   Layout& y = c->y;
   y.L = cfg->n_layers; y.H_kv = cfg->n_kv_heads; y.H_q = cfg->n_q_heads; y.D = cfg->head_dim;
-  y.G = cfg->group_size; y.S = cfg->n_sink; y.W = cfg->n_recent; y.B = cfg->batch;
-  y.n_blocks = c->cv.n_blocks;
+  y.S = cfg->n_sink; y.W = cfg->n_recent; y.B = cfg->batch;
+  y.n_slots = c->bm.n_slots; y.shared = c->bm.shared ? 1 : 0;
   if (c->dry) { *out = c; return POD_OK; }
 
   cudaError_t e = cudaSetDevice(cfg->device);
@@ -247,6 +298,8 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
   }
   y.seq_row_base = reinterpret_cast<const int64_t*>(c->arena + c->cv.off_rowbase);
   y.seq_cap_d = reinterpret_cast<const int32_t*>(c->arena + c->cv.off_capd);
+  y.low = reinterpret_cast<const int32_t*>(c->arena + c->cv.off_low);
+  y.slot = reinterpret_cast<const int32_t*>(c->arena + c->cv.off_slot);
   bool ok = true;
   // Tiles of the decode kernel may extend past the rows a head holds into neighbouring rows;
   // their logits are masked, but the rows must hold finite numbers, so the arena starts zeroed.
@@ -254,6 +307,8 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
   ok = ok && make_tensor_map(c);
   ok = ok && cudaMemcpy(c->arena + c->cv.off_rowbase, c->cv.seq_row_base.data(), (size_t)cfg->batch * 8, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->arena + c->cv.off_capd, c->cv.seq_cap_d.data(), (size_t)cfg->batch * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->arena + c->cv.off_low, c->bm.low.data(), c->bm.low.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->arena + c->cv.off_slot, c->bm.slot.data(), c->bm.slot.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess;
   int sm = 0;
   ok = ok && cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess;
   const int res = ok ? decode_resident_ctas_per_sm(cfg->head_dim) : 0;
@@ -273,6 +328,37 @@ int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* a
   const char* fst = getenv("POD_SPLIT_TOKENS");
   c->force_split_tokens = fst ? atoi(fst) : 0;
   *out = c;
+  return POD_OK;
+}
+
+int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity, void* arena_device,
+                     size_t arena_bytes, pod_cache** out) {
+  return create_impl(cfg, seq_capacity, nullptr, arena_device, arena_bytes, out);
+}
+
+int pod_cache_create_blocks(const pod_config* cfg, const int32_t* seq_capacity, const int32_t* lowest_layer,
+                            void* arena_device, size_t arena_bytes, pod_cache** out) {
+  if (out) *out = nullptr;
+  if (!lowest_layer) return POD_ERR_INVALID;
+  return create_impl(cfg, seq_capacity, lowest_layer, arena_device, arena_bytes, out);
+}
+
+// Algorithm 1 (Section 2.1): for each head, layer 0 opens a block; each next layer joins the
+// current block if its similarity to every layer already in that block reaches the threshold,
+// otherwise it opens a new block.
+int pod_greedy_layer_blocks(const float* sim, int n_heads, int n_layers, float threshold, int32_t* lowest_layer) {
+  if (!sim || !lowest_layer || n_heads < 1 || n_layers < 1) return POD_ERR_INVALID;
+  for (int h = 0; h < n_heads; ++h) {
+    const float* sh = sim + (size_t)h * n_layers * n_layers;
+    int start = 0;                                   // lowest layer of the current block
+    lowest_layer[h] = 0;
+    for (int l = 1; l < n_layers; ++l) {
+      bool similar_to_all = true;
+      for (int m = start; m < l && similar_to_all; ++m) similar_to_all = sh[(size_t)l * n_layers + m] >= threshold;
+      if (!similar_to_all) start = l;
+      lowest_layer[(size_t)l * n_heads + h] = start;
+    }
+  }
   return POD_OK;
 }
 
@@ -325,26 +411,35 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
   const pod_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return POD_ERR_INVALID;
   if (((uintptr_t)q % 16) != 0 || ((uintptr_t)out % 16) != 0) return POD_ERR_INVALID;
-  const int low = layer - layer % g.group_size, block = layer / g.group_size;
-  const bool lowest = (low == layer);
-  int32_t* sl = &c->stash_len[(size_t)block * g.batch];
+  const int H = g.n_kv_heads;
   const int add = fused ? 1 : 0;
+  auto stash_len_of = [&](int head) { return &c->stash_len[(size_t)c->slot_of(layer, head) * g.batch]; };
   if (fused)
     for (int b = 0; b < g.batch; ++b)
       if ((int64_t)c->h_len(layer, b) + 1 > c->cap[b]) return POD_ERR_CAPACITY;
-  if (!lowest) {
+  for (int h = 0; h < H; ++h) {          // every head whose block started at a lower layer
+    const int low = c->low_of(layer, h);
+    if (low == layer) continue;
+    const int32_t* sl = stash_len_of(h);
     for (int b = 0; b < g.batch; ++b) {
       const int32_t n = c->h_len(layer, b) + add;
       if (n != c->h_len(low, b)) return POD_ERR_ORDER;       // block must hold equal lengths
       if (n > 0 && sl[b] != n) return POD_ERR_ORDER;         // lowest layer's q not stashed at this step
     }
   }
+  auto note_stash = [&]() {              // heads for which this layer is the lowest of their block
+    for (int h = 0; h < H; ++h)
+      if (c->low_of(layer, h) == layer) {
+        int32_t* sl = stash_len_of(h);
+        for (int b = 0; b < g.batch; ++b) sl[b] = c->h_len(layer, b);
+      }
+  };
   if (fused) {                          // from here on the host lengths are the new ones
     for (int b = 0; b < g.batch; ++b) c->h_len(layer, b) += 1;
     c->memo_sum = -1;
   }
   if (c->dry) {
-    if (lowest) for (int b = 0; b < g.batch; ++b) sl[b] = c->h_len(layer, b);
+    note_stash();
     return POD_DRY_RUN;
   }
   const DecodePlan plan = plan_decode(c, layer);
@@ -356,15 +451,13 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
   p.new_v = static_cast<const uint16_t*>(v_new);
   p.len_out = fused ? c->d_len_copy(layer, c->len_cur[layer] ^ 1) : nullptr;
   p.q = static_cast<const uint16_t*>(q);
-  uint16_t* stash = reinterpret_cast<uint16_t*>(c->arena + c->cv.off_stash) + (size_t)block * g.batch * g.n_q_heads * g.head_dim;
-  p.q_low = lowest ? p.q : stash;
-  p.stash = (lowest && g.group_size > 1) ? stash : nullptr;
+  p.stash = reinterpret_cast<uint16_t*>(c->arena + c->cv.off_stash);
   p.part_acc = reinterpret_cast<float*>(c->arena + c->cv.off_pacc);
   p.part_ml = reinterpret_cast<float*>(c->arena + c->cv.off_pml);
   p.out = static_cast<uint16_t*>(out);
   p.err_flag = reinterpret_cast<int32_t*>(c->arena + c->cv.off_err);
   p.sched = reinterpret_cast<int32_t*>(c->arena + c->cv.off_sched);
-  p.layer = layer; p.block = block;
+  p.layer = layer;
   p.split_tokens = plan.split_tokens; p.max_splits = c->cv.max_splits;
   {
     // A warp sees about split_tokens / (tile tokens x warps) tiles; it should make a dozen draws.
@@ -374,18 +467,16 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     p.static_eighths = c->static_eighths;
   }
   p.scale_log2 = c->scale * 1.4426950408889634f;
-  // Shared distant logits: a lowest layer of a block of several layers stores them; another
-  // layer reads them if they are the ones of its block at exactly these lengths, else it falls
-  // back to scoring the block's keys itself.
-  p.score_mode = 0;
-  if (g.group_size > 1) {
-    if (lowest) {
-      p.score_mode = 1;
-    } else if (c->score_block == block) {
-      bool same = true;
-      for (int b = 0; b < g.batch; ++b) same = same && c->score_len[b] == c->h_len(layer, b);
-      if (same) p.score_mode = 2;
-    }
+  // Shared distant logits, head by head: the lowest layer of a block of several layers stores them
+  // (the kernel decides that from the block tables); a head of another layer reads them if its
+  // store holds the logits of its block at exactly these lengths, else it scores the block's keys.
+  for (int w = 0; w < 8; ++w) p.score_read_mask[w] = 0u;
+  for (int h = 0; h < H && h < 256; ++h) {
+    const int low = c->low_of(layer, h);
+    if (low == layer || c->score_low[h] != low) continue;
+    bool same = true;
+    for (int b = 0; b < g.batch; ++b) same = same && c->score_len[(size_t)h * g.batch + b] == c->h_len(layer, b);
+    if (same) p.score_read_mask[h >> 5] |= 1u << (h & 31);
   }
   // A launch that appends and attends streams only rows written before this step (the new token's
   // and the displaced token's rows are handled apart); the one launch that may still be running is
@@ -418,10 +509,11 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
       ++kernels;
     }
   }
-  if (lowest) for (int b = 0; b < g.batch; ++b) sl[b] = c->h_len(layer, b);
-  if (p.score_mode == 1) {
-    c->score_block = block;
-    for (int b = 0; b < g.batch; ++b) c->score_len[b] = c->h_len(layer, b);
+  note_stash();
+  for (int h = 0; h < H; ++h) {          // heads whose block starts here and goes on: their logits are stored now
+    if (c->low_of(layer, h) != layer || layer + 1 >= g.n_layers || c->low_of(layer + 1, h) != layer) continue;
+    c->score_low[h] = layer;
+    for (int b = 0; b < g.batch; ++b) c->score_len[(size_t)h * g.batch + b] = c->h_len(layer, b);
   }
   c->last_decode_layer = layer;
   c->last_split_tokens = plan.split_tokens; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;
@@ -453,7 +545,8 @@ int64_t pod_cache_bytes(const pod_cache* c, int which) {
       const int64_t n_p = n < SW ? n : SW, n_d = n - n_p;
       if (which == POD_BYTES_DENSE_EQUIV) { total += g.n_kv_heads * row * 2 * n; continue; }
       total += g.n_kv_heads * row * (2 * n_p + n_d);
-      if (l % g.group_size == 0) total += g.n_kv_heads * row * n_d;
+      for (int h = 0; h < g.n_kv_heads; ++h)
+        if (c->low_of(l, h) == l) total += row * n_d;       // distant keys are kept once per block
     }
   }
   return total;
@@ -470,10 +563,10 @@ int pod_cache_reset(pod_cache* c, int seq) {
   const int b0 = seq < 0 ? 0 : seq, b1 = seq < 0 ? g.batch : seq + 1;
   for (int l = 0; l < g.n_layers; ++l)
     for (int b = b0; b < b1; ++b) c->h_len(l, b) = 0;
-  for (int blk = 0; blk < c->cv.n_blocks; ++blk)
-    for (int b = b0; b < b1; ++b) c->stash_len[(size_t)blk * g.batch + b] = -1;
+  for (int sl = 0; sl < c->bm.n_slots; ++sl)
+    for (int b = b0; b < b1; ++b) c->stash_len[(size_t)sl * g.batch + b] = -1;
   c->memo_sum = -1;
-  c->score_block = -1;
+  for (auto& x : c->score_low) x = -1;
   c->last_decode_layer = -1;
   if (c->dry) return POD_DRY_RUN;
   cudaError_t e = cudaSetDevice(g.device);
@@ -492,7 +585,8 @@ int pod_cache_read_region(const pod_cache* c, int region, int layer_or_block, in
   const pod_config& g = c->cfg;
   if (seq < 0 || seq >= g.batch || kv_head < 0 || kv_head >= g.n_kv_heads || first < 0 || count < 0) return POD_ERR_INVALID;
   const bool is_block = (region == POD_REGION_DIST_K);
-  if (layer_or_block < 0 || layer_or_block >= (is_block ? c->cv.n_blocks : g.n_layers)) return POD_ERR_INVALID;
+  const int n_head_blocks = c->bm.head_base[kv_head + 1] - c->bm.head_base[kv_head];
+  if (layer_or_block < 0 || layer_or_block >= (is_block ? n_head_blocks : g.n_layers)) return POD_ERR_INVALID;
   const int64_t cap_d = c->cv.seq_cap_d[seq];
   int64_t row, extent;
   switch (region) {
@@ -500,7 +594,7 @@ int pod_cache_read_region(const pod_cache* c, int region, int layer_or_block, in
     case POD_REGION_SINK_V: row = prox_row(c->y, layer_or_block, 1, kv_head); extent = g.n_sink; break;
     case POD_REGION_RING_K: row = prox_row(c->y, layer_or_block, 0, kv_head) + g.n_sink; extent = g.n_recent; break;
     case POD_REGION_RING_V: row = prox_row(c->y, layer_or_block, 1, kv_head) + g.n_sink; extent = g.n_recent; break;
-    case POD_REGION_DIST_K: row = distk_row(c->y, layer_or_block, kv_head, cap_d); extent = cap_d; break;
+    case POD_REGION_DIST_K: row = distk_row(c->y, c->bm.head_base[kv_head] + layer_or_block, cap_d); extent = cap_d; break;
     case POD_REGION_DIST_V: row = distv_row(c->y, layer_or_block, kv_head, cap_d); extent = cap_d; break;
     default: return POD_ERR_INVALID;
   }

@@ -35,19 +35,34 @@ constexpr int SCHED_TICKET = 16;      // [0] = chunk counter, [SCHED_TICKET] = f
 // Sequence b owns a contiguous block starting at row seq_row_base[b]:
 //   prox  [L][2 (K, V)][H_kv][n_s + n_r]     rows [0, n_s) = sink, row n_s + slot = ring slot
 //   distV [L][H_kv][cap_d[b]]                 index p - n_s
-//   distK [n_blocks][H_kv][cap_d[b]]          index p - n_s, key of the block's lowest layer
-//   guard [32]                                only when G > 1: rows that stay zero
-//   score [H_kv][score_rows_per_head]         only when G > 1: the distant logits of the block being
+//   distK [n_slots][cap_d[b]]                 index p - n_s, key of a block's lowest layer; one slot per
+//                                             (head, block of that head), a head's slots adjacent
+//   guard [32]                                only when layers share: rows that stay zero
+//   score [H_kv][score_rows_per_head]         only when layers share: the distant logits of the block being
 //                                             decoded (fp32, log2 units), one group of 16 tokens x r
 //                                             query heads = r * 64 bytes in mma fragment order
 // with cap_d[b] = max(0, capacity[b] - n_s - n_r).  Sink and ring of one (layer, head) are
 // adjacent so that the proximal tokens of a head are one contiguous stream (the softmax does
 // not care about token order, so ring slots are read in slot order).
+//
+// Blocks are per KV head (Section 2.1, Algorithm 1): low[l][h] is the lowest layer of the block
+// that holds layer l for head h, slot[l][h] the index of that block's key store.  Null tables mean
+// that every layer is its own block (slot = l * H_kv + h).
 struct Layout {
-  int32_t L, H_kv, H_q, D, G, S, W, B, n_blocks;
+  int32_t L, H_kv, H_q, D, S, W, B;
+  int32_t n_slots;              // key stores = (layer, head) pairs that are lowest in their block
+  int32_t shared;               // 1 if some block has more than one layer
   const int64_t* seq_row_base;  // device [B]
   const int32_t* seq_cap_d;     // device [B]
+  const int32_t* low;           // device [L][H_kv] or nullptr
+  const int32_t* slot;          // device [L][H_kv] or nullptr
 };
+__device__ inline int lowest_of(const Layout& y, int layer, int head) {
+  return y.low ? y.low[layer * y.H_kv + head] : layer;
+}
+__device__ inline int slot_of(const Layout& y, int layer, int head) {
+  return y.slot ? y.slot[layer * y.H_kv + head] : layer * y.H_kv + head;
+}
 
 __host__ __device__ inline int64_t prox_row(const Layout& y, int layer, int kv /*0=K,1=V*/, int head) {
   return (((int64_t)layer * 2 + kv) * y.H_kv + head) * (int64_t)(y.S + y.W);
@@ -58,15 +73,15 @@ __host__ __device__ inline int64_t dist_base_row(const Layout& y) {
 __host__ __device__ inline int64_t distv_row(const Layout& y, int layer, int head, int64_t cap_d) {
   return dist_base_row(y) + ((int64_t)layer * y.H_kv + head) * cap_d;
 }
-__host__ __device__ inline int64_t distk_row(const Layout& y, int block, int head, int64_t cap_d) {
-  return dist_base_row(y) + (((int64_t)y.L + block) * y.H_kv + head) * cap_d;
+__host__ __device__ inline int64_t distk_row(const Layout& y, int slot, int64_t cap_d) {
+  return dist_base_row(y) + ((int64_t)y.L * y.H_kv + slot) * cap_d;
 }
 
 // Bytes of one 16-token group of shared distant logits (r query heads), and rows one head's
 // groups take (a row is D bf16).
 __host__ __device__ inline int score_group_bytes(const Layout& y) { return (y.H_q / y.H_kv) * 64; }
 __host__ __device__ inline int64_t score_rows_per_head(const Layout& y, int64_t cap_d) {
-  if (y.G <= 1) return 0;
+  if (!y.shared) return 0;
   const int64_t bytes = 2 * ((cap_d + 31) / 32) * score_group_bytes(y);   // read two groups at a time
   return (bytes + y.D * 2 - 1) / (y.D * 2);
 }
@@ -75,10 +90,10 @@ __host__ __device__ inline int64_t score_rows_per_head(const Layout& y, int64_t 
 // separates them from the key and value rows before them.
 constexpr int SCORE_GUARD_ROWS = 32;
 __host__ __device__ inline int64_t score_rows_per_seq(const Layout& y, int64_t cap_d) {
-  return y.G <= 1 ? 0 : SCORE_GUARD_ROWS + y.H_kv * score_rows_per_head(y, cap_d);
+  return !y.shared ? 0 : SCORE_GUARD_ROWS + y.H_kv * score_rows_per_head(y, cap_d);
 }
 __host__ __device__ inline int64_t score_row(const Layout& y, int head, int64_t cap_d) {
-  return dist_base_row(y) + ((int64_t)y.L + y.n_blocks) * y.H_kv * cap_d + SCORE_GUARD_ROWS +
+  return dist_base_row(y) + ((int64_t)y.L * y.H_kv + y.n_slots) * cap_d + SCORE_GUARD_ROWS +
          head * score_rows_per_head(y, cap_d);
 }
 
@@ -102,23 +117,24 @@ struct DecodeParams {
   const uint16_t* new_v;
   int32_t* len_out;
   const uint16_t* q;       // [B][H_q][D] queries of this layer
-  const uint16_t* q_low;   // [B][H_q][D] queries of the block's lowest layer (== q if lowest)
-  uint16_t* stash;         // where a lowest layer saves q for its block, else nullptr
+  uint16_t* stash;         // [n_slots][B][r][D]: a head's lowest layer saves its queries for the block here
   float* part_acc;         // [B][H_q][max_splits][D]
   float* part_ml;          // [B][H_q][max_splits][2]  (running max in log2 units, sum)
   uint16_t* out;           // [B][H_q][D]
   int32_t* err_flag;
   int32_t* sched;          // [B][H_kv][SCHED_STRIDE] zeroed chunk counters and tickets (the kernel re-zeroes them)
-  int32_t layer, block, split_tokens, max_splits;
+  int32_t layer, split_tokens, max_splits;
   int32_t tiles_per_chunk; // tiles a warp takes per draw from the head's chunk counter
   int32_t static_eighths;  // eighths of a warp's fair share of chunks that are assigned without a draw
   float scale_log2;        // sm_scale * log2(e)
   // Small batches carry the per-sequence lengths and row offsets by value (the host mirrors the
   // device lengths exactly), which takes two dependent global loads off every CTA's start-up.
-  // Shared distant logits (Section 2.2: a block shares the attention scores of its lowest layer):
-  // 1 = this launch is a lowest layer and stores them, 2 = this launch reads them instead of the
-  // block's keys, 0 = neither (dense, or the stored logits belong to other lengths).
-  int32_t score_mode;
+  // Shared distant logits (Section 2.2: a block shares the attention scores of its lowest layer).
+  // A head for which this layer is the lowest of a block with more layers stores them; a head for
+  // which it is not reads them instead of the block's keys when its bit is set here (the host sets
+  // it when the stored logits are those of the head's block at these lengths), else it scores the
+  // block's keys itself.  Bit h & 31 of word h >> 5; heads >= 256 never read stored logits.
+  uint32_t score_read_mask[8];
   int32_t early_ok;        // 1: no unfinished launch writes cache rows this launch streams (the two rows a
                            //    fused launch changes itself aside): tiles may be requested before the
                            //    wait for the previous kernel of the stream

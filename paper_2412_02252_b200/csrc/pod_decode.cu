@@ -222,7 +222,12 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int n_p = min(n, y.S + y.W), n_d = n - n_p;
   // A layer that reads the block's stored logits needs no key rows: its distant tiles hold 32
   // value rows (both halves of a stage), so the bytes in flight per stage stay the same.
-  const bool sc_write = p.score_mode == 1, sc_read = p.score_mode == 2;
+  // blocks are per KV head: is this layer the lowest of this head's block, and does the block go on?
+  const int low_layer = lowest_of(y, p.layer, kvh);
+  const int kslot = slot_of(y, p.layer, kvh);
+  const bool is_low = low_layer == p.layer;
+  const bool sc_write = y.shared && is_low && p.layer + 1 < y.L && lowest_of(y, p.layer + 1, kvh) == p.layer;
+  const bool sc_read = !is_low && kvh < 256 && ((p.score_read_mask[kvh >> 5] >> (kvh & 31)) & 1u);
   const int DT = sc_read ? 2 * TOK : TOK;         // tokens per distant tile
   const int ntp = (n_p + TOK - 1) / TOK, ntd = (n_d + DT - 1) / DT;
   const int ntiles = ntp + ntd;
@@ -237,7 +242,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // arena rows of this (sequence, layer, head): tile coordinates of the tensor map
   const int rowKp = (int)(seq_row + prox_row(y, p.layer, 0, kvh));
   const int rowVp = (int)(seq_row + prox_row(y, p.layer, 1, kvh));
-  const int rowKd = (int)(seq_row + distk_row(y, p.block, kvh, cap_d));
+  const int rowKd = (int)(seq_row + distk_row(y, kslot, cap_d));
   const int rowVd = (int)(seq_row + distv_row(y, p.layer, kvh, cap_d));
   // shared distant logits of this head: groups of 16 tokens x r heads, fp32, fragment order
   const int sc_group_b = score_group_bytes(y);
@@ -341,12 +346,13 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     }
   }
 
-  // a lowest layer saves its query for the other layers of the block
-  if (p.stash != nullptr && split == 0 && warp == 0 && lane < D / 8) {
-    for (int h = 0; h < r; ++h) {
-      const int64_t o = ((int64_t)b * y.H_q + kvh * r + h) * D + lane * 8;
-      *reinterpret_cast<uint4*>(p.stash + o) = *reinterpret_cast<const uint4*>(p.q + o);
-    }
+  // a head's lowest layer saves its queries for the other layers of the block
+  const int64_t q_own = ((int64_t)b * y.H_q + kvh * r) * D;         // this head's r query rows in q
+  const int64_t q_st = ((int64_t)kslot * y.B + b) * r * D;          // and in the stash of its block
+  if (sc_write && split == 0 && warp == 0 && lane < D / 8) {
+    for (int h = 0; h < r; ++h)
+      *reinterpret_cast<uint4*>(p.stash + q_st + h * D + lane * 8) =
+          *reinterpret_cast<const uint4*>(p.q + q_own + h * D + lane * 8);
   }
 
   // ---- per-lane state -------------------------------------------------------------------
@@ -354,13 +360,14 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int qcol = (lane & 3) * 2;     // first of the two columns this lane holds in a fragment
   uint32_t qp[D / 16][2], qd[D / 16][2];   // A fragments of Q (rows 0..7; rows 8..15 are zero):
   {                                        // own query (proximal tiles), lowest layer's (distant)
-    const int64_t qo = ((int64_t)b * y.H_q + kvh * r + qrow) * D + qcol;
+    const uint16_t* qo = p.q + q_own + qrow * D + qcol;
+    const uint16_t* ql = is_low ? qo : p.stash + q_st + qrow * D + qcol;
 #pragma unroll
     for (int kk = 0; kk < D / 16; ++kk) {
-      qp[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(p.q + qo + kk * 16) : 0u;
-      qp[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(p.q + qo + kk * 16 + 8) : 0u;
-      qd[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(p.q_low + qo + kk * 16) : 0u;
-      qd[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(p.q_low + qo + kk * 16 + 8) : 0u;
+      qp[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(qo + kk * 16) : 0u;
+      qp[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(qo + kk * 16 + 8) : 0u;
+      qd[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(ql + kk * 16) : 0u;
+      qd[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(ql + kk * 16 + 8) : 0u;
     }
   }
   // O^T accumulators: ot[cb][0], [1] = channel cb*16 + qrow of heads qcol, qcol + 1;
@@ -378,7 +385,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     __shared__ __align__(16) uint16_t s_sp[4][128];     // new K, new V, displaced K, displaced V
     constexpr int LPR = D / 8;                          // lanes per row, 16 bytes each
     uint16_t* arena_w = const_cast<uint16_t*>(p.arena);
-    const bool lowest = (p.layer % y.G) == 0;
+    const bool lowest = is_low;
     if (lane < 2 * LPR) {
       const bool isv = lane >= LPR;
       const int sub = lane % LPR;

@@ -110,26 +110,26 @@ extern "C" int pod_dense_decode_attn_static(const void* kv_device, int capacity,
   const int grid_splits = (n_tokens + split_tokens - 1) / split_tokens;
 
   DecodeParams p{};
-  p.y.L = 1; p.y.H_kv = n_kv_heads; p.y.H_q = n_q_heads; p.y.D = head_dim; p.y.G = 1;
-  p.y.S = 0; p.y.W = capacity; p.y.B = 1; p.y.n_blocks = 1;
+  p.y.L = 1; p.y.H_kv = n_kv_heads; p.y.H_q = n_q_heads; p.y.D = head_dim;
+  p.y.S = 0; p.y.W = capacity; p.y.B = 1; p.y.n_slots = n_kv_heads; p.y.shared = 0;
+  p.y.low = nullptr; p.y.slot = nullptr;               // one layer: every layer is its own block
   p.y.seq_row_base = nullptr; p.y.seq_cap_d = nullptr;        // not read: scalars go by value
   p.arena = static_cast<const uint16_t*>(kv_device);
   p.len = nullptr;
   p.q = static_cast<const uint16_t*>(q_device);
-  p.q_low = p.q;
   p.stash = nullptr;
   p.part_acc = reinterpret_cast<float*>(su->scratch + OFF_PACC);
   p.part_ml = reinterpret_cast<float*>(su->scratch + OFF_PML);
   p.out = static_cast<uint16_t*>(out_device);
   p.err_flag = reinterpret_cast<int32_t*>(su->scratch + OFF_ERR);
   p.sched = reinterpret_cast<int32_t*>(su->scratch + OFF_SCHED);
-  p.layer = 0; p.block = 0; p.split_tokens = split_tokens; p.max_splits = STATIC_MAX_SPLITS;
+  p.layer = 0; p.split_tokens = split_tokens; p.max_splits = STATIC_MAX_SPLITS;
   p.tiles_per_chunk = split_tokens / (decode_tile_tokens() * decode_warps_per_cta() * 16);
   if (p.tiles_per_chunk < 1) p.tiles_per_chunk = 1;
   if (p.tiles_per_chunk > 16) p.tiles_per_chunk = 16;
   p.static_eighths = 5;
   p.scale_log2 = (sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim)) * 1.4426950408889634f;
-  p.score_mode = 0;
+  for (int w = 0; w < 8; ++w) p.score_read_mask[w] = 0u;
   p.early_ok = 0;
   p.by_value = 1;
   p.v_len[0] = n_tokens; p.v_cap_d[0] = 0; p.v_row_base[0] = 0;

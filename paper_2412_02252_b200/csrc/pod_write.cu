@@ -35,8 +35,6 @@ __global__ void __launch_bounds__(256) pod_write_kernel(const WriteParams p) {
 
   const int64_t cap_d = y.seq_cap_d[b];
   uint16_t* seq_base = p.arena + y.seq_row_base[b] * D;
-  const bool lowest = (p.layer % y.G) == 0;
-  const int block = p.layer / y.G;
   const int ring_first = max(S, n1 - W);     // first position that is in the ring after the call
 
   for (int item = item0; item < n_items; item += item_stride) {
@@ -51,7 +49,8 @@ __global__ void __launch_bounds__(256) pod_write_kernel(const WriteParams p) {
     uint16_t* prox = seq_base + prox_row(y, p.layer, kv, h) * D;
     uint16_t* dist = nullptr;                // distant store of this item's kind, if it is kept
     if (kv) dist = seq_base + distv_row(y, p.layer, h, cap_d) * D;
-    else if (lowest) dist = seq_base + distk_row(y, block, h, cap_d) * D;
+    else if (lowest_of(y, p.layer, h) == p.layer)          // keys survive once per block of this head
+      dist = seq_base + distk_row(y, slot_of(y, p.layer, h), cap_d) * D;
 
     if (pos < S) {
       *reinterpret_cast<uint4*>(prox + (int64_t)pos * D + sub * 8) = val;

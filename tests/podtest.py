@@ -13,11 +13,14 @@ MAX_ABS, REL_L2 = 1e-2, 5e-3      # bf16 inputs, fp32 accumulation, bf16 output
 
 
 class Case:
-    def __init__(self, *, seed, L, G, Hq, Hkv, d, S, W, lens, outliers=False, caps=None, scale=0.0):
+    def __init__(self, *, seed, L, G, Hq, Hkv, d, S, W, lens, outliers=False, caps=None, scale=0.0, lowest=None):
         self.seed, self.L, self.G, self.Hq, self.Hkv, self.d = seed, L, G, Hq, Hkv, d
         self.S, self.W, self.lens, self.outliers, self.scale = S, W, list(lens), outliers, scale
         self.B = len(self.lens)
         self.caps = list(caps) if caps is not None else [max(1, n) for n in self.lens]
+        # per-head blocks: lowest[l][h]; None = runs of G layers for every head
+        self.lowest = O.uniform_lowest_map(L, Hkv, G).tolist() if lowest is None else [list(r) for r in lowest]
+        self.head_wise = lowest is not None
         self.cfg = B.make_config(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, group_size=G,
                                  n_sink=S, n_recent=W, batch=self.B, sm_scale=scale, device=0)
 
@@ -31,7 +34,7 @@ class Case:
 
     # ---- CUDA path ---------------------------------------------------------------------------
     def make_cache(self):
-        return B.PodCache(self.cfg, self.caps)
+        return B.PodCache(self.cfg, self.caps, lowest_layer=self.lowest if self.head_wise else None)
 
     def prefill(self, cache, upto=None, chunk=8192, layers=None):
         """Writes positions [len so far, upto[b]) of every sequence, layer by layer."""
@@ -65,7 +68,7 @@ class Case:
         if n == 0:
             return np.zeros(self.d)
         kvh = h // (self.Hq // self.Hkv)
-        low = O.lowest_layer(layer, self.G)
+        low = self.lowest[layer][kvh]
         f = lambda tag, l: self.kv(tag, l, b, 0, n, "cpu", heads=[kvh])[:, 0].double().numpy()
         K_l, V_l = f(synth.TAG_K, layer), f(synth.TAG_V, layer)
         K_a = K_l if low == layer else f(synth.TAG_K, low)

@@ -184,6 +184,59 @@ def test_fused_append_decode_order_and_capacity_rules():
         assert e.value.status == B.POD_ERR_INVALID
 
 
+def test_greedy_layer_blocks_matches_the_oracle():
+    """The library's Algorithm 1 against the oracle's on random similarities and on the hand-worked case."""
+    import numpy as np
+    rng = np.random.default_rng(11)
+    for H, L, thr in [(1, 5, 0.5), (4, 9, 0.5), (3, 12, 0.3), (2, 7, 0.8)]:
+        sim = rng.random((H, L, L)).astype(np.float32)
+        want = O.lowest_map_from_blocks(O.greedy_layer_blocks(sim.astype(np.float64), thr), L)
+        got = B.pod_greedy_layer_blocks(sim.tolist(), thr)
+        assert got == want.tolist()
+    sim = np.eye(5)[None].copy()
+    for a, b, v in [(0, 1, .8), (0, 2, .4), (1, 2, .9), (0, 3, .9), (1, 3, .6), (2, 3, .7), (2, 4, .9), (3, 4, .2)]:
+        sim[0, a, b] = sim[0, b, a] = v
+    assert [row[0] for row in B.pod_greedy_layer_blocks(sim.tolist(), 0.5)] == [0, 0, 2, 2, 4]
+
+
+def test_head_wise_block_maps_on_a_host_only_cache():
+    cfg = _cfg(n_layers=4, n_kv_heads=2, n_q_heads=8, group_size=1)
+    p = _fake_ptr()
+    low = [[0, 0], [0, 1], [2, 1], [2, 1]]              # head 0: {0,1},{2,3}; head 1: {0},{1,2,3}
+    for bad in ([[0, 0], [0, 0], [1, 0], [1, 0]], [[1, 0], [1, 1], [2, 1], [2, 1]], [[0, 0], [0, 2], [2, 2], [2, 2]]):
+        with pytest.raises(B.PodError) as e:
+            B.PodCache(cfg, [600], lowest_layer=bad)
+        assert e.value.status == B.POD_ERR_INVALID
+        assert B.pod_cache_required_bytes(cfg, [600], lowest_layer=bad) == 0
+    assert B.pod_cache_required_bytes(cfg, [600], lowest_layer=low) > 0
+    c = B.PodCache(cfg, [600], lowest_layer=low)
+    for l in range(4):
+        c.write(l, 0, p, p, 500)
+    live, dense = O.pod_cache_bytes([500], n_layers=4, n_kv_heads=2, head_dim=64, lowest=low, n_s=16, n_r=64)
+    assert c.bytes(B.POD_BYTES_LIVE) == live and c.bytes(B.POD_BYTES_DENSE_EQUIV) == dense
+    # layer 1: head 0 needs layer 0's query of this step, head 1 starts a block here
+    with pytest.raises(B.PodError) as e:
+        c.decode_attn(1, p, p)
+    assert e.value.status == B.POD_ERR_ORDER
+    assert c.decode_attn(0, p, p) == B.POD_DRY_RUN
+    assert c.decode_attn(1, p, p) == B.POD_DRY_RUN
+    assert c.decode_attn(2, p, p) == B.POD_DRY_RUN      # head 0 lowest, head 1 follows layer 1 (decoded)
+    assert c.decode_attn(3, p, p) == B.POD_DRY_RUN
+    c.write(0, 0, p, p, 1)
+    c.write(1, 0, p, p, 1)
+    c.write(2, 0, p, p, 1)
+    assert c.decode_attn(0, p, p) == B.POD_DRY_RUN
+    with pytest.raises(B.PodError) as e:                 # head 1 of layer 2 follows layer 1, not decoded at this length
+        c.decode_attn(2, p, p)
+    assert e.value.status == B.POD_ERR_ORDER
+    assert c.decode_attn(1, p, p) == B.POD_DRY_RUN
+    assert c.decode_attn(2, p, p) == B.POD_DRY_RUN
+    # a uniform map given explicitly is the same cache as group_size
+    cu = B.PodCache(_cfg(n_layers=4, group_size=1), [600], lowest_layer=[[0, 0], [0, 0], [2, 2], [2, 2]])
+    cg = B.PodCache(_cfg(n_layers=4, group_size=2), [600])
+    assert cu.bytes(B.POD_BYTES_ALLOCATED) == cg.bytes(B.POD_BYTES_ALLOCATED)
+
+
 def test_dense_configuration_needs_no_order():
     cfg = _cfg(group_size=1)
     c = B.PodCache(cfg, [64])

@@ -17,7 +17,7 @@ REGIONS = [("sinkK", B.POD_REGION_SINK_K), ("sinkV", B.POD_REGION_SINK_V),
 
 
 def _oracle_cache(case, b):
-    return O.PodCacheOracle(case.L, case.Hkv, case.d, case.G, case.S, case.W, case.caps[b])
+    return O.PodCacheOracle(case.L, case.Hkv, case.d, case.G, case.S, case.W, case.caps[b], lowest=case.lowest)
 
 
 def _compare_layout(case, cache, oracles):
@@ -27,6 +27,8 @@ def _compare_layout(case, cache, oracles):
             for i in range(count):
                 for h in range(case.Hkv):
                     ref, first = oc.valid_rows(name, i, h)
+                    if ref.shape[0] == 0:              # nothing valid (or this head has fewer blocks)
+                        continue
                     got = cache.read_region(rid, i, b, h, first, ref.shape[0])
                     np.testing.assert_array_equal(got, ref, err_msg=f"{name}[{i}] seq {b} head {h}")
 
@@ -234,6 +236,71 @@ def test_shared_logits_fallback_and_mixed_calls():
         torch.cuda.synchronize()
         _check_all_heads(case, outs, step=step, lens=lens)
     assert cache.device_status() == B.POD_OK
+
+
+HEAD_WISE = [[0, 0, 0, 0], [0, 1, 0, 1], [0, 1, 2, 1], [3, 1, 2, 1], [3, 4, 2, 1], [3, 4, 2, 5]]
+
+
+@pytest.mark.parametrize("d", [128, 64])
+def test_head_wise_blocks_layout_and_attention(d):
+    """Blocks chosen per KV head (Algorithm 1's output shape): a layer is the lowest of its block for
+    some heads and not for others.  Prefill, two-call steps, one-launch steps across ring wraps; cache
+    contents bit for bit against the oracle's layout, outputs against the definition."""
+    lens0 = [70, 23, 0]
+    case = Case(seed=17, L=6, G=1, Hq=8, Hkv=4, d=d, S=4, W=16, lens=lens0, caps=[n + 30 for n in lens0],
+                lowest=HEAD_WISE)
+    cache = case.make_cache()
+    case.prefill(cache, chunk=33)
+    ocs = [_oracle_cache(case, b) for b in range(case.B)]
+    for b, oc in enumerate(ocs):
+        for l in range(case.L):
+            if lens0[b]:
+                oc.write(l, synth.bf16_bits(case.kv(synth.TAG_K, l, b, 0, lens0[b], "cpu")),
+                         synth.bf16_bits(case.kv(synth.TAG_V, l, b, 0, lens0[b], "cpu")))
+    _compare_layout(case, cache, ocs)
+    _check_all_heads(case, case.decode_all(cache))
+    live, dense = O.pod_cache_bytes(lens0, n_layers=6, n_kv_heads=4, head_dim=d, lowest=HEAD_WISE, n_s=4, n_r=16)
+    assert cache.bytes(B.POD_BYTES_LIVE) == live and cache.bytes(B.POD_BYTES_DENSE_EQUIV) == dense
+    stream = torch.cuda.current_stream().cuda_stream
+    outs = torch.empty(case.L, case.B, case.Hq, case.d, dtype=torch.bfloat16, device="cuda")
+    for step in range(1, 26):
+        lens = [n + step for n in lens0]
+        for l in range(case.L):
+            k = torch.stack([case.kv(synth.TAG_K, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            v = torch.stack([case.kv(synth.TAG_V, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            if step % 3:
+                cache.append_decode_attn(l, k, v, case.q(l, step, "cuda"), outs[l], stream)
+            else:
+                cache.write(l, -1, k, v, 1, stream)
+                cache.decode_attn(l, case.q(l, step, "cuda"), outs[l], stream)
+            kb, vb = synth.bf16_bits(k), synth.bf16_bits(v)
+            for b, oc in enumerate(ocs):
+                oc.append(l, kb[b], vb[b])
+        torch.cuda.synchronize()
+        if step in (1, 2, 3, 16, 17, 18, 21, 24, 25):
+            _check_all_heads(case, outs, step=step, lens=lens)
+            _compare_layout(case, cache, ocs)
+    assert cache.device_status() == B.POD_OK
+
+
+def test_head_wise_blocks_from_greedy_grouping_many_tiles():
+    """A map produced by the library's greedy grouping from a seeded similarity tensor, on a context
+    of several thousand tokens (many tiles and splits per head)."""
+    rng = np.random.default_rng(5)
+    L, Hkv = 8, 2
+    sim = rng.random((Hkv, L, L)) * 0.7 + 0.25
+    sim = np.maximum(sim, sim.transpose(0, 2, 1))
+    lowest = B.pod_greedy_layer_blocks(sim.tolist(), 0.5)
+    assert lowest == O.lowest_map_from_blocks(O.greedy_layer_blocks(sim.astype(np.float32).astype(np.float64), 0.5), L).tolist()
+    assert any(lowest[l][0] != lowest[l][1] for l in range(L))         # the heads really differ
+    case = Case(seed=18, L=L, G=1, Hq=8, Hkv=Hkv, d=128, S=16, W=256, lens=[5000, 3333], lowest=lowest)
+    cache = case.make_cache()
+    case.prefill(cache)
+    outs = case.decode_all(cache)
+    for l in range(L):
+        for b in range(2):
+            for h in (0, 3, 4, 7):
+                assert_close(outs[l, b, h], case.oracle_head(l, b, h), f"layer {l} seq {b} head {h}")
 
 
 def test_custom_scale():
