@@ -148,7 +148,7 @@ struct pod_cache {
   // last launch (diagnostics)
   int32_t last_split_tokens = 0, last_ctas = 0, last_kernels = 0;
   // planner memo
-  int64_t memo_sum = -1; int32_t memo_max = -1; DecodePlan memo_plan{};
+  int64_t memo_sum = -1; int32_t memo_max = -1; int memo_light = -1; DecodePlan memo_plan{};
 
   // Device lengths are kept twice.  A launch that appends and attends at once reads one copy and
   // writes the other (its CTAs start at different times, so nobody may change what they read);
@@ -193,36 +193,54 @@ bool make_tensor_map(pod_cache* c) {
 
 // Picks the tokens-per-split that minimises a simple time model: the CTAs run in waves of
 // (SMs x resident CTAs), every CTA costs its tokens plus a fixed overhead.
-DecodePlan plan_decode(pod_cache* c, int layer) {
+// Picks the rows-per-split that minimises a simple time model: the CTAs run in waves of
+// (SMs x resident CTAs), every CTA costs its rows plus a fixed overhead.  A head that reads keys and
+// values streams 2 n rows, a head that reads the block's stored logits n + n_p; n_light heads of
+// this launch are of the second kind.
+DecodePlan plan_decode(pod_cache* c, int layer, int n_light) {
   const pod_config& g = c->cfg;
+  const int n_heavy = g.n_kv_heads - n_light;
+  const int64_t SW = (int64_t)g.n_sink + g.n_recent;
   int64_t sum = 0; int32_t nmax = 0;
   for (int b = 0; b < g.batch; ++b) { const int32_t n = c->h_len(layer, b); sum += n; if (n > nmax) nmax = n; }
-  if (sum == c->memo_sum && nmax == c->memo_max) return c->memo_plan;
-  DecodePlan best{1, 1, 0};
+  if (sum == c->memo_sum && nmax == c->memo_max && n_light == c->memo_light) return c->memo_plan;
+  auto heavy_rows = [](int64_t n) { return 2 * n; };
+  auto light_rows = [SW](int64_t n) { return n + (n < SW ? n : SW); };
+  auto count = [&](int64_t st, int64_t* ctas, int64_t* most) {
+    *ctas = 0; *most = 0;
+    for (int b = 0; b < g.batch; ++b) {
+      const int64_t n = c->h_len(layer, b);
+      const int64_t kh = (heavy_rows(n) + st - 1) / st, kl = (light_rows(n) + st - 1) / st;
+      *ctas += n_heavy * kh + n_light * kl;
+      const int64_t m = n_heavy > 0 ? kh : kl;
+      if (m > *most) *most = m;
+    }
+  };
+  const int64_t wmax = n_heavy > 0 ? heavy_rows(nmax) : light_rows(nmax);
+  DecodePlan best{2, 1, 0};
   if (nmax > 0 && c->force_split_tokens > 0) {      // POD_SPLIT_TOKENS: tuning experiments
-    int st = c->force_split_tokens;
-    if (st < (nmax + c->cv.max_splits - 1) / c->cv.max_splits) st = (nmax + c->cv.max_splits - 1) / c->cv.max_splits;
-    int64_t ctas = 0;
-    for (int b = 0; b < g.batch; ++b) ctas += ((int64_t)c->h_len(layer, b) + st - 1) / st;
-    best = DecodePlan{st, (nmax + st - 1) / st, (int32_t)(ctas * g.n_kv_heads)};
+    int64_t st = 2 * (int64_t)c->force_split_tokens;
+    if (st < (wmax + c->cv.max_splits - 1) / c->cv.max_splits) st = (wmax + c->cv.max_splits - 1) / c->cv.max_splits;
+    int64_t ctas, most;
+    count(st, &ctas, &most);
+    best = DecodePlan{(int32_t)st, (int32_t)most, (int32_t)ctas};
   } else if (nmax > 0) {
     const int64_t slots = (int64_t)c->sm_count * c->resident;
     double best_cost = 1e300;
-    int last_st = -1;
+    int64_t last_st = -1;
     for (int k = 1; k <= c->cv.max_splits; ++k) {
-      const int st = (nmax + k - 1) / k;
+      const int64_t st = (wmax + k - 1) / k;
       if (st == last_st) continue;
       last_st = st;
-      int64_t ctas = 0;
-      for (int b = 0; b < g.batch; ++b) ctas += ((int64_t)c->h_len(layer, b) + st - 1) / st;
-      ctas *= g.n_kv_heads;
+      int64_t ctas, most;
+      count(st, &ctas, &most);
       const int64_t waves = (ctas + slots - 1) / slots;
-      const double cost = (double)waves * (st + SPLIT_OVERHEAD_TOKENS);
-      if (cost < best_cost * 0.999) { best_cost = cost; best = DecodePlan{st, (nmax + st - 1) / st, (int32_t)ctas}; }
-      if (st <= 64) break;
+      const double cost = (double)waves * (st + 2 * SPLIT_OVERHEAD_TOKENS);
+      if (cost < best_cost * 0.999) { best_cost = cost; best = DecodePlan{(int32_t)st, (int32_t)most, (int32_t)ctas}; }
+      if (st <= 128) break;
     }
   }
-  c->memo_sum = sum; c->memo_max = nmax; c->memo_plan = best;
+  c->memo_sum = sum; c->memo_max = nmax; c->memo_light = n_light; c->memo_plan = best;
   return best;
 }
 
@@ -442,7 +460,6 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     note_stash();
     return POD_DRY_RUN;
   }
-  const DecodePlan plan = plan_decode(c, layer);
   DecodeParams p;
   p.y = c->y;
   p.arena = reinterpret_cast<const uint16_t*>(c->arena);
@@ -458,25 +475,27 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
   p.err_flag = reinterpret_cast<int32_t*>(c->arena + c->cv.off_err);
   p.sched = reinterpret_cast<int32_t*>(c->arena + c->cv.off_sched);
   p.layer = layer;
-  p.split_tokens = plan.split_tokens; p.max_splits = c->cv.max_splits;
-  {
-    // A warp sees about split_tokens / (tile tokens x warps) tiles; it should make a dozen draws.
-    int tch = plan.split_tokens / (decode_tile_tokens() * decode_warps_per_cta() * 16);
-    if (c->force_chunk_tiles > 0) tch = c->force_chunk_tiles;
-    p.tiles_per_chunk = tch < 1 ? 1 : (tch > 256 ? 256 : tch);
-    p.static_eighths = c->static_eighths;
-  }
   p.scale_log2 = c->scale * 1.4426950408889634f;
   // Shared distant logits, head by head: the lowest layer of a block of several layers stores them
   // (the kernel decides that from the block tables); a head of another layer reads them if its
   // store holds the logits of its block at exactly these lengths, else it scores the block's keys.
   for (int w = 0; w < 8; ++w) p.score_read_mask[w] = 0u;
+  int n_light = 0;                       // heads of this launch that read stored logits
   for (int h = 0; h < H && h < 256; ++h) {
     const int low = c->low_of(layer, h);
     if (low == layer || c->score_low[h] != low) continue;
     bool same = true;
     for (int b = 0; b < g.batch; ++b) same = same && c->score_len[(size_t)h * g.batch + b] == c->h_len(layer, b);
-    if (same) p.score_read_mask[h >> 5] |= 1u << (h & 31);
+    if (same) { p.score_read_mask[h >> 5] |= 1u << (h & 31); ++n_light; }
+  }
+  const DecodePlan plan = plan_decode(c, layer, n_light);
+  p.split_rows = plan.split_rows; p.max_splits = c->cv.max_splits;
+  {
+    // A warp sees about split_rows / (2 x tile tokens x warps) tiles; it should make a dozen draws.
+    int tch = plan.split_rows / (2 * decode_tile_tokens() * decode_warps_per_cta() * 16);
+    if (c->force_chunk_tiles > 0) tch = c->force_chunk_tiles;
+    p.tiles_per_chunk = tch < 1 ? 1 : (tch > 256 ? 256 : tch);
+    p.static_eighths = c->static_eighths;
   }
   // A launch that appends and attends streams only rows written before this step (the new token's
   // and the displaced token's rows are handled apart); the one launch that may still be running is
@@ -516,7 +535,7 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     for (int b = 0; b < g.batch; ++b) c->score_len[(size_t)h * g.batch + b] = c->h_len(layer, b);
   }
   c->last_decode_layer = layer;
-  c->last_split_tokens = plan.split_tokens; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;
+  c->last_split_tokens = plan.split_rows / 2; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;
   return POD_OK;
 }
 

@@ -123,7 +123,9 @@ struct DecodeParams {
   uint16_t* out;           // [B][H_q][D]
   int32_t* err_flag;
   int32_t* sched;          // [B][H_kv][SCHED_STRIDE] zeroed chunk counters and tickets (the kernel re-zeroes them)
-  int32_t layer, split_tokens, max_splits;
+  int32_t layer, max_splits;
+  int32_t split_rows;      // K or V rows a CTA should stream: a head that reads keys and values has 2 n rows of
+                           // work, a head that reads stored logits n + n_p; its CTAs = ceil(work / split_rows)
   int32_t tiles_per_chunk; // tiles a warp takes per draw from the head's chunk counter
   int32_t static_eighths;  // eighths of a warp's fair share of chunks that are assigned without a draw
   float scale_log2;        // sm_scale * log2(e)
@@ -145,7 +147,7 @@ struct DecodeParams {
 };
 
 struct DecodePlan {
-  int32_t split_tokens;   // tokens per split
+  int32_t split_rows;     // rows of work per split
   int32_t grid_splits;    // grid.x
   int32_t n_ctas;         // CTAs that do work
 };

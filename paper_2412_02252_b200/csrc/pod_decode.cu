@@ -215,8 +215,6 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     cap_d = y.seq_cap_d[b];
     seq_row = y.seq_row_base[b];
   }
-  const int nsplit = min(p.max_splits, (n + p.split_tokens - 1) / p.split_tokens);
-  if (split >= nsplit) return;
 
   // ---- tiles and chunks of this (sequence, KV head) -----------------------------------------
   const int n_p = min(n, y.S + y.W), n_d = n - n_p;
@@ -228,6 +226,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const bool is_low = low_layer == p.layer;
   const bool sc_write = y.shared && is_low && p.layer + 1 < y.L && lowest_of(y, p.layer + 1, kvh) == p.layer;
   const bool sc_read = !is_low && kvh < 256 && ((p.score_read_mask[kvh >> 5] >> (kvh & 31)) & 1u);
+  // CTAs of this head: in proportion to the rows it streams (keys and values, or values and the
+  // proximal keys only), so that heads with different roles in one launch finish together
+  const int64_t work_rows = sc_read ? (int64_t)n + min(n, y.S + y.W) : 2 * (int64_t)n;
+  const int nsplit = (int)min((int64_t)p.max_splits, (work_rows + p.split_rows - 1) / p.split_rows);
+  if (split >= nsplit) return;
   const int DT = sc_read ? 2 * TOK : TOK;         // tokens per distant tile
   const int ntp = (n_p + TOK - 1) / TOK, ntd = (n_d + DT - 1) / DT;
   const int ntiles = ntp + ntd;
