@@ -237,6 +237,23 @@ def test_head_wise_block_maps_on_a_host_only_cache():
     assert cu.bytes(B.POD_BYTES_ALLOCATED) == cg.bytes(B.POD_BYTES_ALLOCATED)
 
 
+def test_largest_cache_is_bounded_by_32_bit_row_indices():
+    """Tile coordinates are 32-bit row indices: a cache whose regions would hold 2^31 rows or more is
+    refused at creation (and sized 0), the largest one below that is accepted on a host-only cache."""
+    cfg = _cfg(n_layers=32, n_q_heads=32, n_kv_heads=8, head_dim=128, group_size=2, n_sink=16, n_recent=2048)
+    rows_per_token = 32 * 8 + 16 * 8                     # value rows of every layer + key rows of every block
+    too_many = (2 ** 31) // rows_per_token + 4096
+    assert B.pod_cache_required_bytes(cfg, [too_many]) == 0
+    with pytest.raises(B.PodError) as e:
+        B.PodCache(cfg, [too_many])
+    assert e.value.status == B.POD_ERR_INVALID
+    ok = (2 ** 31) // rows_per_token - 8192
+    need = B.pod_cache_required_bytes(cfg, [ok])
+    assert need > ok * rows_per_token * 256
+    c = B.PodCache(cfg, [ok])
+    assert c.bytes(B.POD_BYTES_ALLOCATED) == need
+
+
 def test_dense_configuration_needs_no_order():
     cfg = _cfg(group_size=1)
     c = B.PodCache(cfg, [64])
