@@ -167,6 +167,31 @@ def pod_attention_gate(q_l, q_a, K_l, K_a, V_l, n_s, n_r, scale=None):
     return g * oP + (1.0 - g) * oD, g
 
 
+def pod_attention_gate_skip(q_l, q_a, K_l, K_a, V_l, n_s, n_r, tau, scale=None):
+    """Appendix "Computation Optimization for Distant Tokens": for a layer that is not the lowest of
+    its block the gate g of Eq. 2 is evaluated first (the distant logits are the lowest layer's, so
+    their sum is known before any distant value is read); if g >= tau the attention to the distant
+    tokens is omitted.  Reading of "omitted": the output is then the proximal output o^P alone (the
+    gate is treated as 1); otherwise Eq. 2 is applied unchanged.  The caller applies this to layers
+    other than a block's lowest only.  Returns (o [d], g, skipped)."""
+    d = q_l.shape[0]
+    scale = 1.0 / math.sqrt(d) if scale is None else scale
+    a, prox = pod_logits(q_l, q_a, K_l, K_a, n_s, n_r, scale)
+    aP, VP = a[prox], V_l[prox]
+    aD, VD = a[~prox], V_l[~prox]
+    oP = _softmax(aP) @ VP
+    if aD.size == 0:                      # no distant tokens: nothing to omit
+        return oP, 1.0, False
+    shift = max(aP.max(), aD.max())
+    sP = np.exp(aP - shift).sum()
+    sD = np.exp(aD - shift).sum()
+    g = sP / (sP + sD)
+    if g >= tau:
+        return oP, g, True
+    oD = _softmax(aD) @ VD
+    return g * oP + (1.0 - g) * oD, g, False
+
+
 def _softmax(a):
     e = np.exp(a - a.max())
     return e / e.sum()
@@ -175,7 +200,8 @@ def _softmax(a):
 # --------------------------------------------------------------------------------------
 # all heads of one layer, full history
 # --------------------------------------------------------------------------------------
-def pod_decode_layer(q, K, V, layer, *, group_size=None, lowest=None, n_s, n_r, scale=None, form="joint"):
+def pod_decode_layer(q, K, V, layer, *, group_size=None, lowest=None, n_s, n_r, scale=None, form="joint",
+                     tau=None, info=None):
     """One layer's decode attention for one sequence from the uncompressed history.
 
     q: [L][H_q][d] queries of every layer at this step (only rows ``layer`` and its blocks'
@@ -183,6 +209,9 @@ def pod_decode_layer(q, K, V, layer, *, group_size=None, lowest=None, n_s, n_r, 
     every head) or ``lowest`` (a per-head lowest map [L][H_kv]).  Query head h reads KV head h // r,
     r = H_q / H_kv (grouped-query attention).  Returns o [H_q][d] (float64).
     An empty history (n == 0) gives zeros (convention of this build; the paper is silent).
+    ``tau``: gate threshold of the distant-skip optimisation (None = off); heads for which ``layer``
+    is not the lowest layer of their block skip the distant tokens when g >= tau.  ``info``, if a
+    list, receives (g, skipped) per query head.
     """
     L, n, H_kv, d = K.shape
     H_q = q.shape[1]
@@ -195,6 +224,14 @@ def pod_decode_layer(q, K, V, layer, *, group_size=None, lowest=None, n_s, n_r, 
     for h in range(H_q):
         kv = h // r
         a = int(low[layer, kv])                 # lowest layer of this head's block
+        if tau is not None and a != layer:
+            out[h], g, skipped = pod_attention_gate_skip(q[layer, h], q[a, h], K[layer, :, kv], K[a, :, kv],
+                                                         V[layer, :, kv], n_s, n_r, tau, scale)
+            if info is not None:
+                info.append((g, skipped))
+            continue
+        if info is not None:
+            info.append((None, False))
         out[h], _ = fn(q[layer, h], q[a, h], K[layer, :, kv], K[a, :, kv], V[layer, :, kv],
                        n_s, n_r, scale)
     return out

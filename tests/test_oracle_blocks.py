@@ -179,3 +179,70 @@ def test_head_wise_byte_counts():
     shared = float(np.mean(low != np.arange(L)[:, None]))
     assert abs((1 - live / dense) - O.pod_saving_closed_form(n, n_layers=L, n_s=S, n_r=W, shared_fraction=shared)) < 1e-12
     assert abs(O.pod_saving_closed_form(10 ** 9, n_layers=32, n_s=16, n_r=4080, shared_fraction=0.7) - 0.35) < 1e-5
+
+
+# --------------------------------------------------------------------------- gate threshold (distant skip)
+def _one_head(rng, n, d):
+    bf = lambda x: (x.astype(np.float32).view(np.uint32) & 0xFFFF0000).view(np.float32).astype(np.float64)
+    return (bf(rng.standard_normal(d)), bf(rng.standard_normal(d)), bf(rng.standard_normal((n, d))),
+            bf(rng.standard_normal((n, d))), bf(rng.standard_normal((n, d))))
+
+
+def test_gate_skip_limits_and_identity():
+    """tau above 1 never skips and gives the joint softmax; tau = 0 always skips and gives textbook
+    attention over the proximal tokens alone (torch SDPA); in between the decision is g >= tau, and
+    the two candidate outputs differ by exactly (1 - g)(o^P - o^D)."""
+    import torch
+    rng = np.random.default_rng(4)
+    n, d, S, W = 60, 16, 3, 9
+    q_l, q_a, K_l, K_a, V_l = _one_head(rng, n, d)
+    full, _ = O.pod_attention_joint(q_l, q_a, K_l, K_a, V_l, S, W)
+    o, g, skipped = O.pod_attention_gate_skip(q_l, q_a, K_l, K_a, V_l, S, W, tau=1.5)
+    assert not skipped and 0 < g < 1
+    np.testing.assert_allclose(o, full, rtol=0, atol=1e-12)
+    o0, g0, skipped0 = O.pod_attention_gate_skip(q_l, q_a, K_l, K_a, V_l, S, W, tau=0.0)
+    assert skipped0 and g0 == g
+    prox = np.array([p < S or p >= n - W for p in range(n)])
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.tensor(q_l)[None, None], torch.tensor(K_l[prox])[None], torch.tensor(V_l[prox])[None])[0, 0].numpy()
+    np.testing.assert_allclose(o0, ref, rtol=0, atol=1e-12)
+    # the decision flips exactly at g
+    assert O.pod_attention_gate_skip(q_l, q_a, K_l, K_a, V_l, S, W, tau=g)[2]
+    assert not O.pod_attention_gate_skip(q_l, q_a, K_l, K_a, V_l, S, W, tau=np.nextafter(g, 1.0))[2]
+    # o_full = g o^P + (1 - g) o^D  =>  o^P - o_full = (1 - g)(o^P - o^D)
+    dist = ~prox
+    a = (K_a[dist] @ q_a) / np.sqrt(d)
+    w = np.exp(a - a.max()); w /= w.sum()
+    oD = w @ V_l[dist]
+    np.testing.assert_allclose(o0 - full, (1 - g) * (o0 - oD), rtol=0, atol=1e-12)
+    # no distant tokens: nothing to skip, result is dense attention
+    o_s, g_s, sk = O.pod_attention_gate_skip(q_l, q_a, K_l[:10], K_a[:10], V_l[:10], S, W, tau=0.0)
+    assert g_s == 1.0 and not sk
+
+
+def test_gate_skip_applies_to_non_lowest_layers_only_and_is_monotone_in_tau():
+    rng = np.random.default_rng(6)
+    L, n, Hq, Hkv, d, S, W = 4, 80, 4, 2, 8, 2, 10
+    q, K, V = _inputs(rng, L, n, Hq, Hkv, d)
+    K[1, S:n - W] *= 0.05                                       # irrelevant: layer 1 scores with layer 0's keys
+    q[0] *= 0.2                                                 # weak distant logits for block 0 ...
+    q[1] *= 3.0                                                 # ... strong proximal ones at layer 1
+    for l in range(L):
+        info = []
+        got = O.pod_decode_layer(q, K, V, l, group_size=2, n_s=S, n_r=W, tau=0.0, info=info)
+        if l % 2 == 0:                                          # lowest layers never skip
+            assert all(not sk for _, sk in info)
+            np.testing.assert_array_equal(got, O.pod_decode_layer(q, K, V, l, group_size=2, n_s=S, n_r=W))
+        else:
+            assert all(sk for _, sk in info)
+    prev = None
+    for tau in (1.1, 0.9, 0.7, 0.5, 0.3, 0.0):
+        info = []
+        O.pod_decode_layer(q, K, V, 1, group_size=2, n_s=S, n_r=W, tau=tau, info=info)
+        skipped = [sk for _, sk in info]
+        assert skipped == [g >= tau for g, _ in info]
+        if prev is not None:
+            assert all(b or not a for a, b in zip(prev, skipped))     # once skipped, skipped for smaller tau
+        prev = skipped
+    gs = [g for g, _ in info]
+    assert max(gs) > 0.5                                              # the construction gives a confident gate
