@@ -191,7 +191,7 @@ def run_ours(args):
     head_wise = "head_wise_new_block_p" in w
     total_steps = args.warmup + args.steps
     e2e_steps = max(3, min(args.steps, 20))
-    extra = 2 * total_steps + 2 * (e2e_steps + 3) + 8     # headroom for every timed pass
+    extra = 2 * total_steps + 2 * (e2e_steps + 3) + 12    # headroom for every timed pass
     dev = torch.device("cuda", local)
     stream = torch.cuda.current_stream().cuda_stream
 
@@ -244,7 +244,17 @@ def run_ours(args):
         else:
             for l in range(L):
                 cache.append_decode_attn(l, kpi[l], vpi[l], qpi[l], op[l], stream)
-            launches[0] += L * cache.last_launch()["n_kernels"]
+            launches[0] += launches_per_step
+
+    launches_per_step = L          # one launch per layer; set after the first step if the gate adds launches
+
+    def count_launches_per_step(cache):
+        """Kernels one step launches (a gated layer is two launches), counted on one untimed step."""
+        i, total = 0, 0
+        for l in range(L):
+            cache.append_decode_attn(l, kp[i][l], vp[i][l], qp[i][l], op[l], stream)
+            total += cache.last_launch()["n_kernels"]
+        return total
 
     def barrier():
         torch.cuda.synchronize()
@@ -270,6 +280,9 @@ def run_ours(args):
         return reduce_max(x, dist, dev)
 
     cache = build_cache(G, use_map=head_wise)
+    if args.gate_tau is not None:
+        cache.set_gate_threshold(args.gate_tau)
+        launches_per_step = count_launches_per_step(cache)
     sampler = ClockSampler(local) if rank == 0 else None
     if sampler:
         sampler.start()
@@ -361,6 +374,7 @@ def run_ours(args):
                    "n_recent": W, "l2": "inputs larger than L2 (a step reads %.1f GiB)" % (L * alg_bytes / 2**30),
                    "blocks": ("head-wise, seeded" if head_wise else "runs of %d layers" % G) +
                              ": %d of %d (layer, KV head) pairs keep their own distant keys" % (n_low_pairs, L * Hkv),
+                   "gate_tau": args.gate_tau,
                    "split_tokens": geo["split_tokens"], "ctas": geo["n_ctas"]},
         "decode_tokens_per_s": round(agg["decode_tokens_per_s"], 1),
         "hbm_gbs_step": round(L * alg_bytes / (ms * 1e-3 / args.steps) / 1e9, 1),
@@ -476,6 +490,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-KV baseline leg")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--gate-tau", type=float, default=None,
+                    help="gate threshold of the distant-skip approximation (default: off, exact attention)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

@@ -163,6 +163,21 @@ int pod_decode_attn(pod_cache* c, int layer, const void* q_device, void* out_dev
 int pod_append_decode_attn(pod_cache* c, int layer, const void* k_device, const void* v_device,
                            const void* q_device, void* out_device, void* cuda_stream);
 
+/* Gate threshold of the paper's appendix "Computation Optimization for Distant Tokens".  For a head
+ * of a layer that is not the lowest layer of the head's block, the gate of Eq. 2,
+ * g = sum exp(a^P) / (sum exp(a^P) + sum exp(a^D)), can be evaluated before any distant value is
+ * read: a^D are the lowest layer's logits, whose sum that layer has left behind.  With a threshold
+ * 0 <= tau <= 1 set, such a head omits its distant tokens when g >= tau: its output is then the
+ * softmax over its proximal tokens alone (reading of "omitted": the gate is taken as 1).  Heads of
+ * lowest layers, and heads that cannot use their block's stored logits (see pod_decode_attn's call
+ * order), always attend to everything.  tau > 1 (the default) switches the gate off.  A gated
+ * pod_decode_attn / pod_append_decode_attn of such a layer runs as two launches: the proximal
+ * tokens, then the distant tokens of the KV heads in which some query head did not skip (the
+ * distant values are shared by the query heads of a KV head).  The decision is taken in fp32 on
+ * the device; results depend on tau by design (an approximation, as in the paper).
+ * Errors: INVALID (tau negative or not a number). */
+int pod_cache_set_gate_threshold(pod_cache* c, float tau);
+
 /* Byte accounting (host integers).  Live bytes of a sequence of length n (at the layer with
  * the most tokens): row * H_kv * (L * (2 n_p + n_d) + ceil(L / G) * n_d), n_p = min(n, n_s+n_r),
  * n_d = n - n_p; the saving against dense is (n_d / n) (1 - ceil(L/G)/L) / 2 -- only keys
@@ -226,7 +241,7 @@ const char* pod_strerror(int status);
  * the counters that must start at zero on the given stream.  Two calls whose kernels may run at
  * the same time on one device (different streams, different threads) race on the array: order
  * them.  Asynchronous on cuda_stream like pod_decode_attn. */
-#define POD_STATIC_SCRATCH_BYTES 2138368
+#define POD_STATIC_SCRATCH_BYTES 2171136
 int pod_dense_decode_attn_static(const void* kv_device, int capacity, int n_tokens,
                                  const void* q_device, void* out_device, int n_q_heads,
                                  int n_kv_heads, int head_dim, float sm_scale, void* cuda_stream);

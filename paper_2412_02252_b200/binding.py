@@ -48,6 +48,7 @@ def _load() -> ctypes.CDLL:
         "pod_cache_write": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_void_p]),
         "pod_decode_attn": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
         "pod_append_decode_attn": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+        "pod_cache_set_gate_threshold": (c_int, [c_void_p, c_float]),
         "pod_cache_bytes": (c_int64, [c_void_p, c_int]),
         "pod_cache_seq_len": (c_int, [c_void_p, c_int, c_int]),
         "pod_cache_reset": (c_int, [c_void_p, c_int]),
@@ -68,7 +69,7 @@ def _load() -> ctypes.CDLL:
 lib = _load()
 EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_required_bytes_blocks",
            "pod_cache_create_blocks", "pod_greedy_layer_blocks", "pod_cache_destroy", "pod_cache_write",
-           "pod_decode_attn", "pod_append_decode_attn", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
+           "pod_decode_attn", "pod_append_decode_attn", "pod_cache_set_gate_threshold", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
            "pod_cache_read_region", "pod_cache_device_status", "pod_cache_last_cuda_error",
            "pod_cache_last_launch", "pod_strerror", "pod_dense_decode_attn_static"]
 
@@ -169,6 +170,9 @@ class PodCache:
     def append_decode_attn(self, layer: int, k, v, q, out, stream: int = 0) -> int:
         return _check(lib.pod_append_decode_attn(self._h, layer, _ptr(k), _ptr(v), _ptr(q), _ptr(out), stream),
                       "pod_append_decode_attn")
+
+    def set_gate_threshold(self, tau: float) -> int:
+        return _check(lib.pod_cache_set_gate_threshold(self._h, tau), "pod_cache_set_gate_threshold")
 
     def bytes(self, which: int) -> int:
         return lib.pod_cache_bytes(self._h, which)

@@ -81,7 +81,7 @@ bool build_block_map(const pod_config& c, const int32_t* lowest, BlockMap* m) {
 struct Carve {
   std::vector<int64_t> seq_row_base;   // rows
   std::vector<int32_t> seq_cap_d;
-  size_t off_len, off_rowbase, off_capd, off_low, off_slot, off_stash, off_pacc, off_pml, off_err, off_sched, total;
+  size_t off_len, off_rowbase, off_capd, off_low, off_slot, off_stash, off_pacc, off_pml, off_dlse, off_sacc, off_sml, off_err, off_sched, total;
   int64_t total_rows;
   int max_splits;
 };
@@ -115,7 +115,10 @@ bool carve(const pod_config& c, const BlockMap& m, const int32_t* cap, Carve* ou
   out->off_slot = off;     off = align_up(off + (size_t)c.n_layers * c.n_kv_heads * 4);
   out->off_stash = off;    off = align_up(off + (size_t)m.n_slots * c.batch * (c.n_q_heads / c.n_kv_heads) * row_bytes);
   out->off_pacc = off;     off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * c.head_dim * 4);
-  out->off_pml = off;      off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * 2 * 4);
+  out->off_pml = off;      off = align_up(off + (size_t)c.batch * c.n_q_heads * out->max_splits * 4 * 4);
+  out->off_dlse = off;     off = align_up(off + (size_t)c.batch * c.n_q_heads * 4);
+  out->off_sacc = off;     off = align_up(off + (size_t)c.batch * c.n_q_heads * c.head_dim * 4);
+  out->off_sml = off;      off = align_up(off + (size_t)c.batch * c.n_q_heads * 2 * 4);
   out->off_err = off;      off = align_up(off + 4);
   out->off_sched = off;    off = align_up(off + (size_t)c.batch * c.n_kv_heads * SCHED_STRIDE * 4);
   out->total = off;
@@ -142,13 +145,14 @@ struct pod_cache {
   int force_split_tokens = 0;          // POD_SPLIT_TOKENS > 0 overrides the planner
   int force_chunk_tiles = 0;           // POD_CHUNK_TILES > 0 overrides the tiles per draw
   int static_eighths = 5;              // POD_STATIC_EIGHTHS: share of a warp's chunks assigned without a draw
+  float gate_tau = 2.f;                // gate threshold; above 1 = the distant tokens are never skipped
   float scale = 0.f;
   Layout y{};
   CUtensorMap tmap{};                  // the region rows of the arena as a [rows][d] bf16 tensor
   // last launch (diagnostics)
   int32_t last_split_tokens = 0, last_ctas = 0, last_kernels = 0;
   // planner memo
-  int64_t memo_sum = -1; int32_t memo_max = -1; int memo_light = -1; DecodePlan memo_plan{};
+  int64_t memo_sum = -1; int32_t memo_max = -1; int memo_light = -1, memo_segment = -1; DecodePlan memo_plan{};
 
   // Device lengths are kept twice.  A launch that appends and attends at once reads one copy and
   // writes the other (its CTAs start at different times, so nobody may change what they read);
@@ -197,15 +201,19 @@ bool make_tensor_map(pod_cache* c) {
 // (SMs x resident CTAs), every CTA costs its rows plus a fixed overhead.  A head that reads keys and
 // values streams 2 n rows, a head that reads the block's stored logits n + n_p; n_light heads of
 // this launch are of the second kind.
-DecodePlan plan_decode(pod_cache* c, int layer, int n_light) {
+DecodePlan plan_decode(pod_cache* c, int layer, int n_light, int segment) {
   const pod_config& g = c->cfg;
   const int n_heavy = g.n_kv_heads - n_light;
   const int64_t SW = (int64_t)g.n_sink + g.n_recent;
   int64_t sum = 0; int32_t nmax = 0;
   for (int b = 0; b < g.batch; ++b) { const int32_t n = c->h_len(layer, b); sum += n; if (n > nmax) nmax = n; }
-  if (sum == c->memo_sum && nmax == c->memo_max && n_light == c->memo_light) return c->memo_plan;
-  auto heavy_rows = [](int64_t n) { return 2 * n; };
-  auto light_rows = [SW](int64_t n) { return n + (n < SW ? n : SW); };
+  if (sum == c->memo_sum && nmax == c->memo_max && n_light == c->memo_light && segment == c->memo_segment)
+    return c->memo_plan;
+  // segment 1 streams the proximal tokens only, segment 2 the distant tokens only, 0 both
+  auto prox = [SW, segment](int64_t n) { return segment == 2 ? (int64_t)0 : (n < SW ? n : SW); };
+  auto dist = [SW, segment](int64_t n) { return segment == 1 ? (int64_t)0 : (n > SW ? n - SW : (int64_t)0); };
+  auto heavy_rows = [&](int64_t n) { return 2 * (prox(n) + dist(n)); };
+  auto light_rows = [&](int64_t n) { return 2 * prox(n) + dist(n); };
   auto count = [&](int64_t st, int64_t* ctas, int64_t* most) {
     *ctas = 0; *most = 0;
     for (int b = 0; b < g.batch; ++b) {
@@ -218,13 +226,13 @@ DecodePlan plan_decode(pod_cache* c, int layer, int n_light) {
   };
   const int64_t wmax = n_heavy > 0 ? heavy_rows(nmax) : light_rows(nmax);
   DecodePlan best{2, 1, 0};
-  if (nmax > 0 && c->force_split_tokens > 0) {      // POD_SPLIT_TOKENS: tuning experiments
+  if (wmax > 0 && c->force_split_tokens > 0) {      // POD_SPLIT_TOKENS: tuning experiments
     int64_t st = 2 * (int64_t)c->force_split_tokens;
     if (st < (wmax + c->cv.max_splits - 1) / c->cv.max_splits) st = (wmax + c->cv.max_splits - 1) / c->cv.max_splits;
     int64_t ctas, most;
     count(st, &ctas, &most);
     best = DecodePlan{(int32_t)st, (int32_t)most, (int32_t)ctas};
-  } else if (nmax > 0) {
+  } else if (wmax > 0) {
     const int64_t slots = (int64_t)c->sm_count * c->resident;
     double best_cost = 1e300;
     int64_t last_st = -1;
@@ -240,7 +248,7 @@ DecodePlan plan_decode(pod_cache* c, int layer, int n_light) {
       if (st <= 128) break;
     }
   }
-  c->memo_sum = sum; c->memo_max = nmax; c->memo_light = n_light; c->memo_plan = best;
+  c->memo_sum = sum; c->memo_max = nmax; c->memo_light = n_light; c->memo_segment = segment; c->memo_plan = best;
   return best;
 }
 
@@ -488,19 +496,12 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     for (int b = 0; b < g.batch; ++b) same = same && c->score_len[(size_t)h * g.batch + b] == c->h_len(layer, b);
     if (same) { p.score_read_mask[h >> 5] |= 1u << (h & 31); ++n_light; }
   }
-  const DecodePlan plan = plan_decode(c, layer, n_light);
-  p.split_rows = plan.split_rows; p.max_splits = c->cv.max_splits;
-  {
-    // A warp sees about split_rows / (2 x tile tokens x warps) tiles; it should make a dozen draws.
-    int tch = plan.split_rows / (2 * decode_tile_tokens() * decode_warps_per_cta() * 16);
-    if (c->force_chunk_tiles > 0) tch = c->force_chunk_tiles;
-    p.tiles_per_chunk = tch < 1 ? 1 : (tch > 256 ? 256 : tch);
-    p.static_eighths = c->static_eighths;
-  }
-  // A launch that appends and attends streams only rows written before this step (the new token's
-  // and the displaced token's rows are handled apart); the one launch that may still be running is
-  // the previous one on this cache, which touches other rows if it was a decode of another layer.
-  p.early_ok = (fused && c->last_decode_layer >= 0 && c->last_decode_layer != layer) ? 1 : 0;
+  p.dlse = reinterpret_cast<float*>(c->arena + c->cv.off_dlse);
+  p.state_acc = reinterpret_cast<float*>(c->arena + c->cv.off_sacc);
+  p.state_ml = reinterpret_cast<float*>(c->arena + c->cv.off_sml);
+  p.gate_tau = c->gate_tau;
+  p.max_splits = c->cv.max_splits;
+  p.static_eighths = c->static_eighths;
   p.by_value = g.batch <= SMALL_BATCH ? 1 : 0;
   for (int b = 0; b < SMALL_BATCH; ++b) {
     const bool in = p.by_value && b < g.batch;
@@ -508,16 +509,40 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     p.v_cap_d[b] = in ? c->cv.seq_cap_d[b] : 0;
     p.v_row_base[b] = in ? c->cv.seq_row_base[b] : 0;
   }
+  // With a gate threshold set, a layer in which some head reads its block's logits runs as two
+  // launches: the proximal tokens (which decides, per query head, whether the distant tokens are
+  // omitted), then the distant tokens of the KV heads that still need them.
+  const bool gated = c->gate_tau <= 1.f && n_light > 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int kernels = 0;
-  if (plan.n_ctas > 0) {
+  DecodePlan plan{2, 1, 0};
+  for (int pass = 0; pass < (gated ? 2 : 1); ++pass) {
+    p.segment = gated ? pass + 1 : 0;
+    plan = plan_decode(c, layer, n_light, p.segment);
+    p.split_rows = plan.split_rows;
+    {
+      // A warp sees about split_rows / (2 x tile tokens x warps) tiles; it should make a dozen draws.
+      int tch = plan.split_rows / (2 * decode_tile_tokens() * decode_warps_per_cta() * 16);
+      if (c->force_chunk_tiles > 0) tch = c->force_chunk_tiles;
+      p.tiles_per_chunk = tch < 1 ? 1 : (tch > 256 ? 256 : tch);
+    }
+    // A launch that appends and attends streams only rows written before this step (the new token's
+    // and the displaced token's rows are handled apart); the one launch that may still be running is
+    // the previous one on this cache, which touches other rows if it was a decode of another layer.
+    // The distant launch of a gated layer follows its own proximal launch, which moved rows: no early start.
+    p.early_ok = (fused && pass == 0 && c->last_decode_layer >= 0 && c->last_decode_layer != layer) ? 1 : 0;
+    if (pass == 1) {                      // the append is done: the distant launch only attends
+      p.new_k = nullptr; p.new_v = nullptr; p.len_out = nullptr;
+      p.len = c->d_len(layer);
+    }
+    if (plan.n_ctas == 0) continue;
     const int e = launch_decode(c->tmap, p, plan.grid_splits, s);
     if (e != 0) {
-      if (fused) { for (int b = 0; b < g.batch; ++b) c->h_len(layer, b) -= 1; c->memo_sum = -1; }
+      if (fused && pass == 0) { for (int b = 0; b < g.batch; ++b) c->h_len(layer, b) -= 1; c->memo_sum = -1; }
       return cuda_fail(c, (cudaError_t)e);
     }
     ++kernels;
-    if (fused) c->len_cur[layer] ^= 1;
+    if (fused && pass == 0) c->len_cur[layer] ^= 1;
   }
   {
     bool any_empty = false;
@@ -535,8 +560,14 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     for (int b = 0; b < g.batch; ++b) c->score_len[(size_t)h * g.batch + b] = c->h_len(layer, b);
   }
   c->last_decode_layer = layer;
-  c->last_split_tokens = plan.split_rows / 2; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;
+  c->last_split_tokens = plan.split_rows / 2; c->last_ctas = plan.n_ctas; c->last_kernels = kernels;   // of the last launch
   return POD_OK;
+}
+
+int pod_cache_set_gate_threshold(pod_cache* c, float tau) {
+  if (!c || !(tau >= 0.f)) return POD_ERR_INVALID;      // rejects NaN too
+  c->gate_tau = tau;
+  return c->dry ? POD_DRY_RUN : POD_OK;
 }
 
 int pod_decode_attn(pod_cache* c, int layer, const void* q, void* out, void* stream) {

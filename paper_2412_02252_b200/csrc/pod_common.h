@@ -28,6 +28,7 @@ constexpr int DECODE_CTAS_PER_SM = POD_DECODE_CTAS_PER_SM;  // register budget o
 // Scheduling words of one (sequence, KV head): 128 bytes apart so that heads do not share a line.
 constexpr int SCHED_STRIDE = 32;      // int32 per (sequence, KV head)
 constexpr int SCHED_TICKET = 16;      // [0] = chunk counter, [SCHED_TICKET] = finished-CTA tickets
+constexpr int SCHED_NEED = 2;         // [SCHED_NEED] = query heads of this KV head that still need their distant tokens (gate)
 
 // Physical layout of the arena.  All offsets are in rows; one row is one head's d bf16
 // values (128 B at d = 64, 256 B at d = 128), so every region base is 128-byte aligned.
@@ -119,10 +120,22 @@ struct DecodeParams {
   const uint16_t* q;       // [B][H_q][D] queries of this layer
   uint16_t* stash;         // [n_slots][B][r][D]: a head's lowest layer saves its queries for the block here
   float* part_acc;         // [B][H_q][max_splits][D]
-  float* part_ml;          // [B][H_q][max_splits][2]  (running max in log2 units, sum)
+  float* part_ml;          // [B][H_q][max_splits][4]  (running max in log2 units, sum, distant part of the sum, -)
   uint16_t* out;           // [B][H_q][D]
   int32_t* err_flag;
   int32_t* sched;          // [B][H_kv][SCHED_STRIDE] zeroed chunk counters and tickets (the kernel re-zeroes them)
+  // Gate threshold (paper appendix "Computation Optimization for Distant Tokens"): a gated decode of a
+  // layer is two launches.  segment 1 streams the proximal tokens only and evaluates the gate of
+  // Eq. 2 per query head against the distant log-sum-exp its block's lowest layer left in dlse: heads
+  // that skip (g >= gate_tau), or have no distant tokens, get their final output; the others leave
+  // their proximal state (acc, max, sum) and a bit in the SCHED_NEED word.  segment 2 streams the
+  // distant tokens of KV heads with a bit set and merges with that state.  segment 0 = one launch over
+  // the whole context, no gate.
+  int32_t segment;
+  float gate_tau;
+  float* dlse;             // [B][H_q] log2 of the sum of 2^logit over the distant tokens, written by a head's lowest layer
+  float* state_acc;        // [B][H_q][D]
+  float* state_ml;         // [B][H_q][2]
   int32_t layer, max_splits;
   int32_t split_rows;      // K or V rows a CTA should stream: a head that reads keys and values has 2 n rows of
                            // work, a head that reads stored logits n + n_p; its CTAs = ceil(work / split_rows)

@@ -161,10 +161,10 @@ struct Cfg {
   static constexpr int N_BARS = NW * NSTAGE + NW;     // one per stage, one per warp for the combine
   static constexpr int SMEM = RING_B + SC_B + N_BARS * 8 + 1024;   // + slack to align to 1024
   // the combine reuses each warp's ring: (max, sum) pairs, split weights, then partial rows
-  static constexpr int CML_OFF = 0, CW_OFF = MAX_SPLITS_CAP * 8, CROW_OFF = CW_OFF + MAX_SPLITS_CAP * 4;
+  static constexpr int CML_OFF = 0, CW_OFF = MAX_SPLITS_CAP * 16, CROW_OFF = CW_OFF + MAX_SPLITS_CAP * 4;
   static constexpr int CROWS = (WARP_B - CROW_OFF) / (D * 4);   // partial rows per round
   static_assert(CROWS >= 8, "a warp's ring must hold a few partial rows for the combine");
-  static_assert(WARP_B >= (8 * D + 16) * 4, "merge scratch must fit the warp's ring");
+  static_assert(WARP_B >= (8 * D + 24) * 4, "merge scratch must fit the warp's ring");
 };
 
 template <int D>
@@ -218,6 +218,8 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
 
   // ---- tiles and chunks of this (sequence, KV head) -----------------------------------------
   const int n_p = min(n, y.S + y.W), n_d = n - n_p;
+  // a gated decode streams the proximal tokens (segment 1) and the distant tokens (segment 2) in two launches
+  const int n_p_s = p.segment == 2 ? 0 : n_p, n_d_s = p.segment == 1 ? 0 : n_d;
   // A layer that reads the block's stored logits needs no key rows: its distant tiles hold 32
   // value rows (both halves of a stage), so the bytes in flight per stage stay the same.
   // blocks are per KV head: is this layer the lowest of this head's block, and does the block go on?
@@ -228,11 +230,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const bool sc_read = !is_low && kvh < 256 && ((p.score_read_mask[kvh >> 5] >> (kvh & 31)) & 1u);
   // CTAs of this head: in proportion to the rows it streams (keys and values, or values and the
   // proximal keys only), so that heads with different roles in one launch finish together
-  const int64_t work_rows = sc_read ? (int64_t)n + min(n, y.S + y.W) : 2 * (int64_t)n;
+  const int64_t work_rows = sc_read ? (int64_t)n_p_s * 2 + n_d_s : 2 * ((int64_t)n_p_s + n_d_s);
   const int nsplit = (int)min((int64_t)p.max_splits, (work_rows + p.split_rows - 1) / p.split_rows);
   if (split >= nsplit) return;
   const int DT = sc_read ? 2 * TOK : TOK;         // tokens per distant tile
-  const int ntp = (n_p + TOK - 1) / TOK, ntd = (n_d + DT - 1) / DT;
+  const int ntp = (n_p_s + TOK - 1) / TOK, ntd = (n_d_s + DT - 1) / DT;
   const int ntiles = ntp + ntd;
   const int tch = p.tiles_per_chunk;
   const int nwh = nsplit * NW;                    // warps working on this head
@@ -251,6 +253,8 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int sc_group_b = score_group_bytes(y);
   unsigned char* sc_base = reinterpret_cast<unsigned char*>(const_cast<uint16_t*>(p.arena)) +
                            (seq_row + score_row(y, kvh, cap_d)) * (int64_t)(D * 2);
+
+  if (p.segment == 2 && sched[SCHED_NEED] == 0) return;   // every query head of this KV head skipped: no distant work
 
   // ---- the warp's walk over its chunks (all values uniform across the warp) -----------------
   if (!waited && k_static * tch < NSTAGE) {       // the first tiles need draws: no early start
@@ -379,6 +383,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
 #pragma unroll
   for (int cb = 0; cb < D / 16; ++cb) { ot[cb][0] = ot[cb][1] = ot[cb][2] = ot[cb][3] = 0.f; }
   float m_row = -INFINITY, l_row = 0.f;   // running max (log2 units) and sum of head qrow
+  float ld_row = 0.f;                     // the distant tokens' part of l_row (same scaling)
   bool failed = false;
   uint32_t round = 0;                     // stage s holds its (round)-th tile: barrier parity round & 1
   int fail_stage = 0;
@@ -411,7 +416,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     __syncwarp();
     // one token: logit of head qrow from this lane's Q fragments (quad-reduced), then the same
     // online-softmax update as a tile, in fp32
-    auto add_token = [&](const uint16_t* krow, const uint16_t* vrow, const uint32_t (&qf)[D / 16][2], float* logit_dst) {
+    auto add_token = [&](const uint16_t* krow, const uint16_t* vrow, const uint32_t (&qf)[D / 16][2], float* logit_dst, bool distant) {
       float dot = 0.f;
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
@@ -430,6 +435,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       const float pr = ex2(a - m_new);
       m_row = m_new;
       l_row = l_row * alpha + ((lane & 3) == 0 ? pr : 0.f);   // l_row holds per-lane partial sums
+      ld_row = ld_row * alpha + ((distant && (lane & 3) == 0) ? pr : 0.f);
       const float al0 = __shfl_sync(0xffffffffu, alpha, qcol * 4), al1 = __shfl_sync(0xffffffffu, alpha, qcol * 4 + 4);
       const float p0 = __shfl_sync(0xffffffffu, pr, qcol * 4), p1 = __shfl_sync(0xffffffffu, pr, qcol * 4 + 4);
 #pragma unroll
@@ -440,11 +446,12 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
         ot[cb][2] = ot[cb][2] * al0 + p0 * v1; ot[cb][3] = ot[cb][3] * al1 + p1 * v1;
       }
     };
-    add_token(s_sp[0], s_sp[1], qp, nullptr);           // the new token is proximal: own query
-    if (rB >= 0) {                                      // the displaced token is distant: block's query
+    add_token(s_sp[0], s_sp[1], qp, nullptr, false);    // the new token is proximal: own query
+    if (rB >= 0 && p.segment != 1) {                    // the displaced token is distant: block's query (a
+                                                        // proximal-only launch leaves it to the distant launch)
       float* slot = reinterpret_cast<float*>(sc_base + (int64_t)(rB / TOK) * sc_group_b + (qrow * 4 + ((cB & 7) >> 1)) * 16) +
                     ((cB >> 3) * 2 + (cB & 1));
-      add_token(s_sp[2], s_sp[3], qd, sc_write ? slot : nullptr);
+      add_token(s_sp[2], s_sp[3], qd, sc_write ? slot : nullptr, true);
     }
   }
 
@@ -509,7 +516,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       // one online-softmax step (base 2) over 16 tokens: logits l (log2 units; tokens qcol, +1,
       // +8, +9 of head qrow), `cnt` valid tokens, token `mcol` left out, value fragments vf
       auto softmax_pv = [&](float l00, float l01, float l10, float l11, int cnt, int mcol, const uint32_t (&vf)[D / 16][4],
-                            float* store) {
+                            float* store, bool distant) {
         float a00 = (qcol < cnt && qcol != mcol) ? l00 : -INFINITY;
         float a01 = (qcol + 1 < cnt && qcol + 1 != mcol) ? l01 : -INFINITY;
         float a10 = (qcol + 8 < cnt && qcol + 8 != mcol) ? l10 : -INFINITY;
@@ -532,6 +539,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
           const float alpha = ex2(m_row - m_new);     // 0 on the first tile, 1 if unchanged
           m_row = m_new;
           l_row *= alpha;
+          ld_row *= alpha;
           // the accumulators of this lane belong to heads qcol and qcol + 1
           const float al0 = __shfl_sync(0xffffffffu, alpha, qcol * 4);
           const float al1 = __shfl_sync(0xffffffffu, alpha, qcol * 4 + 4);
@@ -542,6 +550,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
         const float m_use = (m_row == -INFINITY) ? 0.f : m_row;
         a00 = ex2(a00 - m_use); a01 = ex2(a01 - m_use); a10 = ex2(a10 - m_use); a11 = ex2(a11 - m_use);
         l_row += (a00 + a01) + (a10 + a11);
+        if (distant) ld_row += (a00 + a01) + (a10 + a11);
         const uint32_t pb0 = pack_bf16(a00, a01), pb1 = pack_bf16(a10, a11);
         // O^T += V^T P^T
 #pragma unroll
@@ -549,8 +558,8 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       };
 
       if (from_scores) {
-        softmax_pv(sca.x, sca.y, sca.z, sca.w, min(TOK, rem), mtile, fa, nullptr);
-        if (rem > TOK) softmax_pv(scb.x, scb.y, scb.z, scb.w, min(TOK, rem - TOK), mtile - TOK, fb, nullptr);
+        softmax_pv(sca.x, sca.y, sca.z, sca.w, min(TOK, rem), mtile, fa, nullptr, true);
+        if (rem > TOK) softmax_pv(scb.x, scb.y, scb.z, scb.w, min(TOK, rem - TOK), mtile - TOK, fb, nullptr, true);
       } else {
         // S = Q K^T, two accumulation chains per token half
         float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -568,7 +577,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
         if (dist && sc_write && qrow < r)
           store = reinterpret_cast<float*>(sc_base + (int64_t)(vt - ntp) * sc_group_b + (qrow * 4 + (lane & 3)) * 16);
         softmax_pv((s0[0] + t0[0]) * p.scale_log2, (s0[1] + t0[1]) * p.scale_log2, (s1[0] + t1[0]) * p.scale_log2,
-                   (s1[1] + t1[1]) * p.scale_log2, min(TOK, rem), mtile, fb, store);
+                   (s1[1] + t1[1]) * p.scale_log2, min(TOK, rem), mtile, fb, store, dist);
       }
     }
   }
@@ -587,8 +596,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // ---- merge the warps of the CTA -------------------------------------------------------------
   l_row += __shfl_xor_sync(0xffffffffu, l_row, 1);
   l_row += __shfl_xor_sync(0xffffffffu, l_row, 2);
+  ld_row += __shfl_xor_sync(0xffffffffu, ld_row, 1);
+  ld_row += __shfl_xor_sync(0xffffffffu, ld_row, 2);
   __syncwarp();
-  float* mine = reinterpret_cast<float*>(wbuf);    // [8 heads][D] acc, then [8] max, [8] sum
+  float* mine = reinterpret_cast<float*>(wbuf);    // [8 heads][D] acc, then [8] max, [8] sum, [8] distant sum
   if (qcol < r) {
 #pragma unroll
     for (int cb = 0; cb < D / 16; ++cb) {
@@ -600,7 +611,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       }
     }
   }
-  if ((lane & 3) == 0) { mine[8 * D + qrow] = m_row; mine[8 * D + 8 + qrow] = l_row; }
+  if ((lane & 3) == 0) { mine[8 * D + qrow] = m_row; mine[8 * D + 8 + qrow] = l_row; mine[8 * D + 16 + qrow] = ld_row; }
   __syncthreads();
 
   for (int idx = threadIdx.x; idx < r * D; idx += NW * 32) {
@@ -609,7 +620,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
 #pragma unroll
     for (int w = 0; w < NW; ++w)
       M = fmaxf(M, reinterpret_cast<const float*>(smem + w * C::WARP_B)[8 * D + h]);
-    float a = 0.f, l = 0.f;
+    float a = 0.f, l = 0.f, ld = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) {
       const float* ow = reinterpret_cast<const float*>(smem + w * C::WARP_B);
@@ -617,10 +628,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       const float sc = (mw == -INFINITY) ? 0.f : ex2(mw - M);
       a += ow[h * D + c] * sc;
       l += ow[8 * D + 8 + h] * sc;
+      ld += ow[8 * D + 16 + h] * sc;
     }
     const int64_t ph = ((int64_t)b * y.H_q + kvh * r + h) * p.max_splits + split;
     p.part_acc[ph * D + c] = a;
-    if (c == 0) { p.part_ml[ph * 2] = M; p.part_ml[ph * 2 + 1] = l; }
+    if (c == 0) *reinterpret_cast<float4*>(p.part_ml + ph * 4) = make_float4(M, l, ld, 0.f);
   }
 
   // ---- ticket: the CTA that publishes the last partial of this (sequence, KV head) combines ----
@@ -633,7 +645,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     int got;
     asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(got) : "l"(sched + SCHED_TICKET) : "memory");
     s_last = (got == nsplit - 1);
-    if (s_last) { sched[SCHED_TICKET] = 0; sched[0] = 0; }   // ready for the next launch
+    if (s_last) {                                            // ready for the next launch
+      sched[SCHED_TICKET] = 0; sched[0] = 0;
+      if (p.segment == 1) sched[SCHED_NEED] = 0;             // this CTA's warps set the bits below
+    }
   }
   __syncthreads();
   if (!s_last) return;
@@ -646,46 +661,68 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int64_t ph0 = ((int64_t)b * y.H_q + kvh * r) * p.max_splits;     // partial row of (head 0, split 0)
   uint32_t cphase = 0;
   bool cfail = false;
+  const int need_in = p.segment == 2 ? sched[SCHED_NEED] : 0;   // heads that left a proximal state to merge with
   for (int h = warp; h < r && !cfail; h += NW) {
+    if (p.segment == 2 && !((need_in >> h) & 1)) continue;      // this head took its output from the proximal launch
     const int64_t ph = ph0 + (int64_t)h * p.max_splits;
+    const int64_t hq = (int64_t)b * y.H_q + kvh * r + h;         // query head
     float acc[CPL];
 #pragma unroll
     for (int j = 0; j < CPL; ++j) acc[j] = 0.f;
-    float inv = 0.f;
+    float inv = 0.f, m_all = -INFINITY, l_all = 0.f;
+    // state of the proximal launch (segment 2): one more partial (max, sum, acc); requested early
+    float st_m = -INFINITY, st_l = 0.f, st_w = 0.f, st_acc[CPL];
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) st_acc[j] = 0.f;
+    if (p.segment == 2) {
+      st_m = p.state_ml[hq * 2]; st_l = p.state_ml[hq * 2 + 1];
+#pragma unroll
+      for (int j = 0; j < CPL; ++j) st_acc[j] = p.state_acc[hq * D + lane * CPL + j];
+    }
     for (int r0 = 0; r0 < nsplit; r0 += C::CROWS) {
       const int r1 = min(nsplit, r0 + C::CROWS);
       if (lane == 0) {
         fence_async_global();
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        const uint32_t ml_bytes = (uint32_t)p.max_splits * 8u;
+        const uint32_t ml_bytes = (uint32_t)p.max_splits * 16u;
         mbar_expect_tx(cbar, (uint32_t)(r1 - r0) * D * 4u + (r0 == 0 ? ml_bytes : 0u));
-        if (r0 == 0) bulk_load(w_ml, p.part_ml + ph * 2, ml_bytes, cbar);
+        if (r0 == 0) bulk_load(w_ml, p.part_ml + ph * 4, ml_bytes, cbar);
         bulk_load(w_rows, p.part_acc + (ph + r0) * D, (uint32_t)(r1 - r0) * D * 4u, cbar);
       }
       if (!__all_sync(0xffffffffu, mbar_wait(cbar, cphase & 1))) { cfail = true; break; }
       ++cphase;
       if (r0 == 0) {                          // weights 2^(m_s - M) of the splits and 1 / sum, once per head
-        float2 ml[MAX_SPLITS_CAP / 32];
-        float mloc = -INFINITY;
+        float4 ml[MAX_SPLITS_CAP / 32];       // (max, sum, distant part of the sum, -) of a split
+        float mloc = st_m;
 #pragma unroll
         for (int k = 0; k < MAX_SPLITS_CAP / 32; ++k) {
           const int sp = lane + 32 * k;
-          ml[k] = sp < nsplit ? lds_f32x2(w_ml + sp * 8) : make_float2(-INFINITY, 0.f);
+          ml[k] = sp < nsplit ? lds_f32x4(w_ml + sp * 16) : make_float4(-INFINITY, 0.f, 0.f, 0.f);
           mloc = fmaxf(mloc, ml[k].x);
         }
 #pragma unroll
         for (int o2 = 16; o2 >= 1; o2 >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o2));
-        float lloc = 0.f;
+        float lloc = 0.f, ldloc = 0.f;
 #pragma unroll
         for (int k = 0; k < MAX_SPLITS_CAP / 32; ++k) {
           const int sp = lane + 32 * k;
           const float wgt = (ml[k].x == -INFINITY) ? 0.f : ex2(ml[k].x - mloc);
           if (sp < nsplit) sts_f32(w_w + sp * 4, wgt);
           lloc += ml[k].y * wgt;
+          ldloc += ml[k].z * wgt;
         }
 #pragma unroll
-        for (int o2 = 16; o2 >= 1; o2 >>= 1) lloc += __shfl_xor_sync(0xffffffffu, lloc, o2);
+        for (int o2 = 16; o2 >= 1; o2 >>= 1) {
+          lloc += __shfl_xor_sync(0xffffffffu, lloc, o2);
+          ldloc += __shfl_xor_sync(0xffffffffu, ldloc, o2);
+        }
+        st_w = (st_m == -INFINITY) ? 0.f : ex2(st_m - mloc);
+        lloc += st_l * st_w;
+        m_all = mloc; l_all = lloc;
         inv = lloc > 0.f ? 1.f / lloc : 0.f;
+        // the head's lowest layer leaves the log-sum-exp of its distant logits for the gate of the
+        // block's other layers (a proximal-only launch sees no distant token: the distant launch writes it)
+        if (sc_write && p.segment != 1 && lane == 0) p.dlse[hq] = ldloc > 0.f ? mloc + __log2f(ldloc) : -INFINITY;
         __syncwarp();
       }
       // eight rows per trip, the last trip padded with weight 0 on a valid row
@@ -713,7 +750,30 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       __syncwarp();                           // the rows are overwritten by the next round
     }
     if (cfail) break;
-    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * y.H_q + kvh * r + h) * D + lane * CPL;
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) acc[j] += st_acc[j] * st_w;
+    if (p.segment == 1) {
+      // Gate of Eq. 2 from the proximal sum of this launch and the distant sum the block's lowest
+      // layer left: g = S_P / (S_P + S_D).  A head that reads the block's logits and has g >= tau
+      // omits its distant tokens; so does any head without distant tokens.  The others leave their
+      // proximal state for the distant launch.
+      bool final_out = n_d == 0;
+      if (!final_out && sc_read) {
+        const float lse_p = m_all + __log2f(l_all), lse_d = p.dlse[hq];
+        const float g = 1.f / (1.f + ex2(lse_d - lse_p));
+        final_out = g >= p.gate_tau;
+      }
+      if (!final_out) {
+        if (lane == 0) {
+          p.state_ml[hq * 2] = m_all; p.state_ml[hq * 2 + 1] = l_all;
+          atomicOr(sched + SCHED_NEED, 1 << h);
+        }
+#pragma unroll
+        for (int j = 0; j < CPL; ++j) p.state_acc[hq * D + lane * CPL + j] = acc[j];
+        continue;
+      }
+    }
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + hq * D + lane * CPL;
 #pragma unroll
     for (int j = 0; j < CPL; j += 2)
       *reinterpret_cast<__nv_bfloat162*>(dst + j) = __floats2bfloat162_rn(acc[j] * inv, acc[j + 1] * inv);

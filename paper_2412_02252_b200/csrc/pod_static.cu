@@ -21,9 +21,9 @@ constexpr int STATIC_MAX_Q_HEADS = 64;
 constexpr int STATIC_MAX_SPLITS = 64;
 constexpr int STATIC_MAX_DEVICES = 64;
 constexpr size_t OFF_PACC = 0;                                                         // fp32 [64][64][128]
-constexpr size_t OFF_PML = (size_t)STATIC_MAX_Q_HEADS * STATIC_MAX_SPLITS * 128 * 4;   // fp32 [64][64][2]
+constexpr size_t OFF_PML = (size_t)STATIC_MAX_Q_HEADS * STATIC_MAX_SPLITS * 128 * 4;   // fp32 [64][64][4]
 constexpr size_t SCHED_BYTES = (size_t)STATIC_MAX_Q_HEADS * SCHED_STRIDE * 4;          // int32 [64 KV heads][32]
-constexpr size_t OFF_SCHED = OFF_PML + (size_t)STATIC_MAX_Q_HEADS * STATIC_MAX_SPLITS * 2 * 4;
+constexpr size_t OFF_SCHED = OFF_PML + (size_t)STATIC_MAX_Q_HEADS * STATIC_MAX_SPLITS * 4 * 4;
 constexpr size_t OFF_ERR = OFF_SCHED + SCHED_BYTES;
 constexpr size_t STATIC_BYTES = OFF_ERR + 256;
 static_assert(STATIC_BYTES == POD_STATIC_SCRATCH_BYTES, "header and library disagree on the scratch size");
@@ -131,6 +131,7 @@ extern "C" int pod_dense_decode_attn_static(const void* kv_device, int capacity,
   p.scale_log2 = (sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim)) * 1.4426950408889634f;
   for (int w = 0; w < 8; ++w) p.score_read_mask[w] = 0u;
   p.early_ok = 0;
+  p.segment = 0; p.gate_tau = 2.f; p.dlse = nullptr; p.state_acc = nullptr; p.state_ml = nullptr;
   p.by_value = 1;
   p.v_len[0] = n_tokens; p.v_cap_d[0] = 0; p.v_row_base[0] = 0;
 

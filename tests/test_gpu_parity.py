@@ -303,6 +303,81 @@ def test_head_wise_blocks_from_greedy_grouping_many_tiles():
                 assert_close(outs[l, b, h], case.oracle_head(l, b, h), f"layer {l} seq {b} head {h}")
 
 
+def _gate_case(seed, n, lowest=None, G=2):
+    """Inputs for the gate tests: the queries of some heads of the non-lowest layers are scaled up, so
+    that their proximal logits dominate (g close to 1), others are left alone (g small)."""
+    case = Case(seed=seed, L=4, G=G, Hq=8, Hkv=2, d=128, S=4, W=64, lens=[n], caps=[n + 8], lowest=lowest)
+    dev = "cuda"
+    K = [case.kv(synth.TAG_K, l, 0, 0, n + 2, dev) for l in range(case.L)]
+    V = [case.kv(synth.TAG_V, l, 0, 0, n + 2, dev) for l in range(case.L)]
+    gain = torch.tensor([[1, 1, 1, 1, 1, 1, 1, 1], [4, 1, 3, 1, 4, 4, 3, 5], [1, 1, 1, 1, 1, 1, 1, 1],
+                         [1, 5, 1, 2.5, 1, 1, 1, 1]], dtype=torch.float32, device=dev)
+    qs = [[(case.q(l, step, dev).float() * gain[l][None, :, None]).to(torch.bfloat16) for l in range(case.L)]
+          for step in range(2)]
+    return case, K, V, qs
+
+
+def _gate_check(case, K, V, q_step, outs, n, tau, expect_some=True):
+    """Every head against the oracle's gated result; a head whose g lies within 0.01 of tau may match
+    either candidate (the device takes the decision in fp32 from its own sums)."""
+    Kh = torch.stack([k[:n] for k in K]).double().cpu().numpy()
+    Vh = torch.stack([v[:n] for v in V]).double().cpu().numpy()
+    qh = torch.stack([q[0] for q in q_step]).double().cpu().numpy()
+    kinds = set()
+    for l in range(case.L):
+        info = []
+        kw = dict(lowest=np.array(case.lowest), n_s=case.S, n_r=case.W)
+        ref = O.pod_decode_layer(qh, Kh, Vh, l, tau=tau, info=info, **kw)
+        for h in range(case.Hq):
+            g, skipped = info[h]
+            if g is not None and abs(g - tau) < 0.01:
+                alt = O.pod_decode_layer(qh, Kh, Vh, l, tau=(0.0 if not skipped else 2.0), **kw)[h]
+                got = outs[l, 0, h].double().cpu().numpy()
+                assert min(np.abs(got - ref[h]).max(), np.abs(got - alt).max()) <= 1e-2
+                continue
+            assert_close(outs[l, 0, h], ref[h], f"tau {tau} layer {l} head {h} g {g} skipped {skipped}")
+            kinds.add(("skip" if skipped else "full") if g is not None else "lowest")
+    if expect_some:
+        assert kinds == {"skip", "full", "lowest"}, kinds
+
+
+@pytest.mark.parametrize("head_wise", [False, True])
+def test_gate_threshold_skips_distant_tokens(head_wise):
+    """pod_cache_set_gate_threshold: heads of non-lowest layers whose gate g reaches tau give the softmax
+    over their proximal tokens alone, the others (and all heads of lowest layers) the full result; both
+    kinds occur inside one KV head.  Two-call form, then one-launch steps; tau = 0 and tau off."""
+    n = 1500
+    lowest = [[0, 0], [0, 1], [2, 1], [2, 1]] if head_wise else None
+    case, K, V, qs = _gate_case(19, n, lowest=lowest)
+    cache = case.make_cache()
+    stream = torch.cuda.current_stream().cuda_stream
+    for l in range(case.L):
+        cache.write(l, 0, K[l][:n], V[l][:n], n, stream)
+    outs = torch.empty(case.L, 1, case.Hq, case.d, dtype=torch.bfloat16, device="cuda")
+
+    def decode(q_step):
+        for l in range(case.L):
+            cache.decode_attn(l, q_step[l], outs[l], stream)
+        torch.cuda.synchronize()
+
+    for tau in (0.5, 0.0, 2.0):
+        cache.set_gate_threshold(tau)
+        decode(qs[0])
+        _gate_check(case, K, V, qs[0], outs, n, tau, expect_some=(tau == 0.5))
+    assert cache.last_launch()["n_kernels"] == 1                     # gate off: one launch
+    cache.set_gate_threshold(0.5)
+    for step in (1, 2):                                              # one-launch form with the gate on
+        for l in range(case.L):
+            cache.append_decode_attn(l, K[l][n + step - 1:n + step], V[l][n + step - 1:n + step], qs[step - 1][l],
+                                     outs[l], stream)
+        torch.cuda.synchronize()
+        _gate_check(case, K, V, qs[step - 1], outs, n + step, 0.5)
+    assert cache.last_launch()["n_kernels"] == 2                     # proximal launch + distant launch
+    assert cache.device_status() == B.POD_OK
+    with pytest.raises(B.PodError):
+        cache.set_gate_threshold(-0.1)
+
+
 def test_custom_scale():
     case = Case(seed=6, L=2, G=2, Hq=4, Hkv=1, d=64, S=2, W=6, lens=[50], scale=0.31)
     cache = case.make_cache()
