@@ -195,6 +195,37 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     stream = torch.cuda.current_stream().cuda_stream
 
+    def time_prefill_write(reps=6):
+        """pod_cache_write of one sequence's whole context (n tokens, one call per layer) into a
+        two-layer cache with blocks of two layers: layer 0 keeps its distant keys, layer 1 drops them.
+        Calls are issued back to back (each appends n more tokens) and timed with CUDA events."""
+        T_ = min(n, 32768)
+        cfg = B.make_config(n_layers=2, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, group_size=2,
+                            n_sink=S, n_recent=W, batch=1, device=local)
+        pc = B.PodCache(cfg, [T_ * (reps + 2)])
+        k = synth.gen_kv(seed, synth.TAG_K, 0, 0, 0, T_, Hkv, d, outliers=w["outliers"], device=dev)
+        v = synth.gen_kv(seed, synth.TAG_V, 0, 0, 0, T_, Hkv, d, outliers=w["outliers"], device=dev)
+        out, row = {}, d * 2
+        for l, name in ((0, "lowest_layer"), (1, "other_layer")):
+            pc.write(l, 0, k, v, T_, stream)                      # fills the window; untimed
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                pc.write(l, 0, k, v, T_, stream)
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / reps
+            keeps = Hkv if l == 0 else 0                          # heads whose distant keys this layer keeps
+            # read: every value row, the key rows that are kept (all for layer 0, the last W for layer 1),
+            # and the W rows per head and kind that leave the ring; written: the same rows at their new places
+            rows = T_ * Hkv + T_ * keeps + W * (Hkv - keeps) + W * (Hkv + keeps)
+            out[name] = {"us": round(us, 2), "gbs": round(2 * rows * row / (us * 1e-6) / 1e9, 1)}
+        pc.destroy()
+        out["tokens_per_call"] = T_
+        out["note"] = "bytes read + written per call over the mean of back-to-back calls"
+        return out
+
     def build_cache(group, use_map=False):
         cfg = B.make_config(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, group_size=group,
                             n_sink=S, n_recent=W, batch=Bn, device=local)
@@ -335,6 +366,7 @@ def run_ours(args):
     del cache
     torch.cuda.empty_cache()
 
+    prefill = time_prefill_write() if rank == 0 else None
     # ---- dense-KV baseline: the same kernels with every layer its own block (G = 1) ---------------
     dense_us = None
     if world == 1 and not args.no_dense:
@@ -392,6 +424,7 @@ def run_ours(args):
         "gpu_launches": n_launch,
         "clocks": clocks,
         "cache_bytes": {"pod_live": live, "dense_equiv": dense_equiv, "saving": round(1 - live / dense_equiv, 5)},
+        "prefill_write": prefill,
         "two_call_us_per_layer_step": round(ms_two * 1e3 / (args.steps * L * world), 3),
         "dense_kv_baseline_us_per_layer_step": None if dense_us is None else round(dense_us, 3),
     }

@@ -105,6 +105,7 @@ struct WriteParams {
   const uint16_t* v;
   int32_t* len;          // device lengths of this layer, [B]
   int32_t layer, seq, n0, T;
+  int32_t bulk_blocks;   // leading blocks of the grid that copy tokens going straight to the distant stores
 };
 
 struct DecodeParams {
