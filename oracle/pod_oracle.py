@@ -237,6 +237,24 @@ def pod_decode_layer(q, K, V, layer, *, group_size=None, lowest=None, n_s, n_r, 
     return out
 
 
+def pod_prefill_layer(q, K, V, layer, *, group_size=None, lowest=None, n_s, n_r, scale=None):
+    """PoD attention of one layer for EVERY position of a sequence (prefill; Section 2.2 and the
+    masks of Fig. 2, middle): position i attends to the tokens up to and including itself, the
+    proximal ones being the first n_s and the last n_r of those, exactly as the decode step of a
+    sequence that ends at i does.
+
+    q: [L][n][H_q][d] queries of every layer and position; K, V: [L][n][H_kv][d].
+    Returns o [n][H_q][d] (float64).  Written as n independent decode steps on prefixes.
+    """
+    L, n, H_kv, d = K.shape
+    H_q = q.shape[2]
+    out = np.zeros((n, H_q, d))
+    for i in range(n):
+        out[i] = pod_decode_layer(q[:, i], K[:, :i + 1], V[:, :i + 1], layer, group_size=group_size,
+                                  lowest=lowest, n_s=n_s, n_r=n_r, scale=scale)
+    return out
+
+
 # --------------------------------------------------------------------------------------
 # the PoD cache layout, maintained token by token (layout form)
 # --------------------------------------------------------------------------------------

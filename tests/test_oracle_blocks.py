@@ -246,3 +246,38 @@ def test_gate_skip_applies_to_non_lowest_layers_only_and_is_monotone_in_tau():
         prev = skipped
     gs = [g for g, _ in info]
     assert max(gs) > 0.5                                              # the construction gives a confident gate
+
+
+# --------------------------------------------------------------------------- prefill (all positions)
+def test_prefill_oracle_against_causal_attention_and_explicit_masks():
+    """For a lowest layer the prefill form is ordinary causal attention (torch SDPA, is_causal); for
+    another layer it equals a softmax over a matrix of logits assembled with the proximal / distant
+    masks of Fig. 2 (middle) written out explicitly; its last row is the decode step."""
+    import torch
+    rng = np.random.default_rng(8)
+    L, n, Hq, Hkv, d, S, W = 2, 45, 4, 2, 8, 3, 7
+    bf = lambda x: (x.astype(np.float32).view(np.uint32) & 0xFFFF0000).view(np.float32).astype(np.float64)
+    q = bf(rng.standard_normal((L, n, Hq, d)))
+    K, V = bf(rng.standard_normal((L, n, Hkv, d))), bf(rng.standard_normal((L, n, Hkv, d)))
+    r = Hq // Hkv
+    o0 = O.pod_prefill_layer(q, K, V, 0, group_size=2, n_s=S, n_r=W)
+    for h in range(Hq):
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            torch.tensor(q[0, :, h])[None], torch.tensor(K[0, :, h // r])[None], torch.tensor(V[0, :, h // r])[None],
+            is_causal=True)[0].numpy()
+        np.testing.assert_allclose(o0[:, h], ref, rtol=0, atol=1e-12)
+    o1 = O.pod_prefill_layer(q, K, V, 1, group_size=2, n_s=S, n_r=W)
+    i = np.arange(n)[:, None]
+    j = np.arange(n)[None, :]
+    causal = j <= i
+    prox = (j < S) | (j > i - W)                 # the last W tokens up to and including i
+    for h in range(Hq):
+        kv = h // r
+        own = q[1, :, h] @ K[1, :, kv].T / np.sqrt(d)
+        low = q[0, :, h] @ K[0, :, kv].T / np.sqrt(d)
+        a = np.where(prox, own, low)
+        a = np.where(causal, a, -np.inf)
+        w = np.exp(a - a.max(axis=1, keepdims=True))
+        w /= w.sum(axis=1, keepdims=True)
+        np.testing.assert_allclose(o1[:, h], w @ V[1, :, kv], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(o1[-1], O.pod_decode_layer(q[:, -1], K, V, 1, group_size=2, n_s=S, n_r=W), rtol=0, atol=0)
