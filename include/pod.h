@@ -210,6 +210,28 @@ int pod_cache_last_launch(const pod_cache* c, int32_t* split_tokens, int32_t* n_
 
 const char* pod_strerror(int status);
 
+/* PoD attention for every position of a sequence (prefill; Section 2.2, Eq. 1, Eq. 2 and the masks of
+ * Fig. 2, middle), from the layer's dense projections, on the tcgen05 tensor cores.  Position i attends
+ * to positions j <= i; of those the first n_sink and the last n_recent (i included) are proximal, with
+ * logits sm_scale <q[i][h], k[j][h / r]>; the others are distant, with logits
+ * sm_scale <q_low[i][h], k_low[j][h / r]>, q_low / k_low being the queries and keys of the lowest layer
+ * of the head's block.  out[i][h] = one softmax over both groups applied to v.  It is what
+ * pod_decode_attn returns at each step of a sequence fed token by token.
+ *   q, q_low, out : device bf16 [n_tokens][n_q_heads][head_dim];  k, k_low, v : device bf16
+ *                   [n_tokens][n_kv_heads][head_dim]; head_dim must be 128.
+ *   q_low, k_low  : NULL for a layer that is the lowest of every head's block (ordinary causal attention).
+ *   head_shares   : host int32 [n_kv_heads] or NULL; with q_low given, KV head h takes its distant logits
+ *                   from q_low / k_low if head_shares is NULL or head_shares[h] != 0 (head-wise blocks).
+ * The cache is not touched: write k, v with pod_cache_write.  Runs on the current device; the first call
+ * on a device allocates one status word and looks up the driver's tensor-map encoder.  Asynchronous on
+ * cuda_stream.  Errors: INVALID, CUDA.  pod_prefill_status synchronises the device and returns
+ * POD_ERR_DEVICE if a launch gave up a bounded wait since the last call (its output is then invalid). */
+int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, int n_sink, int n_recent,
+                     float sm_scale, const void* q_device, const void* k_device, const void* v_device,
+                     const void* q_low_device, const void* k_low_device, const int32_t* head_shares,
+                     void* out_device, void* cuda_stream);
+int pod_prefill_status(void);
+
 /* Decode attention without any allocation.  (The paper has no counterpart of this call; it is a
  * packaging variant of pod_decode_attn for one sequence of ordinary, unshared K/V.)
  *

@@ -57,6 +57,9 @@ def _load() -> ctypes.CDLL:
         "pod_cache_last_cuda_error": (c_int, [c_void_p]),
         "pod_cache_last_launch": (c_int, [c_void_p, P(c_int32), P(c_int32), P(c_int32)]),
         "pod_strerror": (c_char_p, [c_int]),
+        "pod_prefill_attn": (c_int, [c_int, c_int, c_int, c_int, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p,
+                                     c_void_p, c_void_p, P(c_int32), c_void_p, c_void_p]),
+        "pod_prefill_status": (c_int, []),
         "pod_dense_decode_attn_static": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_int,
                                                  c_int, c_float, c_void_p]),
     }
@@ -71,7 +74,7 @@ EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_required_b
            "pod_cache_create_blocks", "pod_greedy_layer_blocks", "pod_cache_destroy", "pod_cache_write",
            "pod_decode_attn", "pod_append_decode_attn", "pod_cache_set_gate_threshold", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
            "pod_cache_read_region", "pod_cache_device_status", "pod_cache_last_cuda_error",
-           "pod_cache_last_launch", "pod_strerror", "pod_dense_decode_attn_static"]
+           "pod_cache_last_launch", "pod_strerror", "pod_prefill_attn", "pod_prefill_status", "pod_dense_decode_attn_static"]
 
 
 class PodError(RuntimeError):
@@ -201,6 +204,21 @@ class PodCache:
         a, b, c = c_int32(), c_int32(), c_int32()
         lib.pod_cache_last_launch(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
         return {"split_tokens": a.value, "n_ctas": b.value, "n_kernels": c.value}
+
+
+def pod_prefill_attn(q, k, v, out, *, n_sink: int, n_recent: int, q_low=None, k_low=None, head_shares=None,
+                     sm_scale: float = 0.0, stream: int = 0) -> int:
+    """PoD attention for every position (prefill) from dense bf16 projections ``q`` [T][H_q][128],
+    ``k``, ``v`` [T][H_kv][128]; ``q_low``/``k_low``: the lowest layer's, for layers that share."""
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    hs = None if head_shares is None else (c_int32 * Hkv)(*[int(x) for x in head_shares])
+    return _check(lib.pod_prefill_attn(T, Hq, Hkv, d, n_sink, n_recent, sm_scale, _ptr(q), _ptr(k), _ptr(v),
+                                       _ptr(q_low), _ptr(k_low), hs, _ptr(out), stream), "pod_prefill_attn")
+
+
+def pod_prefill_status() -> int:
+    return lib.pod_prefill_status()
 
 
 def pod_dense_decode_attn_static(kv, capacity: int, n_tokens: int, q, out, n_q_heads: int, n_kv_heads: int,

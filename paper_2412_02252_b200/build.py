@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpod_b200.so")
-SOURCES = ["pod_api.cu", "pod_write.cu", "pod_decode.cu", "pod_static.cu"]
+SOURCES = ["pod_api.cu", "pod_write.cu", "pod_decode.cu", "pod_static.cu", "pod_prefill.cu"]
 
 
 def _nvcc() -> str:

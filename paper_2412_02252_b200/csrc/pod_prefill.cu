@@ -1,0 +1,415 @@
+// pod_prefill_attn: PoD attention for every position of a sequence (Section 2.2, Eq. 1 and the
+// masks of Fig. 2, middle) on the 5th-generation tensor cores: tcgen05.mma with operands staged
+// in shared memory by TMA and accumulators in tensor memory.
+//
+// Position i attends to positions j <= i.  Of those the first n_s and the last n_r are proximal:
+// their logits are q_l[i] . k_l[j]; the others are distant: their logits are q_a[i] . k_a[j] with a
+// the lowest layer of the head's block (for a head whose block starts at this layer both are the
+// same product).  One softmax over both groups weighs layer l's own values.
+//
+// One CTA = 128 consecutive query positions of one query head; 128 threads, thread t owns query
+// row t.  Key/value tiles of 64 positions stream through a two-stage shared-memory ring (TMA,
+// 128-byte swizzle).  Per tile:
+//   S_own[128 x 64] = Q K^T and, where the tile holds distant tokens of a sharing head,
+//   S_low[128 x 64] = Q_a K_a^T               (tcgen05.mma, M = 128, N = 64, K = 16 x 8 steps, into TMEM)
+//   each thread reads its row of S from TMEM (tcgen05.ld), picks own/low per key, masks, runs the
+//   online softmax in base 2 and writes its row of P (bf16) into a swizzled shared-memory tile
+//   O_tile[128 x 128] = P V                   (tcgen05.mma, A = P K-major, B = V MN-major, K = 16 x 4)
+//   each thread reads its row of O_tile and folds it into its fp32 output row in registers.
+// Tiles that are entirely proximal (or entirely distant) skip the product they do not need.  This
+// first version issues the two products of a tile one after the other (no overlap of softmax and
+// MMA).  Every wait is bounded; a wait that gives up raises the error flag, and the tensor memory
+// is always returned before the CTA exits.
+#include <cudaTypedefs.h>
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include <mutex>
+
+#include "../../include/pod.h"
+#include "pod_common.h"
+
+namespace pod {
+namespace {
+
+constexpr int PD = 128;                 // head_dim
+constexpr int BM = 128;                 // query rows per CTA
+constexpr int BN = 64;                  // keys per tile
+constexpr int NSTG = 2;
+constexpr uint32_t PF_WAIT_LIMIT = 1u << 22;
+
+constexpr int Q_B = BM * PD * 2;        // 32 KiB: two [128][128 B] sub-tiles
+constexpr int KV_B = BN * PD * 2;       // 16 KiB: two [64][128 B] sub-tiles
+constexpr int STAGE_B = 3 * KV_B;       // K, K of the lowest layer, V
+constexpr int P_B = BM * BN * 2;        // 16 KiB: one [128][128 B] tile
+constexpr int OFF_Q = 0, OFF_QL = Q_B, OFF_ST = 2 * Q_B, OFF_P = OFF_ST + NSTG * STAGE_B;
+constexpr int OFF_BAR = OFF_P + P_B;
+constexpr int PF_SMEM = OFF_BAR + 128 + 1024;
+constexpr int TM_COLS = 256;            // S_own 64 + S_low 64 + O_tile 128 fp32 columns
+constexpr int TM_SLOW = 64, TM_O = 128;
+
+struct PrefillParams {
+  int32_t T, H_q, H_kv, S, W;
+  float scale_log2;
+  uint32_t share_mask[8];               // bit h: KV head h takes distant logits from the lowest layer's q, k
+  uint16_t* out;                        // [T][H_q][128] bf16
+  int32_t* err_flag;
+};
+
+__device__ __forceinline__ uint32_t s2u(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < PF_WAIT_LIMIT; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+// [rows][64 bf16] box of a [T][H][128] tensor at (channel x, head, row t); x is 0 or 64
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int x, int head, int t, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(head), "r"(t), "r"(bar) : "memory");
+}
+// Shared-memory matrix descriptor of the tensor cores (128-byte swizzle, descriptor version of
+// sm_100): start address, leading and stride byte offsets in units of 16 bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128; B K-major or MN-major
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// this thread's 32 consecutive fp32 columns of its TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(BM, 1)
+pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQl,
+                   const __grid_constant__ CUtensorMap tmKl, const PrefillParams p) {
+  extern __shared__ unsigned char pf_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pf_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sb = s2u(smem);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;          // long rows first
+  const int hq = blockIdx.y, kvh = hq / (p.H_q / p.H_kv);
+  const int q0 = qb * BM;
+  const bool shares = kvh < 256 && ((p.share_mask[kvh >> 5] >> (kvh & 31)) & 1u);
+  const uint32_t bar_q = sb + OFF_BAR, bar_full = sb + OFF_BAR + 8, bar_s = sb + OFF_BAR + 24, bar_o = sb + OFF_BAR + 32;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 64);
+
+  if (tid == 0) {
+    bar_init(bar_q, 1);
+    bar_init(bar_full, 1);
+    bar_init(bar_full + 8, 1);
+    bar_init(bar_s, 1);
+    bar_init(bar_o, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {                                              // tensor memory for S_own, S_low, O_tile
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s2u(tmem_slot)), "r"(TM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tm = *tmem_slot;
+
+  // keys this block needs: positions [0, min(T, q0 + 128)); tile j covers [64 j, 64 j + 64)
+  const int k_end = min(p.T, q0 + BM);
+  const int n_tiles = (k_end + BN - 1) / BN;
+  // a tile is entirely proximal for every row of the block if it starts after qmax - W (or lies in the
+  // sink), entirely distant if it lies in [S, qmin - W]
+  auto tile_needs = [&](int j, bool& need_own, bool& need_low) {
+    const int k0 = j * BN, k1 = k0 + BN - 1;
+    const bool prox_all = (k1 < p.S) || (k0 > q0 + BM - 1 - p.W);
+    const bool dist_all = (k0 >= p.S) && (k1 <= q0 - p.W);
+    need_low = shares && !prox_all;
+    need_own = !shares || !dist_all;
+  };
+  auto load_tile = [&](int j) {                                 // thread 0
+    const int s = j & 1;
+    bool need_own, need_low;
+    tile_needs(j, need_own, need_low);
+    const uint32_t st = sb + OFF_ST + s * STAGE_B, bar = bar_full + s * 8;
+    bar_expect_tx(bar, KV_B * (1 + (need_own ? 1 : 0) + (need_low ? 1 : 0)));
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      if (need_own) tma_load_3d(st + c * (KV_B / 2), &tmK, c * 64, kvh, j * BN, bar);
+      if (need_low) tma_load_3d(st + KV_B + c * (KV_B / 2), &tmKl, c * 64, kvh, j * BN, bar);
+      tma_load_3d(st + 2 * KV_B + c * (KV_B / 2), &tmV, c * 64, kvh, j * BN, bar);
+    }
+  };
+  if (tid == 0) {
+    bar_expect_tx(bar_q, Q_B * (shares ? 2 : 1));
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      tma_load_3d(sb + OFF_Q + c * (Q_B / 2), &tmQ, c * 64, hq, q0, bar_q);
+      if (shares) tma_load_3d(sb + OFF_QL + c * (Q_B / 2), &tmQl, c * 64, hq, q0, bar_q);
+    }
+    load_tile(0);
+    if (n_tiles > 1) load_tile(1);
+  }
+
+  const int qi = q0 + tid;                                      // this thread's query position
+  float o[PD];
+#pragma unroll
+  for (int c = 0; c < PD; ++c) o[c] = 0.f;
+  float m_row = -INFINITY, l_row = 0.f;
+  bool fail = false;
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;       // this warp's quarter of the TMEM lanes
+  constexpr uint32_t IDESC_S = instr_desc(BN, false), IDESC_O = instr_desc(PD, true);
+
+  for (int j = 0; j < n_tiles; ++j) {
+    const int s = j & 1;
+    bool need_own, need_low;
+    tile_needs(j, need_own, need_low);
+    const uint32_t st = sb + OFF_ST + s * STAGE_B;
+    // ---- S = Q K^T ----------------------------------------------------------------------------------
+    if (tid == 0) {
+      bool ok = bar_wait(bar_full + s * 8, (j >> 1) & 1);
+      if (j == 0) ok = ok && bar_wait(bar_q, 0);
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < PD / 16; ++ks) {                  // 16 channels per step: 4 per 128-byte sub-tile
+          const uint32_t a_off = (ks >> 2) * (Q_B / 2) + (ks & 3) * 32, b_off = (ks >> 2) * (KV_B / 2) + (ks & 3) * 32;
+          if (need_own)
+            umma(tm, smem_desc(sb + OFF_Q + a_off, 16, 1024), smem_desc(st + b_off, 16, 1024), IDESC_S, ks > 0);
+          if (need_low)
+            umma(tm + TM_SLOW, smem_desc(sb + OFF_QL + a_off, 16, 1024), smem_desc(st + KV_B + b_off, 16, 1024), IDESC_S, ks > 0);
+        }
+      }
+      umma_commit(bar_s);                                       // arrives when the products above are done
+      if (!ok) fail = true;
+    }
+    fail = fail || !bar_wait(bar_s, j & 1);
+    if (__syncthreads_or(fail)) { fail = true; break; }
+    tc_fence_after();
+
+    // ---- this thread's row: logits, mask, online softmax, P -----------------------------------------
+    const int k0 = j * BN;
+    auto logit = [&](float own, float low, int kj) -> float {
+      const bool valid = kj <= qi && kj < p.T;
+      const bool prox = kj < p.S || kj > qi - p.W;
+      const float a = (need_low && (!need_own || !prox)) ? low : own;
+      return valid ? a * p.scale_log2 : -INFINITY;
+    };
+    float mx = -INFINITY;
+#pragma unroll
+    for (int ch = 0; ch < BN / 32; ++ch) {
+      float so[32], sl[32];
+      if (need_own) tmem_ld32(tm + lane_base + ch * 32, so);
+      if (need_low) tmem_ld32(tm + TM_SLOW + lane_base + ch * 32, sl);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) mx = fmaxf(mx, logit(need_own ? so[i] : 0.f, need_low ? sl[i] : 0.f, k0 + ch * 32 + i));
+    }
+    const float m_new = fmaxf(m_row, mx);
+    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+    const float alpha = ex2f(m_row - m_use);                    // 0 on the first tile
+    m_row = m_new;
+    float psum = 0.f;
+    unsigned char* prow = smem + OFF_P + tid * 128;             // row tid of the [128][128 B] P tile
+#pragma unroll
+    for (int ch = 0; ch < BN / 32; ++ch) {
+      float so[32], sl[32];
+      if (need_own) tmem_ld32(tm + lane_base + ch * 32, so);
+      if (need_low) tmem_ld32(tm + TM_SLOW + lane_base + ch * 32, sl);
+      uint32_t pk[16];
+#pragma unroll
+      for (int i = 0; i < 32; i += 2) {
+        const float p0 = ex2f(logit(need_own ? so[i] : 0.f, need_low ? sl[i] : 0.f, k0 + ch * 32 + i) - m_use);
+        const float p1 = ex2f(logit(need_own ? so[i + 1] : 0.f, need_low ? sl[i + 1] : 0.f, k0 + ch * 32 + i + 1) - m_use);
+        psum += p0 + p1;
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+        pk[i >> 1] = *reinterpret_cast<uint32_t*>(&b2);
+      }
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4) {                          // 16-byte chunk c of row r lives at chunk c ^ (r & 7)
+        const int chunk = ch * 4 + c4;
+        *reinterpret_cast<uint4*>(prow + ((chunk ^ (tid & 7)) << 4)) = make_uint4(pk[c4 * 4], pk[c4 * 4 + 1], pk[c4 * 4 + 2], pk[c4 * 4 + 3]);
+      }
+    }
+    l_row = l_row * alpha + psum;
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor cores
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- O_tile = P V -----------------------------------------------------------------------------------
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < BN / 16; ++ks)                      // 16 keys per step
+        umma(tm + TM_O, smem_desc(sb + OFF_P + ks * 32, 16, 1024), smem_desc(st + 2 * KV_B + ks * 2048, KV_B / 2, 1024),
+             IDESC_O, ks > 0);
+      umma_commit(bar_o);
+    }
+    fail = !bar_wait(bar_o, j & 1);
+    if (__syncthreads_or(fail)) { fail = true; break; }
+    tc_fence_after();
+#pragma unroll
+    for (int ch = 0; ch < PD / 32; ++ch) {
+      float t[32];
+      tmem_ld32(tm + TM_O + lane_base + ch * 32, t);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[ch * 32 + i] = o[ch * 32 + i] * alpha + t[i];
+    }
+    tc_fence_before();
+    __syncthreads();                                            // stage s, P and the TMEM tiles are free again
+    if (tid == 0 && j + 2 < n_tiles) load_tile(j + 2);
+  }
+
+  if (fail) {
+    if (tid == 0) atomicExch(p.err_flag, 1);
+  } else if (qi < p.T) {
+    const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+    uint16_t* dst = p.out + ((int64_t)qi * p.H_q + hq) * PD;
+#pragma unroll
+    for (int c = 0; c < PD; c += 8) {
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(o[c + 2 * i] * inv, o[c + 2 * i + 1] * inv);
+        w[i] = *reinterpret_cast<uint32_t*>(&b2);
+      }
+      *reinterpret_cast<uint4*>(dst + c) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+  // return the tensor memory; after a failed wait first give outstanding work a bounded chance to land
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    if (fail && tid == 0) { bar_wait(bar_full, 0); bar_wait(bar_full + 8, 0); }
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(TM_COLS) : "memory");
+  }
+}
+
+struct PrefillSetup {
+  bool ready = false;
+  PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+  int32_t* err = nullptr;       // device word
+};
+PrefillSetup g_pf[64];
+std::mutex g_pf_mutex;
+
+bool encode_3d(PFN_cuTensorMapEncodeTiled_v12000 enc, CUtensorMap* tm, const void* base, int T, int H, int rows) {
+  cuuint64_t dims[3] = {(cuuint64_t)PD, (cuuint64_t)H, (cuuint64_t)T};
+  cuuint64_t strides[2] = {(cuuint64_t)PD * 2, (cuuint64_t)H * PD * 2};
+  cuuint32_t box[3] = {64u, 1u, (cuuint32_t)rows};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+}  // namespace pod
+
+using namespace pod;
+
+extern "C" int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, int n_sink, int n_recent,
+                                float sm_scale, const void* q, const void* k, const void* v, const void* q_low,
+                                const void* k_low, const int32_t* head_shares, void* out, void* cuda_stream) {
+  if (!q || !k || !v || !out) return POD_ERR_INVALID;
+  if (head_dim != PD || n_tokens < 1 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads != 0) return POD_ERR_INVALID;
+  if (n_sink < 0 || n_recent < 1 || !(sm_scale >= 0.f) || isinf(sm_scale)) return POD_ERR_INVALID;
+  if (n_q_heads > 65535) return POD_ERR_INVALID;
+  if ((q_low == nullptr) != (k_low == nullptr)) return POD_ERR_INVALID;
+  for (const void* ptr : {q, k, v, q_low, k_low, (const void*)out})
+    if (((uintptr_t)ptr % 16) != 0) return POD_ERR_INVALID;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return POD_ERR_CUDA;
+  PrefillSetup* su = &g_pf[dev];
+  {
+    std::lock_guard<std::mutex> lock(g_pf_mutex);
+    if (!su->ready) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+          qres != cudaDriverEntryPointSuccess || fn == nullptr)
+        return POD_ERR_CUDA;
+      if (cudaMalloc(&su->err, 4) != cudaSuccess || cudaMemset(su->err, 0, 4) != cudaSuccess) return POD_ERR_CUDA;
+      if (cudaFuncSetAttribute(pod_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM) != cudaSuccess)
+        return POD_ERR_CUDA;
+      su->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+      su->ready = true;
+    }
+  }
+  PrefillParams p{};
+  p.T = n_tokens; p.H_q = n_q_heads; p.H_kv = n_kv_heads; p.S = n_sink; p.W = n_recent;
+  p.scale_log2 = (sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim)) * 1.4426950408889634f;
+  p.out = static_cast<uint16_t*>(out);
+  p.err_flag = su->err;
+  if (q_low != nullptr)
+    for (int h = 0; h < n_kv_heads && h < 256; ++h)
+      if (head_shares == nullptr || head_shares[h] != 0) p.share_mask[h >> 5] |= 1u << (h & 31);
+  CUtensorMap tq, tk, tv, tql, tkl;
+  const void* ql = q_low ? q_low : q;
+  const void* kl = k_low ? k_low : k;
+  if (!encode_3d(su->encode, &tq, q, n_tokens, n_q_heads, BM) || !encode_3d(su->encode, &tk, k, n_tokens, n_kv_heads, BN) ||
+      !encode_3d(su->encode, &tv, v, n_tokens, n_kv_heads, BN) || !encode_3d(su->encode, &tql, ql, n_tokens, n_q_heads, BM) ||
+      !encode_3d(su->encode, &tkl, kl, n_tokens, n_kv_heads, BN))
+    return POD_ERR_INVALID;
+  dim3 grid((n_tokens + BM - 1) / BM, n_q_heads);
+  pod_prefill_kernel<<<grid, BM, PF_SMEM, static_cast<cudaStream_t>(cuda_stream)>>>(tq, tk, tv, tql, tkl, p);
+  return cudaGetLastError() == cudaSuccess ? POD_OK : POD_ERR_CUDA;
+}
+
+// POD_ERR_DEVICE if a launch of pod_prefill_attn on the current device gave up a bounded wait since the last call.
+extern "C" int pod_prefill_status(void) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return POD_ERR_CUDA;
+  PrefillSetup* su = &g_pf[dev];
+  if (!su->ready) return POD_OK;
+  int32_t flag = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return POD_ERR_CUDA;
+  if (cudaMemcpy(&flag, su->err, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return POD_ERR_CUDA;
+  if (flag != 0 && cudaMemset(su->err, 0, 4) != cudaSuccess) return POD_ERR_CUDA;
+  return flag ? POD_ERR_DEVICE : POD_OK;
+}
