@@ -7,19 +7,21 @@
 // the lowest layer of the head's block (for a head whose block starts at this layer both are the
 // same product).  One softmax over both groups weighs layer l's own values.
 //
-// One CTA = 128 consecutive query positions of one query head; 128 threads, thread t owns query
-// row t.  Key/value tiles of 64 positions stream through a two-stage shared-memory ring (TMA,
-// 128-byte swizzle).  Per tile:
+// One CTA = 128 consecutive query positions of one query head: four softmax warps (thread t owns query
+// row t) and one producer warp whose lane 0 issues every TMA load and every tcgen05.mma.  Key/value tiles
+// of 64 positions stream through a two-stage shared-memory ring (TMA, 128-byte swizzle).  Per tile j:
 //   S_own[128 x 64] = Q K^T and, where the tile holds distant tokens of a sharing head,
-//   S_low[128 x 64] = Q_a K_a^T               (tcgen05.mma, M = 128, N = 64, K = 16 x 8 steps, into TMEM)
-//   each thread reads its row of S from TMEM (tcgen05.ld), picks own/low per key, masks, runs the
-//   online softmax in base 2 and writes its row of P (bf16) into a swizzled shared-memory tile
-//   O_tile[128 x 128] = P V                   (tcgen05.mma, A = P K-major, B = V MN-major, K = 16 x 4)
-//   each thread reads its row of O_tile and folds it into its fp32 output row in registers.
-// Tiles that are entirely proximal (or entirely distant) skip the product they do not need.  This
-// first version issues the two products of a tile one after the other (no overlap of softmax and
-// MMA).  Every wait is bounded; a wait that gives up raises the error flag, and the tensor memory
-// is always returned before the CTA exits.
+//   S_low[128 x 64] = Q_a K_a^T               (M = 128, N = 64, K = 16 x 8 steps, into one of two TMEM buffers:
+//                                              the products of tile j + 1 run while tile j is in the softmax)
+//   each softmax thread reads its row of S from TMEM (tcgen05.ld), picks own/low per key, masks, and
+//   writes its row of P = 2^(logit - m) as bf16 into one of two swizzled shared-memory tiles
+//   O[128 x 128] += P V                       (A = P K-major, B = V MN-major, K = 16 x 4), accumulated in TMEM.
+// The reference maximum m of a row is only raised when the tile's maximum exceeds it by more than 8 (in
+// log2 units): P then stays below 2^8, and the rows of O in TMEM have to be rescaled (tcgen05.ld / st)
+// only on those rare occasions instead of after every tile; row sum and O share the same m, so the
+// quotient is exact either way.  Tiles that are entirely proximal (or entirely distant) skip the product
+// they do not need.  Warps hand buffers to one another through mbarriers; every wait is bounded, a wait
+// that gives up raises the error flag, and the tensor memory is always returned before the CTA exits.
 #include <cudaTypedefs.h>
 #include <cuda_bf16.h>
 #include <math.h>
@@ -43,10 +45,12 @@ constexpr int KV_B = BN * PD * 2;       // 16 KiB: two [64][128 B] sub-tiles
 constexpr int STAGE_B = 3 * KV_B;       // K, K of the lowest layer, V
 constexpr int P_B = BM * BN * 2;        // 16 KiB: one [128][128 B] tile
 constexpr int OFF_Q = 0, OFF_QL = Q_B, OFF_ST = 2 * Q_B, OFF_P = OFF_ST + NSTG * STAGE_B;
-constexpr int OFF_BAR = OFF_P + P_B;
-constexpr int PF_SMEM = OFF_BAR + 128 + 1024;
-constexpr int TM_COLS = 256;            // S_own 64 + S_low 64 + O_tile 128 fp32 columns
-constexpr int TM_SLOW = 64, TM_O = 128;
+constexpr int OFF_BAR = OFF_P + 2 * P_B;
+constexpr int PF_SMEM = OFF_BAR + 256 + 1024;
+constexpr int PF_THREADS = BM + 32;     // four softmax warps + the producer warp
+constexpr int TM_COLS = 512;            // 2 x (S_own 64 + S_low 64) + O 128 fp32 columns, next power of two
+constexpr int TM_SBUF = 128, TM_SLOW = 64, TM_O = 256;
+constexpr float RESCALE_STEP = 8.f;     // raise a row's reference maximum only past this many log2 units
 
 struct PrefillParams {
   int32_t T, H_q, H_kv, S, W;
@@ -120,13 +124,32 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+        "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+        "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+        "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+        "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+        "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void bar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ float ex2f(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 
-__global__ void __launch_bounds__(BM, 1)
+__global__ void __launch_bounds__(PF_THREADS, 1)
 pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQl,
                    const __grid_constant__ CUtensorMap tmKl, const PrefillParams p) {
@@ -134,23 +157,29 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pf_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sb = s2u(smem);
   const int tid = threadIdx.x, warp = tid >> 5;
+  const bool producer = warp == BM / 32;
   const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;          // long rows first
   const int hq = blockIdx.y, kvh = hq / (p.H_q / p.H_kv);
   const int q0 = qb * BM;
   const bool shares = kvh < 256 && ((p.share_mask[kvh >> 5] >> (kvh & 31)) & 1u);
-  const uint32_t bar_q = sb + OFF_BAR, bar_full = sb + OFF_BAR + 8, bar_s = sb + OFF_BAR + 24, bar_o = sb + OFF_BAR + 32;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 64);
+  // mbarriers: Q landed; per stage: K/V landed; per buffer: S ready, S read, P written, P V done
+  const uint32_t bar_q = sb + OFF_BAR, bar_full = bar_q + 8, bar_sfull = bar_q + 24, bar_sempty = bar_q + 40,
+                 bar_pfull = bar_q + 56, bar_pvdone = bar_q + 72;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 128);
 
   if (tid == 0) {
     bar_init(bar_q, 1);
-    bar_init(bar_full, 1);
-    bar_init(bar_full + 8, 1);
-    bar_init(bar_s, 1);
-    bar_init(bar_o, 1);
+    for (int i = 0; i < 2; ++i) {
+      bar_init(bar_full + i * 8, 1);
+      bar_init(bar_sfull + i * 8, 1);
+      bar_init(bar_sempty + i * 8, BM);
+      bar_init(bar_pfull + i * 8, BM);
+      bar_init(bar_pvdone + i * 8, 1);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 0) {                                              // tensor memory for S_own, S_low, O_tile
+  if (producer) {                                               // tensor memory for the S buffers and O
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s2u(tmem_slot)), "r"(TM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -171,160 +200,196 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     need_low = shares && !prox_all;
     need_own = !shares || !dist_all;
   };
-  auto load_tile = [&](int j) {                                 // thread 0
-    const int s = j & 1;
-    bool need_own, need_low;
-    tile_needs(j, need_own, need_low);
-    const uint32_t st = sb + OFF_ST + s * STAGE_B, bar = bar_full + s * 8;
-    bar_expect_tx(bar, KV_B * (1 + (need_own ? 1 : 0) + (need_low ? 1 : 0)));
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      if (need_own) tma_load_3d(st + c * (KV_B / 2), &tmK, c * 64, kvh, j * BN, bar);
-      if (need_low) tma_load_3d(st + KV_B + c * (KV_B / 2), &tmKl, c * 64, kvh, j * BN, bar);
-      tma_load_3d(st + 2 * KV_B + c * (KV_B / 2), &tmV, c * 64, kvh, j * BN, bar);
-    }
-  };
-  if (tid == 0) {
-    bar_expect_tx(bar_q, Q_B * (shares ? 2 : 1));
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      tma_load_3d(sb + OFF_Q + c * (Q_B / 2), &tmQ, c * 64, hq, q0, bar_q);
-      if (shares) tma_load_3d(sb + OFF_QL + c * (Q_B / 2), &tmQl, c * 64, hq, q0, bar_q);
-    }
-    load_tile(0);
-    if (n_tiles > 1) load_tile(1);
-  }
-
-  const int qi = q0 + tid;                                      // this thread's query position
-  float o[PD];
-#pragma unroll
-  for (int c = 0; c < PD; ++c) o[c] = 0.f;
-  float m_row = -INFINITY, l_row = 0.f;
   bool fail = false;
-  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;       // this warp's quarter of the TMEM lanes
-  constexpr uint32_t IDESC_S = instr_desc(BN, false), IDESC_O = instr_desc(PD, true);
 
-  for (int j = 0; j < n_tiles; ++j) {
-    const int s = j & 1;
-    bool need_own, need_low;
-    tile_needs(j, need_own, need_low);
-    const uint32_t st = sb + OFF_ST + s * STAGE_B;
-    // ---- S = Q K^T ----------------------------------------------------------------------------------
-    if (tid == 0) {
-      bool ok = bar_wait(bar_full + s * 8, (j >> 1) & 1);
-      if (j == 0) ok = ok && bar_wait(bar_q, 0);
-      if (ok) {
+  if (producer) {
+    if ((tid & 31) == 0) {
+      constexpr uint32_t IDESC_S = instr_desc(BN, false), IDESC_O = instr_desc(PD, true);
+      auto load_tile = [&](int j) {
+        const int s = j & 1;
+        bool need_own, need_low;
+        tile_needs(j, need_own, need_low);
+        const uint32_t st = sb + OFF_ST + s * STAGE_B, bar = bar_full + s * 8;
+        bar_expect_tx(bar, KV_B * (1 + (need_own ? 1 : 0) + (need_low ? 1 : 0)));
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          if (need_own) tma_load_3d(st + c * (KV_B / 2), &tmK, c * 64, kvh, j * BN, bar);
+          if (need_low) tma_load_3d(st + KV_B + c * (KV_B / 2), &tmKl, c * 64, kvh, j * BN, bar);
+          tma_load_3d(st + 2 * KV_B + c * (KV_B / 2), &tmV, c * 64, kvh, j * BN, bar);
+        }
+      };
+      auto issue_qk = [&](int j) {                              // S[j & 1] = Q K_j^T (own and/or lowest layer's)
+        bool need_own, need_low;
+        tile_needs(j, need_own, need_low);
+        const uint32_t st = sb + OFF_ST + (j & 1) * STAGE_B, ts = tm + (j & 1) * TM_SBUF;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < PD / 16; ++ks) {                  // 16 channels per step: 4 per 128-byte sub-tile
           const uint32_t a_off = (ks >> 2) * (Q_B / 2) + (ks & 3) * 32, b_off = (ks >> 2) * (KV_B / 2) + (ks & 3) * 32;
           if (need_own)
-            umma(tm, smem_desc(sb + OFF_Q + a_off, 16, 1024), smem_desc(st + b_off, 16, 1024), IDESC_S, ks > 0);
+            umma(ts, smem_desc(sb + OFF_Q + a_off, 16, 1024), smem_desc(st + b_off, 16, 1024), IDESC_S, ks > 0);
           if (need_low)
-            umma(tm + TM_SLOW, smem_desc(sb + OFF_QL + a_off, 16, 1024), smem_desc(st + KV_B + b_off, 16, 1024), IDESC_S, ks > 0);
+            umma(ts + TM_SLOW, smem_desc(sb + OFF_QL + a_off, 16, 1024), smem_desc(st + KV_B + b_off, 16, 1024), IDESC_S, ks > 0);
+        }
+        umma_commit(bar_sfull + (j & 1) * 8);
+      };
+      bar_expect_tx(bar_q, Q_B * (shares ? 2 : 1));
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        tma_load_3d(sb + OFF_Q + c * (Q_B / 2), &tmQ, c * 64, hq, q0, bar_q);
+        if (shares) tma_load_3d(sb + OFF_QL + c * (Q_B / 2), &tmQl, c * 64, hq, q0, bar_q);
+      }
+      load_tile(0);
+      if (n_tiles > 1) load_tile(1);
+      fail = !bar_wait(bar_q, 0) || !bar_wait(bar_full, 0);
+      if (!fail) issue_qk(0);
+      for (int j = 0; j < n_tiles && !fail; ++j) {
+        const int b = j & 1, u = (j >> 1) & 1;
+        if (j + 1 < n_tiles) {                                  // the next tile's products overlap this tile's softmax
+          const int b1 = (j + 1) & 1, u1 = ((j + 1) >> 1) & 1;
+          fail = !bar_wait(bar_full + b1 * 8, u1);
+          if (!fail && j + 1 >= 2) fail = !bar_wait(bar_sempty + b1 * 8, u1 ^ 1);   // S[b1] of tile j - 1 has been read
+          if (fail) break;
+          issue_qk(j + 1);
+        }
+        fail = !bar_wait(bar_pfull + b * 8, u);                 // P[b] of tile j is written
+        if (fail) break;
+        tc_fence_after();
+        const uint32_t st = sb + OFF_ST + b * STAGE_B;
+#pragma unroll
+        for (int ks = 0; ks < BN / 16; ++ks)                    // 16 keys per step; O accumulates over the tiles
+          umma(tm + TM_O, smem_desc(sb + OFF_P + b * P_B + ks * 32, 16, 1024),
+               smem_desc(st + 2 * KV_B + ks * 2048, KV_B / 2, 1024), IDESC_O, (j > 0 || ks > 0) ? 1u : 0u);
+        umma_commit(bar_pvdone + b * 8);
+        if (j + 2 < n_tiles) {                                  // stage b is free once P V of tile j is done
+          fail = !bar_wait(bar_pvdone + b * 8, u);
+          if (fail) break;
+          load_tile(j + 2);
         }
       }
-      umma_commit(bar_s);                                       // arrives when the products above are done
-      if (!ok) fail = true;
+      if (fail) atomicExch(p.err_flag, 1);
     }
-    fail = fail || !bar_wait(bar_s, j & 1);
-    if (__syncthreads_or(fail)) { fail = true; break; }
-    tc_fence_after();
-
-    // ---- this thread's row: logits, mask, online softmax, P -----------------------------------------
-    const int k0 = j * BN;
-    auto logit = [&](float own, float low, int kj) -> float {
-      const bool valid = kj <= qi && kj < p.T;
-      const bool prox = kj < p.S || kj > qi - p.W;
-      const float a = (need_low && (!need_own || !prox)) ? low : own;
-      return valid ? a * p.scale_log2 : -INFINITY;
-    };
-    float mx = -INFINITY;
-#pragma unroll
-    for (int ch = 0; ch < BN / 32; ++ch) {
-      float so[32], sl[32];
-      if (need_own) tmem_ld32(tm + lane_base + ch * 32, so);
-      if (need_low) tmem_ld32(tm + TM_SLOW + lane_base + ch * 32, sl);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) mx = fmaxf(mx, logit(need_own ? so[i] : 0.f, need_low ? sl[i] : 0.f, k0 + ch * 32 + i));
-    }
-    const float m_new = fmaxf(m_row, mx);
-    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-    const float alpha = ex2f(m_row - m_use);                    // 0 on the first tile
-    m_row = m_new;
-    float psum = 0.f;
-    unsigned char* prow = smem + OFF_P + tid * 128;             // row tid of the [128][128 B] P tile
-#pragma unroll
-    for (int ch = 0; ch < BN / 32; ++ch) {
-      float so[32], sl[32];
-      if (need_own) tmem_ld32(tm + lane_base + ch * 32, so);
-      if (need_low) tmem_ld32(tm + TM_SLOW + lane_base + ch * 32, sl);
-      uint32_t pk[16];
-#pragma unroll
-      for (int i = 0; i < 32; i += 2) {
-        const float p0 = ex2f(logit(need_own ? so[i] : 0.f, need_low ? sl[i] : 0.f, k0 + ch * 32 + i) - m_use);
-        const float p1 = ex2f(logit(need_own ? so[i + 1] : 0.f, need_low ? sl[i + 1] : 0.f, k0 + ch * 32 + i + 1) - m_use);
-        psum += p0 + p1;
-        __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-        pk[i >> 1] = *reinterpret_cast<uint32_t*>(&b2);
-      }
-#pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) {                          // 16-byte chunk c of row r lives at chunk c ^ (r & 7)
-        const int chunk = ch * 4 + c4;
-        *reinterpret_cast<uint4*>(prow + ((chunk ^ (tid & 7)) << 4)) = make_uint4(pk[c4 * 4], pk[c4 * 4 + 1], pk[c4 * 4 + 2], pk[c4 * 4 + 3]);
-      }
-    }
-    l_row = l_row * alpha + psum;
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor cores
-    tc_fence_before();
-    __syncthreads();
-
-    // ---- O_tile = P V -----------------------------------------------------------------------------------
-    if (tid == 0) {
+  } else {
+    // ---- softmax warps: thread tid owns query row tid -------------------------------------------------
+    const int qi = q0 + tid;
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;     // this warp's quarter of the TMEM lanes
+    float m_used = -INFINITY, l_row = 0.f;
+    for (int j = 0; j < n_tiles && !fail; ++j) {
+      const int b = j & 1, u = (j >> 1) & 1;
+      bool need_own, need_low;
+      tile_needs(j, need_own, need_low);
+      fail = !bar_wait(bar_sfull + b * 8, u);
+      if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
       tc_fence_after();
+      const uint32_t ts = tm + b * TM_SBUF + lane_base;
+      const int k0 = j * BN;
+      // this row's 64 raw logits, read from TMEM once.  Interior tiles (every key visible to every row of
+      // the block, all proximal or all distant) need no per-key decision; tiles on the diagonal get the
+      // causal mask, tiles that straddle the window edge get the own / lowest-layer choice per key.
+      float a[BN];
 #pragma unroll
-      for (int ks = 0; ks < BN / 16; ++ks)                      // 16 keys per step
-        umma(tm + TM_O, smem_desc(sb + OFF_P + ks * 32, 16, 1024), smem_desc(st + 2 * KV_B + ks * 2048, KV_B / 2, 1024),
-             IDESC_O, ks > 0);
-      umma_commit(bar_o);
-    }
-    fail = !bar_wait(bar_o, j & 1);
-    if (__syncthreads_or(fail)) { fail = true; break; }
-    tc_fence_after();
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        float t[32];
+        tmem_ld32(ts + (need_own ? 0 : TM_SLOW) + ch * 32, t);
 #pragma unroll
-    for (int ch = 0; ch < PD / 32; ++ch) {
-      float t[32];
-      tmem_ld32(tm + TM_O + lane_base + ch * 32, t);
+        for (int i = 0; i < 32; ++i) a[ch * 32 + i] = t[i];
+        if (need_own && need_low) {
+          tmem_ld32(ts + TM_SLOW + ch * 32, t);
 #pragma unroll
-      for (int i = 0; i < 32; ++i) o[ch * 32 + i] = o[ch * 32 + i] * alpha + t[i];
-    }
-    tc_fence_before();
-    __syncthreads();                                            // stage s, P and the TMEM tiles are free again
-    if (tid == 0 && j + 2 < n_tiles) load_tile(j + 2);
-  }
-
-  if (fail) {
-    if (tid == 0) atomicExch(p.err_flag, 1);
-  } else if (qi < p.T) {
-    const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
-    uint16_t* dst = p.out + ((int64_t)qi * p.H_q + hq) * PD;
-#pragma unroll
-    for (int c = 0; c < PD; c += 8) {
-      uint32_t w[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        __nv_bfloat162 b2 = __floats2bfloat162_rn(o[c + 2 * i] * inv, o[c + 2 * i + 1] * inv);
-        w[i] = *reinterpret_cast<uint32_t*>(&b2);
+          for (int i = 0; i < 32; ++i) {
+            const int kj = k0 + ch * 32 + i;
+            const bool prox = kj < p.S || kj > qi - p.W;
+            a[ch * 32 + i] = prox ? a[ch * 32 + i] : t[i];
+          }
+        }
       }
-      *reinterpret_cast<uint4*>(dst + c) = make_uint4(w[0], w[1], w[2], w[3]);
+      if (k0 + BN - 1 > q0) {                                   // diagonal tile: keys after the row's position
+#pragma unroll
+        for (int i = 0; i < BN; ++i) a[i] = (k0 + i <= qi && k0 + i < p.T) ? a[i] : -INFINITY;
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < BN; ++i) mx = fmaxf(mx, a[i]);
+      mx *= p.scale_log2;                                       // the scale is positive: it commutes with the maximum
+      // raise the row's reference maximum only when the tile exceeds it by more than RESCALE_STEP
+      const bool raise = mx > m_used + RESCALE_STEP || (m_used == -INFINITY && mx > -INFINITY);
+      float alpha = 1.f;
+      if (raise) { alpha = ex2f(m_used - mx); m_used = mx; }    // ex2(-inf) = 0 on the first tile
+      if (__any_sync(0xffffffffu, raise) && j > 0) {            // rescale this warp's rows of O in TMEM
+        fail = !bar_wait(bar_pvdone + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);   // nothing is accumulating into O
+        if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int ch = 0; ch < PD / 32; ++ch) {
+          float t[32];
+          tmem_ld32(tm + TM_O + lane_base + ch * 32, t);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) t[i] *= alpha;
+          tmem_st32(tm + TM_O + lane_base + ch * 32, t);
+        }
+        tc_fence_before();
+      }
+      l_row *= alpha;
+      if (j >= 2) {                                             // P[b] was read by P V of tile j - 2
+        fail = !bar_wait(bar_pvdone + b * 8, u ^ 1);
+        if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
+      }
+      const float m_use = (m_used == -INFINITY) ? 0.f : m_used;
+      float psum = 0.f;
+      unsigned char* prow = smem + OFF_P + b * P_B + tid * 128;  // row tid of the [128][128 B] P tile
+#pragma unroll
+      for (int c8 = 0; c8 < BN / 8; ++c8) {                     // eight keys = one 16-byte chunk of the row
+        uint32_t pk[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float p0 = ex2f(fmaf(a[c8 * 8 + 2 * i], p.scale_log2, -m_use));
+          const float p1 = ex2f(fmaf(a[c8 * 8 + 2 * i + 1], p.scale_log2, -m_use));
+          psum += p0 + p1;
+          __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+          pk[i] = *reinterpret_cast<uint32_t*>(&b2);
+        }
+        // 16-byte chunk c of row r lives at chunk c ^ (r & 7)
+        *reinterpret_cast<uint4*>(prow + ((c8 ^ (tid & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+      l_row += psum;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor cores
+      tc_fence_before();
+      bar_arrive(bar_pfull + b * 8);
+      bar_arrive(bar_sempty + b * 8);
+    }
+    if (!fail) {
+      fail = !bar_wait(bar_pvdone + ((n_tiles - 1) & 1) * 8, ((n_tiles - 1) >> 1) & 1);
+      fail = __any_sync(0xffffffffu, fail);
+    }
+    if (fail) {
+      if ((tid & 31) == 0) atomicExch(p.err_flag, 1);
+    } else {
+      tc_fence_after();
+      const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+      uint16_t* dst = p.out + ((int64_t)qi * p.H_q + hq) * PD;
+#pragma unroll
+      for (int ch = 0; ch < PD / 32; ++ch) {
+        float t[32];
+        tmem_ld32(tm + TM_O + lane_base + ch * 32, t);          // warp-collective: rows past T load too
+        if (qi < p.T) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              __nv_bfloat162 b2 = __floats2bfloat162_rn(t[c + 2 * i] * inv, t[c + 2 * i + 1] * inv);
+              w[i] = *reinterpret_cast<uint32_t*>(&b2);
+            }
+            *reinterpret_cast<uint4*>(dst + ch * 32 + c) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
     }
   }
-  // return the tensor memory; after a failed wait first give outstanding work a bounded chance to land
+  // return the tensor memory
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
-    if (fail && tid == 0) { bar_wait(bar_full, 0); bar_wait(bar_full + 8, 0); }
-    __syncwarp();
+  if (producer) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(TM_COLS) : "memory");
   }
@@ -397,7 +462,7 @@ extern "C" int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int
       !encode_3d(su->encode, &tkl, kl, n_tokens, n_kv_heads, BN))
     return POD_ERR_INVALID;
   dim3 grid((n_tokens + BM - 1) / BM, n_q_heads);
-  pod_prefill_kernel<<<grid, BM, PF_SMEM, static_cast<cudaStream_t>(cuda_stream)>>>(tq, tk, tv, tql, tkl, p);
+  pod_prefill_kernel<<<grid, PF_THREADS, PF_SMEM, static_cast<cudaStream_t>(cuda_stream)>>>(tq, tk, tv, tql, tkl, p);
   return cudaGetLastError() == cudaSuccess ? POD_OK : POD_ERR_CUDA;
 }
 
