@@ -9,18 +9,20 @@
 //
 // One CTA = 128 consecutive query positions of one query head: four softmax warps (thread t owns query
 // row t) and one producer warp whose lane 0 issues every TMA load and every tcgen05.mma.  Key/value tiles
-// of 64 positions stream through a two-stage shared-memory ring (TMA, 128-byte swizzle).  Per tile j:
-//   S_own[128 x 64] = Q K^T and, where the tile holds distant tokens of a sharing head,
-//   S_low[128 x 64] = Q_a K_a^T               (M = 128, N = 64, K = 16 x 8 steps, into one of two TMEM buffers:
-//                                              the products of tile j + 1 run while tile j is in the softmax)
-//   each softmax thread reads its row of S from TMEM (tcgen05.ld), picks own/low per key, masks, and
+// of 64 positions stream through a shared-memory ring of three or four stages (TMA, 128-byte swizzle).
+// A tile whose keys are all proximal for every row of the block (or whose head does not share) is scored
+// with Q K^T, one whose keys are all distant with Q_a K_a^T; the few tiles that straddle the edge of the
+// window or of the sink are taken twice, once with each product and the other kind of key masked (the
+// softmax does not care in how many pieces the keys arrive).  Per pass v:
+//   S[128 x 64] = Q K^T  or  Q_a K_a^T       (M = 128, N = 64, K = 16 x 8 steps, into one of two TMEM buffers:
+//                                              the product of pass v + 1 runs while pass v is in the softmax)
+//   each softmax thread reads its row of S from TMEM (tcgen05.ld), masks, and
 //   writes its row of P = 2^(logit - m) as bf16 into one of two swizzled shared-memory tiles
 //   O[128 x 128] += P V                       (A = P K-major, B = V MN-major, K = 16 x 4), accumulated in TMEM.
 // The reference maximum m of a row is only raised when the tile's maximum exceeds it by more than 8 (in
 // log2 units): P then stays below 2^8, and the rows of O in TMEM have to be rescaled (tcgen05.ld / st)
 // only on those rare occasions instead of after every tile; row sum and O share the same m, so the
-// quotient is exact either way.  Tiles that are entirely proximal (or entirely distant) skip the product
-// they do not need.  Warps hand buffers to one another through mbarriers; every wait is bounded, a wait
+// quotient is exact either way.  Warps hand buffers to one another through mbarriers; every wait is bounded, a wait
 // that gives up raises the error flag, and the tensor memory is always returned before the CTA exits.
 #include <cudaTypedefs.h>
 #include <cuda_bf16.h>
@@ -37,19 +39,20 @@ namespace {
 constexpr int PD = 128;                 // head_dim
 constexpr int BM = 128;                 // query rows per CTA
 constexpr int BN = 64;                  // keys per tile
-constexpr int NSTG = 2;
+constexpr int MAX_STG = 4;              // stages of the K/V ring: 4, or 3 when the lowest layer's Q is resident too
 constexpr uint32_t PF_WAIT_LIMIT = 1u << 22;
 
 constexpr int Q_B = BM * PD * 2;        // 32 KiB: two [128][128 B] sub-tiles
 constexpr int KV_B = BN * PD * 2;       // 16 KiB: two [64][128 B] sub-tiles
-constexpr int STAGE_B = 3 * KV_B;       // K, K of the lowest layer, V
+constexpr int STAGE_B = 2 * KV_B;       // K (of this layer or of the lowest layer), V
 constexpr int P_B = BM * BN * 2;        // 16 KiB: one [128][128 B] tile
-constexpr int OFF_Q = 0, OFF_QL = Q_B, OFF_ST = 2 * Q_B, OFF_P = OFF_ST + NSTG * STAGE_B;
+constexpr int OFF_Q = 0, OFF_QL = Q_B;  // stages start after Q, or after Q and Q of the lowest layer
+constexpr int OFF_P = Q_B + MAX_STG * STAGE_B;
 constexpr int OFF_BAR = OFF_P + 2 * P_B;
 constexpr int PF_SMEM = OFF_BAR + 256 + 1024;
 constexpr int PF_THREADS = BM + 32;     // four softmax warps + the producer warp
-constexpr int TM_COLS = 512;            // 2 x (S_own 64 + S_low 64) + O 128 fp32 columns, next power of two
-constexpr int TM_SBUF = 128, TM_SLOW = 64, TM_O = 256;
+constexpr int TM_COLS = 256;            // 2 x S 64 + O 128 fp32 columns
+constexpr int TM_SBUF = 64, TM_O = 128;
 constexpr float RESCALE_STEP = 8.f;     // raise a row's reference maximum only past this many log2 units
 
 struct PrefillParams {
@@ -163,14 +166,16 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const int q0 = qb * BM;
   const bool shares = kvh < 256 && ((p.share_mask[kvh >> 5] >> (kvh & 31)) & 1u);
   // mbarriers: Q landed; per stage: K/V landed; per buffer: S ready, S read, P written, P V done
-  const uint32_t bar_q = sb + OFF_BAR, bar_full = bar_q + 8, bar_sfull = bar_q + 24, bar_sempty = bar_q + 40,
-                 bar_pfull = bar_q + 56, bar_pvdone = bar_q + 72;
+  const uint32_t bar_q = sb + OFF_BAR, bar_full = bar_q + 8, bar_sfull = bar_q + 40, bar_sempty = bar_q + 56,
+                 bar_pfull = bar_q + 72, bar_pvdone = bar_q + 88;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 128);
+  const int nstg = shares ? MAX_STG - 1 : MAX_STG;
+  const uint32_t st0 = sb + (shares ? 2 * Q_B : Q_B);           // first stage of the ring
 
   if (tid == 0) {
     bar_init(bar_q, 1);
+    for (int i = 0; i < MAX_STG; ++i) bar_init(bar_full + i * 8, 1);
     for (int i = 0; i < 2; ++i) {
-      bar_init(bar_full + i * 8, 1);
       bar_init(bar_sfull + i * 8, 1);
       bar_init(bar_sempty + i * 8, BM);
       bar_init(bar_pfull + i * 8, BM);
@@ -191,47 +196,55 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   // keys this block needs: positions [0, min(T, q0 + 128)); tile j covers [64 j, 64 j + 64)
   const int k_end = min(p.T, q0 + BM);
   const int n_tiles = (k_end + BN - 1) / BN;
-  // a tile is entirely proximal for every row of the block if it starts after qmax - W (or lies in the
-  // sink), entirely distant if it lies in [S, qmin - W]
-  auto tile_needs = [&](int j, bool& need_own, bool& need_low) {
+  // kind of tile j for this block: 0 = scored with this layer's q, k (all keys proximal for every row, or
+  // the head does not share); 1 = with the lowest layer's (all keys distant for every row); 2 = both kinds
+  // of key: two passes
+  auto tile_kind = [&](int j) -> int {
+    if (!shares) return 0;
     const int k0 = j * BN, k1 = k0 + BN - 1;
-    const bool prox_all = (k1 < p.S) || (k0 > q0 + BM - 1 - p.W);
-    const bool dist_all = (k0 >= p.S) && (k1 <= q0 - p.W);
-    need_low = shares && !prox_all;
-    need_own = !shares || !dist_all;
+    if ((k1 < p.S) || (k0 > q0 + BM - 1 - p.W)) return 0;
+    if ((k0 >= p.S) && (k1 <= q0 - p.W)) return 1;
+    return 2;
+  };
+  // the passes in order: (tile, 0 = own product / 1 = lowest layer's product)
+  struct Pass { int j, low, mixed; };
+  auto first_pass = [&]() -> Pass { const int k = tile_kind(0); return Pass{0, k == 1, k == 2}; };
+  auto next_pass = [&](Pass c) -> Pass {
+    if (c.mixed && !c.low) return Pass{c.j, 1, 1};
+    const int k = c.j + 1 < n_tiles ? tile_kind(c.j + 1) : 0;
+    return Pass{c.j + 1, k == 1, k == 2};
   };
   bool fail = false;
 
   if (producer) {
     if ((tid & 31) == 0) {
       constexpr uint32_t IDESC_S = instr_desc(BN, false), IDESC_O = instr_desc(PD, true);
-      auto load_tile = [&](int j) {
-        const int s = j & 1;
-        bool need_own, need_low;
-        tile_needs(j, need_own, need_low);
-        const uint32_t st = sb + OFF_ST + s * STAGE_B, bar = bar_full + s * 8;
-        bar_expect_tx(bar, KV_B * (1 + (need_own ? 1 : 0) + (need_low ? 1 : 0)));
+      Pass cl = first_pass();                                   // next pass to load
+      int vl = 0;
+      auto load_next = [&]() {
+        if (cl.j >= n_tiles) return;
+        const uint32_t st = st0 + (vl % nstg) * STAGE_B, bar = bar_full + (vl % nstg) * 8;
+        bar_expect_tx(bar, STAGE_B);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-          if (need_own) tma_load_3d(st + c * (KV_B / 2), &tmK, c * 64, kvh, j * BN, bar);
-          if (need_low) tma_load_3d(st + KV_B + c * (KV_B / 2), &tmKl, c * 64, kvh, j * BN, bar);
-          tma_load_3d(st + 2 * KV_B + c * (KV_B / 2), &tmV, c * 64, kvh, j * BN, bar);
+          tma_load_3d(st + c * (KV_B / 2), cl.low ? &tmKl : &tmK, c * 64, kvh, cl.j * BN, bar);
+          tma_load_3d(st + KV_B + c * (KV_B / 2), &tmV, c * 64, kvh, cl.j * BN, bar);
         }
+        cl = next_pass(cl);
+        ++vl;
       };
-      auto issue_qk = [&](int j) {                              // S[j & 1] = Q K_j^T (own and/or lowest layer's)
-        bool need_own, need_low;
-        tile_needs(j, need_own, need_low);
-        const uint32_t st = sb + OFF_ST + (j & 1) * STAGE_B, ts = tm + (j & 1) * TM_SBUF;
+      Pass cq = first_pass();                                   // next pass whose product is issued
+      auto issue_qk = [&](int v) {                              // S[v & 1] = Q K^T of pass v
+        const uint32_t st = st0 + (v % nstg) * STAGE_B, ts = tm + (v & 1) * TM_SBUF;
+        const uint32_t qa = sb + (cq.low ? OFF_QL : OFF_Q);
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < PD / 16; ++ks) {                  // 16 channels per step: 4 per 128-byte sub-tile
           const uint32_t a_off = (ks >> 2) * (Q_B / 2) + (ks & 3) * 32, b_off = (ks >> 2) * (KV_B / 2) + (ks & 3) * 32;
-          if (need_own)
-            umma(ts, smem_desc(sb + OFF_Q + a_off, 16, 1024), smem_desc(st + b_off, 16, 1024), IDESC_S, ks > 0);
-          if (need_low)
-            umma(ts + TM_SLOW, smem_desc(sb + OFF_QL + a_off, 16, 1024), smem_desc(st + KV_B + b_off, 16, 1024), IDESC_S, ks > 0);
+          umma(ts, smem_desc(qa + a_off, 16, 1024), smem_desc(st + b_off, 16, 1024), IDESC_S, ks > 0);
         }
-        umma_commit(bar_sfull + (j & 1) * 8);
+        umma_commit(bar_sfull + (v & 1) * 8);
+        cq = next_pass(cq);
       };
       bar_expect_tx(bar_q, Q_B * (shares ? 2 : 1));
 #pragma unroll
@@ -239,33 +252,33 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         tma_load_3d(sb + OFF_Q + c * (Q_B / 2), &tmQ, c * 64, hq, q0, bar_q);
         if (shares) tma_load_3d(sb + OFF_QL + c * (Q_B / 2), &tmQl, c * 64, hq, q0, bar_q);
       }
-      load_tile(0);
-      if (n_tiles > 1) load_tile(1);
+      for (int i = 0; i < nstg; ++i) load_next();
       fail = !bar_wait(bar_q, 0) || !bar_wait(bar_full, 0);
       if (!fail) issue_qk(0);
-      for (int j = 0; j < n_tiles && !fail; ++j) {
-        const int b = j & 1, u = (j >> 1) & 1;
-        if (j + 1 < n_tiles) {                                  // the next tile's products overlap this tile's softmax
-          const int b1 = (j + 1) & 1, u1 = ((j + 1) >> 1) & 1;
-          fail = !bar_wait(bar_full + b1 * 8, u1);
-          if (!fail && j + 1 >= 2) fail = !bar_wait(bar_sempty + b1 * 8, u1 ^ 1);   // S[b1] of tile j - 1 has been read
+      for (int v = 0; cq.j < n_tiles || v < vl; ++v) {          // v runs over all passes (vl ends as their number)
+        if (v >= vl) break;
+        const int b = v & 1, u = (v >> 1) & 1;
+        if (cq.j < n_tiles) {                                   // the next pass's product overlaps this pass's softmax
+          const int v1 = v + 1;
+          fail = !bar_wait(bar_full + (v1 % nstg) * 8, (v1 / nstg) & 1);
+          if (!fail && v1 >= 2) fail = !bar_wait(bar_sempty + (v1 & 1) * 8, ((v1 >> 1) & 1) ^ 1);   // S[v1 & 1] of pass v - 1 has been read
           if (fail) break;
-          issue_qk(j + 1);
+          issue_qk(v1);
         }
-        fail = !bar_wait(bar_pfull + b * 8, u);                 // P[b] of tile j is written
+        if (v >= 1 && cl.j < n_tiles) {                         // the stage of pass v - 1 is free once its P V is done
+          fail = !bar_wait(bar_pvdone + ((v - 1) & 1) * 8, ((v - 1) >> 1) & 1);
+          if (fail) break;
+          load_next();
+        }
+        fail = !bar_wait(bar_pfull + b * 8, u);                 // P[b] of pass v is written
         if (fail) break;
         tc_fence_after();
-        const uint32_t st = sb + OFF_ST + b * STAGE_B;
+        const uint32_t st = st0 + (v % nstg) * STAGE_B;
 #pragma unroll
-        for (int ks = 0; ks < BN / 16; ++ks)                    // 16 keys per step; O accumulates over the tiles
+        for (int ks = 0; ks < BN / 16; ++ks)                    // 16 keys per step; O accumulates over the passes
           umma(tm + TM_O, smem_desc(sb + OFF_P + b * P_B + ks * 32, 16, 1024),
-               smem_desc(st + 2 * KV_B + ks * 2048, KV_B / 2, 1024), IDESC_O, (j > 0 || ks > 0) ? 1u : 0u);
+               smem_desc(st + KV_B + ks * 2048, KV_B / 2, 1024), IDESC_O, (v > 0 || ks > 0) ? 1u : 0u);
         umma_commit(bar_pvdone + b * 8);
-        if (j + 2 < n_tiles) {                                  // stage b is free once P V of tile j is done
-          fail = !bar_wait(bar_pvdone + b * 8, u);
-          if (fail) break;
-          load_tile(j + 2);
-        }
       }
       if (fail) atomicExch(p.err_flag, 1);
     }
@@ -274,38 +287,36 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int qi = q0 + tid;
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;     // this warp's quarter of the TMEM lanes
     float m_used = -INFINITY, l_row = 0.f;
-    for (int j = 0; j < n_tiles && !fail; ++j) {
-      const int b = j & 1, u = (j >> 1) & 1;
-      bool need_own, need_low;
-      tile_needs(j, need_own, need_low);
+    int v = 0;
+    for (Pass c = first_pass(); c.j < n_tiles && !fail; c = next_pass(c), ++v) {
+      const int b = v & 1, u = (v >> 1) & 1;
       fail = !bar_wait(bar_sfull + b * 8, u);
       if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
       tc_fence_after();
       const uint32_t ts = tm + b * TM_SBUF + lane_base;
-      const int k0 = j * BN;
+      const int k0 = c.j * BN;
       // this row's 64 raw logits, read from TMEM once.  Interior tiles (every key visible to every row of
-      // the block, all proximal or all distant) need no per-key decision; tiles on the diagonal get the
-      // causal mask, tiles that straddle the window edge get the own / lowest-layer choice per key.
+      // the block) need no per-key decision; tiles on the diagonal get the causal mask, and a pass over a
+      // tile with both kinds of key keeps the kind its product is meant for.
       float a[BN];
 #pragma unroll
       for (int ch = 0; ch < BN / 32; ++ch) {
         float t[32];
-        tmem_ld32(ts + (need_own ? 0 : TM_SLOW) + ch * 32, t);
+        tmem_ld32(ts + ch * 32, t);
 #pragma unroll
         for (int i = 0; i < 32; ++i) a[ch * 32 + i] = t[i];
-        if (need_own && need_low) {
-          tmem_ld32(ts + TM_SLOW + ch * 32, t);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int kj = k0 + ch * 32 + i;
-            const bool prox = kj < p.S || kj > qi - p.W;
-            a[ch * 32 + i] = prox ? a[ch * 32 + i] : t[i];
-          }
-        }
       }
       if (k0 + BN - 1 > q0) {                                   // diagonal tile: keys after the row's position
 #pragma unroll
         for (int i = 0; i < BN; ++i) a[i] = (k0 + i <= qi && k0 + i < p.T) ? a[i] : -INFINITY;
+      }
+      if (c.mixed) {
+#pragma unroll
+        for (int i = 0; i < BN; ++i) {
+          const int kj = k0 + i;
+          const bool prox = kj < p.S || kj > qi - p.W;
+          a[i] = (prox != (c.low != 0)) ? a[i] : -INFINITY;     // own product: proximal keys; lowest layer's: distant keys
+        }
       }
       float mx = -INFINITY;
 #pragma unroll
@@ -315,8 +326,8 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const bool raise = mx > m_used + RESCALE_STEP || (m_used == -INFINITY && mx > -INFINITY);
       float alpha = 1.f;
       if (raise) { alpha = ex2f(m_used - mx); m_used = mx; }    // ex2(-inf) = 0 on the first tile
-      if (__any_sync(0xffffffffu, raise) && j > 0) {            // rescale this warp's rows of O in TMEM
-        fail = !bar_wait(bar_pvdone + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);   // nothing is accumulating into O
+      if (__any_sync(0xffffffffu, raise) && v > 0) {            // rescale this warp's rows of O in TMEM
+        fail = !bar_wait(bar_pvdone + ((v - 1) & 1) * 8, ((v - 1) >> 1) & 1);   // nothing is accumulating into O
         if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
         tc_fence_after();
 #pragma unroll
@@ -330,7 +341,7 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         tc_fence_before();
       }
       l_row *= alpha;
-      if (j >= 2) {                                             // P[b] was read by P V of tile j - 2
+      if (v >= 2) {                                             // P[b] was read by P V of pass v - 2
         fail = !bar_wait(bar_pvdone + b * 8, u ^ 1);
         if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
       }
@@ -358,7 +369,7 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       bar_arrive(bar_sempty + b * 8);
     }
     if (!fail) {
-      fail = !bar_wait(bar_pvdone + ((n_tiles - 1) & 1) * 8, ((n_tiles - 1) >> 1) & 1);
+      fail = !bar_wait(bar_pvdone + ((v - 1) & 1) * 8, ((v - 1) >> 1) & 1);
       fail = __any_sync(0xffffffffu, fail);
     }
     if (fail) {
