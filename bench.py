@@ -54,6 +54,14 @@ def _peaks():
     return 6650.0, "fallback"
 
 
+def _bf16_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f).get("bf16_tflops", 1590.0))
+    return 1590.0
+
+
 def _profile_traffic(workload):
     """DRAM bytes per launch of the split-K kernel from the committed ncu summary, or None."""
     path = os.path.join(ROOT, "profiles", f"pod_decode_splitk_{workload}.md")
@@ -226,6 +234,42 @@ def run_ours(args):
         out["note"] = "bytes read + written per call over the mean of back-to-back calls"
         return out
 
+    def time_prefill_attn(reps=3):
+        """pod_prefill_attn over one sequence's whole context for one layer: once as the lowest layer of
+        its block (plain causal attention) and once as a layer whose heads all take their distant logits
+        from the lowest layer.  FLOPs counted: the causal half of the two products, 4 d per (query, key)
+        pair and head; masked pairs inside a tile and the second pass over edge tiles are not counted."""
+        T_ = min(n, args.prefill_tokens)
+        gen = lambda tag, layer, h: synth.gen_kv(seed, tag, layer, 0, 0, T_, h, d, outliers=w["outliers"] and tag != synth.TAG_Q, device=dev)
+        q, k, v = gen(synth.TAG_Q, 1, Hq), gen(synth.TAG_K, 1, Hkv), gen(synth.TAG_V, 1, Hkv)
+        ql, kl = gen(synth.TAG_Q, 0, Hq), gen(synth.TAG_K, 0, Hkv)
+        o = torch.empty(T_, Hq, d, device=dev, dtype=torch.bfloat16)
+        flops = 4.0 * d * Hq * (T_ * (T_ + 1) / 2)
+        out = {}
+        for name, share in (("lowest_layer", False), ("sharing_layer", True)):
+            f = lambda: B.pod_prefill_attn(q, k, v, o, n_sink=S, n_recent=W, q_low=ql if share else None,
+                                           k_low=kl if share else None, stream=stream)
+            f()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                f()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+            out[name] = {"ms": round(ms, 3), "tflops": round(flops / ms / 1e9, 1)}
+        assert B.pod_prefill_status() == 0
+        out["tokens"] = T_
+        out["peak_tflops"] = _bf16_peak()
+        out["note"] = "causal FLOPs (2 products x 2 d per visible pair) over the mean of back-to-back calls; peak = measured cuBLAS bf16 burst"
+        return out
+
+    if args.only == "prefill-attn":
+        if rank == 0:
+            print(json.dumps({"prefill_attn": time_prefill_attn()}), flush=True)
+        return
+
     def build_cache(group, use_map=False):
         cfg = B.make_config(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, group_size=group,
                             n_sink=S, n_recent=W, batch=Bn, device=local)
@@ -367,6 +411,7 @@ def run_ours(args):
     torch.cuda.empty_cache()
 
     prefill = time_prefill_write() if rank == 0 else None
+    prefill_attn = time_prefill_attn() if rank == 0 and d == 128 else None
     # ---- dense-KV baseline: the same kernels with every layer its own block (G = 1) ---------------
     dense_us = None
     if world == 1 and not args.no_dense:
@@ -425,6 +470,7 @@ def run_ours(args):
         "clocks": clocks,
         "cache_bytes": {"pod_live": live, "dense_equiv": dense_equiv, "saving": round(1 - live / dense_equiv, 5)},
         "prefill_write": prefill,
+        "prefill_attn": prefill_attn,
         "two_call_us_per_layer_step": round(ms_two * 1e3 / (args.steps * L * world), 3),
         "dense_kv_baseline_us_per_layer_step": None if dense_us is None else round(dense_us, 3),
     }
@@ -525,6 +571,10 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--gate-tau", type=float, default=None,
                     help="gate threshold of the distant-skip approximation (default: off, exact attention)")
+    ap.add_argument("--prefill-tokens", type=int, default=32768,
+                    help="positions of the prefill-attention leg (capped at the workload's context)")
+    ap.add_argument("--only", default=None, choices=["prefill-attn"],
+                    help="run one side leg alone and print its object (for profiling)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

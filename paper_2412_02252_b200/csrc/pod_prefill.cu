@@ -7,13 +7,19 @@
 // the lowest layer of the head's block (for a head whose block starts at this layer both are the
 // same product).  One softmax over both groups weighs layer l's own values.
 //
-// One CTA = 128 consecutive query positions of one query head: four softmax warps (thread t owns query
-// row t) and one producer warp whose lane 0 issues every TMA load and every tcgen05.mma.  Key/value tiles
-// of 64 positions stream through a shared-memory ring of three or four stages (TMA, 128-byte swizzle).
-// A tile whose keys are all proximal for every row of the block (or whose head does not share) is scored
-// with Q K^T, one whose keys are all distant with Q_a K_a^T; the few tiles that straddle the edge of the
+// One CTA = 256 consecutive query positions of one query head: two softmax groups of four warps (group g
+// owns rows 128 g .. 128 g + 127, one thread per row) and one producer warp whose lane 0 issues every TMA
+// load and every tcgen05.mma.  Both groups work on the same key/value tile at the same time, so each tile
+// is fetched once per 256 rows and the tensor cores always have the other group's products to run while
+// one group is in its softmax.  Keys and values of 64 positions stream through two rings of three
+// 16 KiB slots (TMA, 128-byte swizzle); a key slot is refilled as soon as its products are done, a value
+// slot after the P V products.
+// A tile whose keys are all distant for every row of the CTA is scored with Q_a K_a^T, one whose keys are
+// all proximal (or whose head does not share) with Q K^T; the few tiles that straddle the edge of the
 // window or of the sink are taken twice, once with each product and the other kind of key masked (the
-// softmax does not care in how many pieces the keys arrive).  Per pass v:
+// softmax does not care in how many pieces, or in which order, the keys arrive).  The passes that use the
+// lowest layer's product run first, with Q_a in the query buffers; then Q of this layer is loaded over it
+// and the other passes follow.  Per pass v and group g:
 //   S[128 x 64] = Q K^T  or  Q_a K_a^T       (M = 128, N = 64, K = 16 x 8 steps, into one of two TMEM buffers:
 //                                              the product of pass v + 1 runs while pass v is in the softmax)
 //   each softmax thread reads its row of S from TMEM (tcgen05.ld), masks, and
@@ -22,8 +28,9 @@
 // The reference maximum m of a row is only raised when the tile's maximum exceeds it by more than 8 (in
 // log2 units): P then stays below 2^8, and the rows of O in TMEM have to be rescaled (tcgen05.ld / st)
 // only on those rare occasions instead of after every tile; row sum and O share the same m, so the
-// quotient is exact either way.  Warps hand buffers to one another through mbarriers; every wait is bounded, a wait
-// that gives up raises the error flag, and the tensor memory is always returned before the CTA exits.
+// quotient is exact either way.  Warps hand buffers to one another through mbarriers; every wait is bounded
+// (a wait gives up only after seconds, long after every copy in flight has landed), a wait that gives up
+// raises the error flag, and the tensor memory is always returned before the CTA exits.
 #include <cudaTypedefs.h>
 #include <cuda_bf16.h>
 #include <math.h>
@@ -37,22 +44,24 @@ namespace pod {
 namespace {
 
 constexpr int PD = 128;                 // head_dim
-constexpr int BM = 128;                 // query rows per CTA
+constexpr int BM = 128;                 // query rows per softmax group
+constexpr int NG = 2;                   // softmax groups per CTA
+constexpr int BLK = NG * BM;            // query rows per CTA
 constexpr int BN = 64;                  // keys per tile
-constexpr int MAX_STG = 4;              // stages of the K/V ring: 4, or 3 when the lowest layer's Q is resident too
+constexpr int NRING = 3;                // slots of the key ring and of the value ring
 constexpr uint32_t PF_WAIT_LIMIT = 1u << 22;
 
 constexpr int Q_B = BM * PD * 2;        // 32 KiB: two [128][128 B] sub-tiles
 constexpr int KV_B = BN * PD * 2;       // 16 KiB: two [64][128 B] sub-tiles
-constexpr int STAGE_B = 2 * KV_B;       // K (of this layer or of the lowest layer), V
 constexpr int P_B = BM * BN * 2;        // 16 KiB: one [128][128 B] tile
-constexpr int OFF_Q = 0, OFF_QL = Q_B;  // stages start after Q, or after Q and Q of the lowest layer
-constexpr int OFF_P = Q_B + MAX_STG * STAGE_B;
-constexpr int OFF_BAR = OFF_P + 2 * P_B;
+constexpr int OFF_Q = 0;                // per group: Q of the lowest layer, later Q of this layer
+constexpr int OFF_K = NG * Q_B, OFF_V = OFF_K + NRING * KV_B;
+constexpr int OFF_P = OFF_V + NRING * KV_B;      // per group two P tiles
+constexpr int OFF_BAR = OFF_P + NG * 2 * P_B;
 constexpr int PF_SMEM = OFF_BAR + 256 + 1024;
-constexpr int PF_THREADS = BM + 32;     // four softmax warps + the producer warp
-constexpr int TM_COLS = 256;            // 2 x S 64 + O 128 fp32 columns
-constexpr int TM_SBUF = 64, TM_O = 128;
+constexpr int PF_THREADS = BLK + 32;    // eight softmax warps + the producer warp
+constexpr int TM_COLS = 512;            // per group 2 x S 64 + O 128 fp32 columns
+constexpr int TM_GROUP = 256, TM_SBUF = 64, TM_O = 128;
 constexpr float RESCALE_STEP = 8.f;     // raise a row's reference maximum only past this many log2 units
 
 struct PrefillParams {
@@ -111,7 +120,7 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// this thread's 32 consecutive fp32 columns of its TMEM lane
+// this thread's 32 consecutive fp32 columns of its TMEM lane (valid after tmem_ld_wait)
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   uint32_t r[32];
   asm volatile(
@@ -123,10 +132,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// the values of earlier tmem_ld32 calls may be used after this
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -160,24 +170,24 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pf_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sb = s2u(smem);
   const int tid = threadIdx.x, warp = tid >> 5;
-  const bool producer = warp == BM / 32;
+  const bool producer = warp == BLK / 32;
   const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;          // long rows first
   const int hq = blockIdx.y, kvh = hq / (p.H_q / p.H_kv);
-  const int q0 = qb * BM;
+  const int q0 = qb * BLK;
   const bool shares = kvh < 256 && ((p.share_mask[kvh >> 5] >> (kvh & 31)) & 1u);
-  // mbarriers: Q landed; per stage: K/V landed; per buffer: S ready, S read, P written, P V done
-  const uint32_t bar_q = sb + OFF_BAR, bar_full = bar_q + 8, bar_sfull = bar_q + 40, bar_sempty = bar_q + 56,
-                 bar_pfull = bar_q + 72, bar_pvdone = bar_q + 88;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 128);
-  const int nstg = shares ? MAX_STG - 1 : MAX_STG;
-  const uint32_t st0 = sb + (shares ? 2 * Q_B : Q_B);           // first stage of the ring
+  // mbarriers: Q landed; per ring slot: K landed, V landed; per group and buffer: S ready, P written, P V done
+  const uint32_t bar_q = sb + OFF_BAR, bar_kfull = bar_q + 8, bar_vfull = bar_q + 32, bar_sfull = bar_q + 56,
+                 bar_pfull = bar_q + 88, bar_pvdone = bar_q + 120;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 192);
 
   if (tid == 0) {
     bar_init(bar_q, 1);
-    for (int i = 0; i < MAX_STG; ++i) bar_init(bar_full + i * 8, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < NRING; ++i) {
+      bar_init(bar_kfull + i * 8, 1);
+      bar_init(bar_vfull + i * 8, 1);
+    }
+    for (int i = 0; i < NG * 2; ++i) {
       bar_init(bar_sfull + i * 8, 1);
-      bar_init(bar_sempty + i * 8, BM);
       bar_init(bar_pfull + i * 8, BM);
       bar_init(bar_pvdone + i * 8, 1);
     }
@@ -193,120 +203,150 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   tc_fence_after();
   const uint32_t tm = *tmem_slot;
 
-  // keys this block needs: positions [0, min(T, q0 + 128)); tile j covers [64 j, 64 j + 64)
-  const int k_end = min(p.T, q0 + BM);
+  // keys this CTA needs: positions [0, min(T, q0 + 256)); tile j covers [64 j, 64 j + 64)
+  const int k_end = min(p.T, q0 + BLK);
   const int n_tiles = (k_end + BN - 1) / BN;
-  // kind of tile j for this block: 0 = scored with this layer's q, k (all keys proximal for every row, or
-  // the head does not share); 1 = with the lowest layer's (all keys distant for every row); 2 = both kinds
-  // of key: two passes
-  auto tile_kind = [&](int j) -> int {
-    if (!shares) return 0;
-    const int k0 = j * BN, k1 = k0 + BN - 1;
-    if ((k1 < p.S) || (k0 > q0 + BM - 1 - p.W)) return 0;
-    if ((k0 >= p.S) && (k1 <= q0 - p.W)) return 1;
-    return 2;
-  };
-  // the passes in order: (tile, 0 = own product / 1 = lowest layer's product)
-  struct Pass { int j, low, mixed; };
-  auto first_pass = [&]() -> Pass { const int k = tile_kind(0); return Pass{0, k == 1, k == 2}; };
-  auto next_pass = [&](Pass c) -> Pass {
-    if (c.mixed && !c.low) return Pass{c.j, 1, 1};
-    const int k = c.j + 1 < n_tiles ? tile_kind(c.j + 1) : 0;
-    return Pass{c.j + 1, k == 1, k == 2};
+  // Tiles [low_a, low_b) hold a key that is distant for some row of the CTA: they get a pass with the lowest
+  // layer's product.  Of those, tiles [dis_a, dis_b) are distant for every row and get no other pass.
+  int low_a = 0, low_b = 0, dis_a = 0, dis_b = 0;
+  if (shares) {
+    low_a = p.S >> 6;                                           // tiles before it lie inside the sink
+    const int e = q0 + BLK - 1 - p.W;                           // the last row's newest distant position
+    low_b = max(low_a, min(e < 0 ? 0 : (e >> 6) + 1, n_tiles));
+    dis_a = (p.S + BN - 1) >> 6;
+    const int f = q0 - p.W - (BN - 1);                          // tile j is distant for the first row too if 64 j <= f
+    dis_b = max(dis_a, min(f < 0 ? 0 : (f >> 6) + 1, low_b));
+  }
+  const int n_low = low_b - low_a, n_skip = dis_b - dis_a;
+  const int n_pass = n_low + n_tiles - n_skip;
+  struct Pass { int j; bool low, mixed; };
+  auto pass_of = [&](int v) -> Pass {
+    if (v < n_low) {
+      const int j = low_a + v;
+      return Pass{j, true, !(j >= dis_a && j < dis_b)};
+    }
+    const int u = v - n_low, j = u < dis_a ? u : u + n_skip;
+    return Pass{j, false, j >= low_a && j < low_b};
   };
   bool fail = false;
 
   if (producer) {
     if ((tid & 31) == 0) {
       constexpr uint32_t IDESC_S = instr_desc(BN, false), IDESC_O = instr_desc(PD, true);
-      Pass cl = first_pass();                                   // next pass to load
-      int vl = 0;
-      auto load_next = [&]() {
-        if (cl.j >= n_tiles) return;
-        const uint32_t st = st0 + (vl % nstg) * STAGE_B, bar = bar_full + (vl % nstg) * 8;
-        bar_expect_tx(bar, STAGE_B);
+      int kl = 0, vl = 0;                                       // next pass whose keys / values are requested
+      auto load_k = [&]() {
+        if (kl >= n_pass) return;
+        const Pass c = pass_of(kl);
+        const uint32_t dst = sb + OFF_K + (kl % NRING) * KV_B, bar = bar_kfull + (kl % NRING) * 8;
+        bar_expect_tx(bar, KV_B);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          tma_load_3d(st + c * (KV_B / 2), cl.low ? &tmKl : &tmK, c * 64, kvh, cl.j * BN, bar);
-          tma_load_3d(st + KV_B + c * (KV_B / 2), &tmV, c * 64, kvh, cl.j * BN, bar);
-        }
-        cl = next_pass(cl);
+        for (int h = 0; h < 2; ++h) tma_load_3d(dst + h * (KV_B / 2), c.low ? &tmKl : &tmK, h * 64, kvh, c.j * BN, bar);
+        ++kl;
+      };
+      auto load_v = [&]() {
+        if (vl >= n_pass) return;
+        const Pass c = pass_of(vl);
+        const uint32_t dst = sb + OFF_V + (vl % NRING) * KV_B, bar = bar_vfull + (vl % NRING) * 8;
+        bar_expect_tx(bar, KV_B);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) tma_load_3d(dst + h * (KV_B / 2), &tmV, h * 64, kvh, c.j * BN, bar);
         ++vl;
       };
-      Pass cq = first_pass();                                   // next pass whose product is issued
-      auto issue_qk = [&](int v) {                              // S[v & 1] = Q K^T of pass v
-        const uint32_t st = st0 + (v % nstg) * STAGE_B, ts = tm + (v & 1) * TM_SBUF;
-        const uint32_t qa = sb + (cq.low ? OFF_QL : OFF_Q);
+      auto load_q = [&](bool low) {
+        bar_expect_tx(bar_q, NG * Q_B);
+#pragma unroll
+        for (int g = 0; g < NG; ++g)
+#pragma unroll
+          for (int h = 0; h < 2; ++h)
+            tma_load_3d(sb + OFF_Q + g * Q_B + h * (Q_B / 2), low ? &tmQl : &tmQ, h * 64, hq, q0 + g * BM, bar_q);
+      };
+      auto issue_qk = [&](int v) {                              // S[g][v & 1] = Q_g K^T of pass v, both groups
+        const uint32_t kb = sb + OFF_K + (v % NRING) * KV_B;
         tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < PD / 16; ++ks) {                  // 16 channels per step: 4 per 128-byte sub-tile
-          const uint32_t a_off = (ks >> 2) * (Q_B / 2) + (ks & 3) * 32, b_off = (ks >> 2) * (KV_B / 2) + (ks & 3) * 32;
-          umma(ts, smem_desc(qa + a_off, 16, 1024), smem_desc(st + b_off, 16, 1024), IDESC_S, ks > 0);
-        }
-        umma_commit(bar_sfull + (v & 1) * 8);
-        cq = next_pass(cq);
-      };
-      bar_expect_tx(bar_q, Q_B * (shares ? 2 : 1));
+        for (int g = 0; g < NG; ++g) {
+          const uint32_t ts = tm + g * TM_GROUP + (v & 1) * TM_SBUF, qa = sb + OFF_Q + g * Q_B;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        tma_load_3d(sb + OFF_Q + c * (Q_B / 2), &tmQ, c * 64, hq, q0, bar_q);
-        if (shares) tma_load_3d(sb + OFF_QL + c * (Q_B / 2), &tmQl, c * 64, hq, q0, bar_q);
-      }
-      for (int i = 0; i < nstg; ++i) load_next();
-      fail = !bar_wait(bar_q, 0) || !bar_wait(bar_full, 0);
+          for (int ks = 0; ks < PD / 16; ++ks) {                // 16 channels per step: 4 per 128-byte sub-tile
+            const uint32_t a_off = (ks >> 2) * (Q_B / 2) + (ks & 3) * 32, b_off = (ks >> 2) * (KV_B / 2) + (ks & 3) * 32;
+            umma(ts, smem_desc(qa + a_off, 16, 1024), smem_desc(kb + b_off, 16, 1024), IDESC_S, ks > 0);
+          }
+          umma_commit(bar_sfull + (g * 2 + (v & 1)) * 8);
+        }
+      };
+      load_q(n_low > 0);
+      for (int i = 0; i < NRING; ++i) { load_k(); load_v(); }
+      fail = !bar_wait(bar_q, 0) || !bar_wait(bar_kfull, 0);
       if (!fail) issue_qk(0);
-      for (int v = 0; cq.j < n_tiles || v < vl; ++v) {          // v runs over all passes (vl ends as their number)
-        if (v >= vl) break;
+      for (int v = 0; v < n_pass && !fail; ++v) {
         const int b = v & 1, u = (v >> 1) & 1;
-        if (cq.j < n_tiles) {                                   // the next pass's product overlaps this pass's softmax
+        const uint32_t qk_done = bar_sfull + ((NG - 1) * 2 + b) * 8;    // the last group's commit covers both products of pass v
+        if (v + 1 < n_pass) {                                   // the next pass's products overlap this pass's softmax
           const int v1 = v + 1;
-          fail = !bar_wait(bar_full + (v1 % nstg) * 8, (v1 / nstg) & 1);
-          if (!fail && v1 >= 2) fail = !bar_wait(bar_sempty + (v1 & 1) * 8, ((v1 >> 1) & 1) ^ 1);   // S[v1 & 1] of pass v - 1 has been read
+          if (v1 == n_low && n_low > 0) {                       // the passes with this layer's own product begin:
+            fail = !bar_wait(qk_done, u);                       // nothing reads the lowest layer's Q any more
+            if (fail) break;
+            load_q(false);
+            fail = !bar_wait(bar_q, 1);
+            if (fail) break;
+          }
+          fail = !bar_wait(bar_kfull + (v1 % NRING) * 8, (v1 / NRING) & 1);
           if (fail) break;
           issue_qk(v1);
         }
-        if (v >= 1 && cl.j < n_tiles) {                         // the stage of pass v - 1 is free once its P V is done
-          fail = !bar_wait(bar_pvdone + ((v - 1) & 1) * 8, ((v - 1) >> 1) & 1);
+        if (kl < n_pass) {                                      // the key slot of pass v is free once its products are done
+          fail = !bar_wait(qk_done, u);
           if (fail) break;
-          load_next();
+          load_k();
         }
-        fail = !bar_wait(bar_pfull + b * 8, u);                 // P[b] of pass v is written
-        if (fail) break;
-        tc_fence_after();
-        const uint32_t st = st0 + (v % nstg) * STAGE_B;
+        if (v >= 1 && vl < n_pass) {                            // the value slot of pass v - 1 is free once its P V are done
+          fail = !bar_wait(bar_pvdone + ((NG - 1) * 2 + ((v - 1) & 1)) * 8, ((v - 1) >> 1) & 1);
+          if (fail) break;
+          load_v();
+        }
+        fail = !bar_wait(bar_vfull + (v % NRING) * 8, (v / NRING) & 1);
+        const uint32_t vb = sb + OFF_V + (v % NRING) * KV_B;
 #pragma unroll
-        for (int ks = 0; ks < BN / 16; ++ks)                    // 16 keys per step; O accumulates over the passes
-          umma(tm + TM_O, smem_desc(sb + OFF_P + b * P_B + ks * 32, 16, 1024),
-               smem_desc(st + KV_B + ks * 2048, KV_B / 2, 1024), IDESC_O, (v > 0 || ks > 0) ? 1u : 0u);
-        umma_commit(bar_pvdone + b * 8);
+        for (int g = 0; g < NG && !fail; ++g) {
+          fail = !bar_wait(bar_pfull + (g * 2 + b) * 8, u);     // P[g][b] of pass v is written
+          if (fail) break;
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < BN / 16; ++ks)                  // 16 keys per step; O accumulates over the passes
+            umma(tm + g * TM_GROUP + TM_O, smem_desc(sb + OFF_P + (g * 2 + b) * P_B + ks * 32, 16, 1024),
+                 smem_desc(vb + ks * 2048, KV_B / 2, 1024), IDESC_O, (v > 0 || ks > 0) ? 1u : 0u);
+          umma_commit(bar_pvdone + (g * 2 + b) * 8);
+        }
       }
       if (fail) atomicExch(p.err_flag, 1);
     }
   } else {
-    // ---- softmax warps: thread tid owns query row tid -------------------------------------------------
-    const int qi = q0 + tid;
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;     // this warp's quarter of the TMEM lanes
+    // ---- softmax warps: thread r of group g owns query row 128 g + r ----------------------------------
+    const int g = warp >> 2, r = tid & (BM - 1);
+    const int qg0 = q0 + g * BM, qi = qg0 + r;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;   // this warp's quarter of the TMEM lanes
+    const uint32_t tmg = tm + g * TM_GROUP + lane_base;
     float m_used = -INFINITY, l_row = 0.f;
-    int v = 0;
-    for (Pass c = first_pass(); c.j < n_tiles && !fail; c = next_pass(c), ++v) {
+    for (int v = 0; v < n_pass; ++v) {
+      const Pass c = pass_of(v);
       const int b = v & 1, u = (v >> 1) & 1;
-      fail = !bar_wait(bar_sfull + b * 8, u);
+      fail = !bar_wait(bar_sfull + (g * 2 + b) * 8, u);
       if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
       tc_fence_after();
-      const uint32_t ts = tm + b * TM_SBUF + lane_base;
       const int k0 = c.j * BN;
       // this row's 64 raw logits, read from TMEM once.  Interior tiles (every key visible to every row of
-      // the block) need no per-key decision; tiles on the diagonal get the causal mask, and a pass over a
+      // the group) need no per-key decision; tiles on the diagonal get the causal mask, and a pass over a
       // tile with both kinds of key keeps the kind its product is meant for.
       float a[BN];
+      {
+        float t0[32], t1[32];
+        tmem_ld32(tmg + b * TM_SBUF, t0);
+        tmem_ld32(tmg + b * TM_SBUF + 32, t1);
+        tmem_ld_wait();
 #pragma unroll
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        float t[32];
-        tmem_ld32(ts + ch * 32, t);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) a[ch * 32 + i] = t[i];
+        for (int i = 0; i < 32; ++i) { a[i] = t0[i]; a[32 + i] = t1[i]; }
       }
-      if (k0 + BN - 1 > q0) {                                   // diagonal tile: keys after the row's position
+      if (k0 + BN - 1 > qg0) {                                  // diagonal tile: keys after the row's position
 #pragma unroll
         for (int i = 0; i < BN; ++i) a[i] = (k0 + i <= qi && k0 + i < p.T) ? a[i] : -INFINITY;
       }
@@ -315,39 +355,41 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int i = 0; i < BN; ++i) {
           const int kj = k0 + i;
           const bool prox = kj < p.S || kj > qi - p.W;
-          a[i] = (prox != (c.low != 0)) ? a[i] : -INFINITY;     // own product: proximal keys; lowest layer's: distant keys
+          a[i] = (prox != c.low) ? a[i] : -INFINITY;            // own product: proximal keys; lowest layer's: distant keys
         }
       }
-      float mx = -INFINITY;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int i = 0; i < BN; ++i) mx = fmaxf(mx, a[i]);
+      for (int i = 0; i < BN; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], a[i]);
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       mx *= p.scale_log2;                                       // the scale is positive: it commutes with the maximum
       // raise the row's reference maximum only when the tile exceeds it by more than RESCALE_STEP
       const bool raise = mx > m_used + RESCALE_STEP || (m_used == -INFINITY && mx > -INFINITY);
       float alpha = 1.f;
       if (raise) { alpha = ex2f(m_used - mx); m_used = mx; }    // ex2(-inf) = 0 on the first tile
       if (__any_sync(0xffffffffu, raise) && v > 0) {            // rescale this warp's rows of O in TMEM
-        fail = !bar_wait(bar_pvdone + ((v - 1) & 1) * 8, ((v - 1) >> 1) & 1);   // nothing is accumulating into O
+        fail = !bar_wait(bar_pvdone + (g * 2 + ((v - 1) & 1)) * 8, ((v - 1) >> 1) & 1);   // nothing is accumulating into O
         if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
         tc_fence_after();
 #pragma unroll
         for (int ch = 0; ch < PD / 32; ++ch) {
           float t[32];
-          tmem_ld32(tm + TM_O + lane_base + ch * 32, t);
+          tmem_ld32(tmg + TM_O + ch * 32, t);
+          tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; ++i) t[i] *= alpha;
-          tmem_st32(tm + TM_O + lane_base + ch * 32, t);
+          tmem_st32(tmg + TM_O + ch * 32, t);
         }
         tc_fence_before();
       }
       l_row *= alpha;
-      if (v >= 2) {                                             // P[b] was read by P V of pass v - 2
-        fail = !bar_wait(bar_pvdone + b * 8, u ^ 1);
+      if (v >= 2) {                                             // P[g][b] was read by P V of pass v - 2
+        fail = !bar_wait(bar_pvdone + (g * 2 + b) * 8, u ^ 1);
         if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
       }
       const float m_use = (m_used == -INFINITY) ? 0.f : m_used;
-      float psum = 0.f;
-      unsigned char* prow = smem + OFF_P + b * P_B + tid * 128;  // row tid of the [128][128 B] P tile
+      float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+      unsigned char* prow = smem + OFF_P + (g * 2 + b) * P_B + r * 128;   // row r of the [128][128 B] P tile
 #pragma unroll
       for (int c8 = 0; c8 < BN / 8; ++c8) {                     // eight keys = one 16-byte chunk of the row
         uint32_t pk[4];
@@ -355,21 +397,21 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int i = 0; i < 4; ++i) {
           const float p0 = ex2f(fmaf(a[c8 * 8 + 2 * i], p.scale_log2, -m_use));
           const float p1 = ex2f(fmaf(a[c8 * 8 + 2 * i + 1], p.scale_log2, -m_use));
-          psum += p0 + p1;
+          ps4[i] += p0 + p1;
           __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
           pk[i] = *reinterpret_cast<uint32_t*>(&b2);
         }
         // 16-byte chunk c of row r lives at chunk c ^ (r & 7)
-        *reinterpret_cast<uint4*>(prow + ((c8 ^ (tid & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        *reinterpret_cast<uint4*>(prow + ((c8 ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
-      l_row += psum;
+      l_row += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor cores
       tc_fence_before();
-      bar_arrive(bar_pfull + b * 8);
-      bar_arrive(bar_sempty + b * 8);
+      bar_arrive(bar_pfull + (g * 2 + b) * 8);
     }
     if (!fail) {
-      fail = !bar_wait(bar_pvdone + ((v - 1) & 1) * 8, ((v - 1) >> 1) & 1);
+      const int vz = n_pass - 1;
+      fail = !bar_wait(bar_pvdone + (g * 2 + (vz & 1)) * 8, (vz >> 1) & 1);
       fail = __any_sync(0xffffffffu, fail);
     }
     if (fail) {
@@ -381,7 +423,8 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
       for (int ch = 0; ch < PD / 32; ++ch) {
         float t[32];
-        tmem_ld32(tm + TM_O + lane_base + ch * 32, t);          // warp-collective: rows past T load too
+        tmem_ld32(tmg + TM_O + ch * 32, t);                     // warp-collective: rows past T load too
+        tmem_ld_wait();
         if (qi < p.T) {
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
@@ -472,7 +515,7 @@ extern "C" int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int
       !encode_3d(su->encode, &tv, v, n_tokens, n_kv_heads, BN) || !encode_3d(su->encode, &tql, ql, n_tokens, n_q_heads, BM) ||
       !encode_3d(su->encode, &tkl, kl, n_tokens, n_kv_heads, BN))
     return POD_ERR_INVALID;
-  dim3 grid((n_tokens + BM - 1) / BM, n_q_heads);
+  dim3 grid((n_tokens + BLK - 1) / BLK, n_q_heads);
   pod_prefill_kernel<<<grid, PF_THREADS, PF_SMEM, static_cast<cudaStream_t>(cuda_stream)>>>(tq, tk, tv, tql, tkl, p);
   return cudaGetLastError() == cudaSuccess ? POD_OK : POD_ERR_CUDA;
 }
