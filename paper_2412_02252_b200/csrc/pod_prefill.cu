@@ -59,7 +59,7 @@ constexpr int OFF_K = NG * Q_B, OFF_V = OFF_K + NRING * KV_B;
 constexpr int OFF_P = OFF_V + NRING * KV_B;      // per group two P tiles
 constexpr int OFF_BAR = OFF_P + NG * 2 * P_B;
 constexpr int PF_SMEM = OFF_BAR + 256 + 1024;
-constexpr int PF_THREADS = BLK + 32;    // eight softmax warps + the producer warp
+constexpr int PF_THREADS = BLK + 64;    // eight softmax warps, the tensor-core warp, the load warp
 constexpr int TM_COLS = 512;            // per group 2 x S 64 + O 128 fp32 columns
 constexpr int TM_GROUP = 256, TM_SBUF = 64, TM_O = 128;
 constexpr float RESCALE_STEP = 8.f;     // raise a row's reference maximum only past this many log2 units
@@ -170,21 +170,24 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pf_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sb = s2u(smem);
   const int tid = threadIdx.x, warp = tid >> 5;
-  const bool producer = warp == BLK / 32;
+  const bool producer = warp == BLK / 32, loader = warp == BLK / 32 + 1;   // tensor-core warp, load warp
   const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;          // long rows first
   const int hq = blockIdx.y, kvh = hq / (p.H_q / p.H_kv);
   const int q0 = qb * BLK;
   const bool shares = kvh < 256 && ((p.share_mask[kvh >> 5] >> (kvh & 31)) & 1u);
-  // mbarriers: Q landed; per ring slot: K landed, V landed; per group and buffer: S ready, P written, P V done
+  // mbarriers: Q landed; per ring slot: K landed, V landed, K slot free, V slot free; per group and buffer:
+  // S ready, P written, P V done
   const uint32_t bar_q = sb + OFF_BAR, bar_kfull = bar_q + 8, bar_vfull = bar_q + 32, bar_sfull = bar_q + 56,
-                 bar_pfull = bar_q + 88, bar_pvdone = bar_q + 120;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 192);
+                 bar_pfull = bar_q + 88, bar_pvdone = bar_q + 120, bar_kfree = bar_q + 152, bar_vfree = bar_q + 176;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 224);
 
   if (tid == 0) {
     bar_init(bar_q, 1);
     for (int i = 0; i < NRING; ++i) {
       bar_init(bar_kfull + i * 8, 1);
       bar_init(bar_vfull + i * 8, 1);
+      bar_init(bar_kfree + i * 8, 1);
+      bar_init(bar_vfree + i * 8, 1);
     }
     for (int i = 0; i < NG * 2; ++i) {
       bar_init(bar_sfull + i * 8, 1);
@@ -230,9 +233,9 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   };
   bool fail = false;
 
-  if (producer) {
+  if (loader) {
+    // ---- load warp: one thread requests Q, then keeps the two rings full --------------------------------
     if ((tid & 31) == 0) {
-      constexpr uint32_t IDESC_S = instr_desc(BN, false), IDESC_O = instr_desc(PD, true);
       int kl = 0, vl = 0;                                       // next pass whose keys / values are requested
       auto load_k = [&]() {
         if (kl >= n_pass) return;
@@ -260,33 +263,55 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           for (int h = 0; h < 2; ++h)
             tma_load_3d(sb + OFF_Q + g * Q_B + h * (Q_B / 2), low ? &tmQl : &tmQ, h * 64, hq, q0 + g * BM, bar_q);
       };
+      load_q(n_low > 0);
+      for (int i = 0; i < NRING; ++i) { load_k(); load_v(); }
+      for (int v = 0; v < n_pass && !fail; ++v) {
+        const bool q_switch = n_low > 0 && v + 1 == n_low;      // pass v is the last with the lowest layer's product
+        if (q_switch || kl < n_pass) {                          // both products of pass v are done: its key slot is free,
+          fail = !bar_wait(bar_kfree + (v % NRING) * 8, (v / NRING) & 1);
+          if (fail) break;
+          if (q_switch) load_q(false);                          // and after the last such pass nothing reads Q_a any more
+          load_k();
+        }
+        if (vl < n_pass) {                                      // the value slot of pass v is free once its P V are done
+          fail = !bar_wait(bar_vfree + (v % NRING) * 8, (v / NRING) & 1);
+          if (fail) break;
+          load_v();
+        }
+      }
+      if (fail) atomicExch(p.err_flag, 1);
+    }
+  } else if (producer) {
+    // ---- tensor-core warp: one thread issues every product -------------------------------------------------
+    if ((tid & 31) == 0) {
+      constexpr uint32_t IDESC_S = instr_desc(BN, false), IDESC_O = instr_desc(PD, true);
+      // Descriptors of the operands' first steps, built once: a later step or slot only adds its byte offset
+      // / 16 to the address field (shared-memory addresses stay below 2^18, so the field never carries).
+      const uint64_t dq0 = smem_desc(sb + OFF_Q, 16, 1024), dk0 = smem_desc(sb + OFF_K, 16, 1024);
+      const uint64_t dp0 = smem_desc(sb + OFF_P, 16, 1024), dv0 = smem_desc(sb + OFF_V, KV_B / 2, 1024);
       auto issue_qk = [&](int v) {                              // S[g][v & 1] = Q_g K^T of pass v, both groups
-        const uint32_t kb = sb + OFF_K + (v % NRING) * KV_B;
+        const uint64_t dk = dk0 + (uint64_t)((v % NRING) * (KV_B >> 4));
         tc_fence_after();
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
-          const uint32_t ts = tm + g * TM_GROUP + (v & 1) * TM_SBUF, qa = sb + OFF_Q + g * Q_B;
+          const uint32_t ts = tm + g * TM_GROUP + (v & 1) * TM_SBUF;
+          const uint64_t dq = dq0 + (uint64_t)(g * (Q_B >> 4));
 #pragma unroll
           for (int ks = 0; ks < PD / 16; ++ks) {                // 16 channels per step: 4 per 128-byte sub-tile
             const uint32_t a_off = (ks >> 2) * (Q_B / 2) + (ks & 3) * 32, b_off = (ks >> 2) * (KV_B / 2) + (ks & 3) * 32;
-            umma(ts, smem_desc(qa + a_off, 16, 1024), smem_desc(kb + b_off, 16, 1024), IDESC_S, ks > 0);
+            umma(ts, dq + (uint64_t)(a_off >> 4), dk + (uint64_t)(b_off >> 4), IDESC_S, ks > 0);
           }
           umma_commit(bar_sfull + (g * 2 + (v & 1)) * 8);
         }
+        umma_commit(bar_kfree + (v % NRING) * 8);
       };
-      load_q(n_low > 0);
-      for (int i = 0; i < NRING; ++i) { load_k(); load_v(); }
       fail = !bar_wait(bar_q, 0) || !bar_wait(bar_kfull, 0);
       if (!fail) issue_qk(0);
       for (int v = 0; v < n_pass && !fail; ++v) {
         const int b = v & 1, u = (v >> 1) & 1;
-        const uint32_t qk_done = bar_sfull + ((NG - 1) * 2 + b) * 8;    // the last group's commit covers both products of pass v
         if (v + 1 < n_pass) {                                   // the next pass's products overlap this pass's softmax
           const int v1 = v + 1;
-          if (v1 == n_low && n_low > 0) {                       // the passes with this layer's own product begin:
-            fail = !bar_wait(qk_done, u);                       // nothing reads the lowest layer's Q any more
-            if (fail) break;
-            load_q(false);
+          if (v1 == n_low && n_low > 0) {                       // the passes with this layer's own product begin
             fail = !bar_wait(bar_q, 1);
             if (fail) break;
           }
@@ -294,18 +319,8 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           if (fail) break;
           issue_qk(v1);
         }
-        if (kl < n_pass) {                                      // the key slot of pass v is free once its products are done
-          fail = !bar_wait(qk_done, u);
-          if (fail) break;
-          load_k();
-        }
-        if (v >= 1 && vl < n_pass) {                            // the value slot of pass v - 1 is free once its P V are done
-          fail = !bar_wait(bar_pvdone + ((NG - 1) * 2 + ((v - 1) & 1)) * 8, ((v - 1) >> 1) & 1);
-          if (fail) break;
-          load_v();
-        }
         fail = !bar_wait(bar_vfull + (v % NRING) * 8, (v / NRING) & 1);
-        const uint32_t vb = sb + OFF_V + (v % NRING) * KV_B;
+        const uint64_t dv = dv0 + (uint64_t)((v % NRING) * (KV_B >> 4));
 #pragma unroll
         for (int g = 0; g < NG && !fail; ++g) {
           fail = !bar_wait(bar_pfull + (g * 2 + b) * 8, u);     // P[g][b] of pass v is written
@@ -313,10 +328,11 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           tc_fence_after();
 #pragma unroll
           for (int ks = 0; ks < BN / 16; ++ks)                  // 16 keys per step; O accumulates over the passes
-            umma(tm + g * TM_GROUP + TM_O, smem_desc(sb + OFF_P + (g * 2 + b) * P_B + ks * 32, 16, 1024),
-                 smem_desc(vb + ks * 2048, KV_B / 2, 1024), IDESC_O, (v > 0 || ks > 0) ? 1u : 0u);
+            umma(tm + g * TM_GROUP + TM_O, dp0 + (uint64_t)((g * 2 + b) * (P_B >> 4) + ks * 2),
+                 dv + (uint64_t)(ks * (2048 >> 4)), IDESC_O, (v > 0 || ks > 0) ? 1u : 0u);
           umma_commit(bar_pvdone + (g * 2 + b) * 8);
         }
+        if (!fail) umma_commit(bar_vfree + (v % NRING) * 8);
       }
       if (fail) atomicExch(p.err_flag, 1);
     }
