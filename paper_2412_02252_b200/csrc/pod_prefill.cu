@@ -8,29 +8,29 @@
 // same product).  One softmax over both groups weighs layer l's own values.
 //
 // One CTA = 256 consecutive query positions of one query head: two softmax groups of four warps (group g
-// owns rows 128 g .. 128 g + 127, one thread per row) and one producer warp whose lane 0 issues every TMA
-// load and every tcgen05.mma.  Both groups work on the same key/value tile at the same time, so each tile
-// is fetched once per 256 rows and the tensor cores always have the other group's products to run while
-// one group is in its softmax.  Keys and values of 64 positions stream through two rings of three
-// 16 KiB slots (TMA, 128-byte swizzle); a key slot is refilled as soon as its products are done, a value
-// slot after the P V products.
+// owns rows 128 g .. 128 g + 127, one thread per row), one warp whose lane 0 issues every tcgen05.mma and
+// one warp whose lane 0 issues every TMA load.  Keys and values arrive in tiles of 128 positions through a
+// ring of five 32 KiB shared-memory slots (K_0, V_0, K_1, V_1, ...; TMA, 128-byte swizzle); both groups
+// use the same tile, so each is fetched once per 256 rows.
 // A tile whose keys are all distant for every row of the CTA is scored with Q_a K_a^T, one whose keys are
 // all proximal (or whose head does not share) with Q K^T; the few tiles that straddle the edge of the
 // window or of the sink are taken twice, once with each product and the other kind of key masked (the
 // softmax does not care in how many pieces, or in which order, the keys arrive).  The passes that use the
 // lowest layer's product run first, with Q_a in the query buffers; then Q of this layer is loaded over it
-// and the other passes follow.  Per pass v and group g:
-//   S[128 x 64] = Q K^T  or  Q_a K_a^T       (M = 128, N = 64, K = 16 x 8 steps, into one of two TMEM buffers:
-//                                              the product of pass v + 1 runs while pass v is in the softmax)
-//   each softmax thread reads its row of S from TMEM (tcgen05.ld), masks, and
-//   writes its row of P = 2^(logit - m) as bf16 into one of two swizzled shared-memory tiles
-//   O[128 x 128] += P V                       (A = P K-major, B = V MN-major, K = 16 x 4), accumulated in TMEM.
-// The reference maximum m of a row is only raised when the tile's maximum exceeds it by more than 8 (in
-// log2 units): P then stays below 2^8, and the rows of O in TMEM have to be rescaled (tcgen05.ld / st)
-// only on those rare occasions instead of after every tile; row sum and O share the same m, so the
-// quotient is exact either way.  Warps hand buffers to one another through mbarriers; every wait is bounded
-// (a wait gives up only after seconds, long after every copy in flight has landed), a wait that gives up
-// raises the error flag, and the tensor memory is always returned before the CTA exits.
+// and the other passes follow.  Per pass v and group g, in tensor memory (per group 128 columns for S and
+// P, 128 for O):
+//   S[128 x 128] = Q K^T  or  Q_a K_a^T      (M = 128, N = 128, K = 16 x 8 steps)
+//   each softmax thread reads its row of S (tcgen05.ld) for the maximum, reads it again in four pieces and
+//   writes P = 2^(logit - m) as packed bf16 over the columns of S it has already consumed (tcgen05.st)
+//   O[128 x 128] += P V                       (A = P from tensor memory, B = V MN-major, K = 16 x 8).
+// The tensor-core thread alternates between the groups (P V of group g, then its next Q K^T), so one group's
+// products run while the other group is in its softmax.  The reference maximum m of a row is only raised
+// when the tile's maximum exceeds it by more than 8 (in log2 units): P then stays below 2^8, and the rows of
+// O have to be rescaled (tcgen05.ld / st) only on those rare occasions instead of after every tile; row sum
+// and O share the same m, so the quotient is exact either way.  Warps hand buffers to one another through
+// mbarriers; every wait is bounded (a wait gives up only after seconds, long after every copy in flight has
+// landed), a wait that gives up raises the error flag, and the tensor memory is always returned before the
+// CTA exits.
 #include <cudaTypedefs.h>
 #include <cuda_bf16.h>
 #include <math.h>
@@ -47,21 +47,19 @@ constexpr int PD = 128;                 // head_dim
 constexpr int BM = 128;                 // query rows per softmax group
 constexpr int NG = 2;                   // softmax groups per CTA
 constexpr int BLK = NG * BM;            // query rows per CTA
-constexpr int BN = 64;                  // keys per tile
-constexpr int NRING = 3;                // slots of the key ring and of the value ring
+constexpr int BN = 128;                 // keys per tile
+constexpr int NRING = 5;                // slots of the K/V ring
 constexpr uint32_t PF_WAIT_LIMIT = 1u << 22;
 
 constexpr int Q_B = BM * PD * 2;        // 32 KiB: two [128][128 B] sub-tiles
-constexpr int KV_B = BN * PD * 2;       // 16 KiB: two [64][128 B] sub-tiles
-constexpr int P_B = BM * BN * 2;        // 16 KiB: one [128][128 B] tile
+constexpr int KV_B = BN * PD * 2;       // 32 KiB: two [128][128 B] sub-tiles
 constexpr int OFF_Q = 0;                // per group: Q of the lowest layer, later Q of this layer
-constexpr int OFF_K = NG * Q_B, OFF_V = OFF_K + NRING * KV_B;
-constexpr int OFF_P = OFF_V + NRING * KV_B;      // per group two P tiles
-constexpr int OFF_BAR = OFF_P + NG * 2 * P_B;
+constexpr int OFF_RING = NG * Q_B;
+constexpr int OFF_BAR = OFF_RING + NRING * KV_B;
 constexpr int PF_SMEM = OFF_BAR + 256 + 1024;
 constexpr int PF_THREADS = BLK + 64;    // eight softmax warps, the tensor-core warp, the load warp
-constexpr int TM_COLS = 512;            // per group 2 x S 64 + O 128 fp32 columns
-constexpr int TM_GROUP = 256, TM_SBUF = 64, TM_O = 128;
+constexpr int TM_COLS = 512;            // per group S / P 128 + O 128 fp32 columns
+constexpr int TM_GROUP = 256, TM_O = 128;
 constexpr float RESCALE_STEP = 8.f;     // raise a row's reference maximum only past this many log2 units
 
 struct PrefillParams {
@@ -115,6 +113,14 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// the same with A read from tensor memory (128 lanes x 8 columns of packed bf16 pairs per step)
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -153,6 +159,16 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
       : "memory");
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
+// 16 consecutive 32-bit columns of this thread's TMEM lane (complete after tmem_st_wait)
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void bar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -175,29 +191,26 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const int hq = blockIdx.y, kvh = hq / (p.H_q / p.H_kv);
   const int q0 = qb * BLK;
   const bool shares = kvh < 256 && ((p.share_mask[kvh >> 5] >> (kvh & 31)) & 1u);
-  // mbarriers: Q landed; per ring slot: K landed, V landed, K slot free, V slot free; per group and buffer:
-  // S ready, P written, P V done
-  const uint32_t bar_q = sb + OFF_BAR, bar_kfull = bar_q + 8, bar_vfull = bar_q + 32, bar_sfull = bar_q + 56,
-                 bar_pfull = bar_q + 88, bar_pvdone = bar_q + 120, bar_kfree = bar_q + 152, bar_vfree = bar_q + 176;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 224);
+  // mbarriers: Q landed; per ring slot: tile landed, slot free; per group: S ready, P written, O complete
+  const uint32_t bar_q = sb + OFF_BAR, bar_full = bar_q + 8, bar_free = bar_q + 48, bar_sfull = bar_q + 88,
+                 bar_pfull = bar_q + 104, bar_odone = bar_q + 120;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 192);
 
   if (tid == 0) {
     bar_init(bar_q, 1);
     for (int i = 0; i < NRING; ++i) {
-      bar_init(bar_kfull + i * 8, 1);
-      bar_init(bar_vfull + i * 8, 1);
-      bar_init(bar_kfree + i * 8, 1);
-      bar_init(bar_vfree + i * 8, 1);
+      bar_init(bar_full + i * 8, 1);
+      bar_init(bar_free + i * 8, 1);
     }
-    for (int i = 0; i < NG * 2; ++i) {
-      bar_init(bar_sfull + i * 8, 1);
-      bar_init(bar_pfull + i * 8, BM);
-      bar_init(bar_pvdone + i * 8, 1);
+    for (int g = 0; g < NG; ++g) {
+      bar_init(bar_sfull + g * 8, 1);
+      bar_init(bar_pfull + g * 8, BM / 32);                     // one arrival per softmax warp
+      bar_init(bar_odone + g * 8, 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (producer) {                                               // tensor memory for the S buffers and O
+  if (producer) {                                               // all of the SM's tensor memory: S / P and O of both groups
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s2u(tmem_slot)), "r"(TM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -206,19 +219,19 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   tc_fence_after();
   const uint32_t tm = *tmem_slot;
 
-  // keys this CTA needs: positions [0, min(T, q0 + 256)); tile j covers [64 j, 64 j + 64)
+  // keys this CTA needs: positions [0, min(T, q0 + 256)); tile j covers [128 j, 128 j + 128)
   const int k_end = min(p.T, q0 + BLK);
   const int n_tiles = (k_end + BN - 1) / BN;
   // Tiles [low_a, low_b) hold a key that is distant for some row of the CTA: they get a pass with the lowest
   // layer's product.  Of those, tiles [dis_a, dis_b) are distant for every row and get no other pass.
   int low_a = 0, low_b = 0, dis_a = 0, dis_b = 0;
   if (shares) {
-    low_a = p.S >> 6;                                           // tiles before it lie inside the sink
+    low_a = p.S / BN;                                           // tiles before it lie inside the sink
     const int e = q0 + BLK - 1 - p.W;                           // the last row's newest distant position
-    low_b = max(low_a, min(e < 0 ? 0 : (e >> 6) + 1, n_tiles));
-    dis_a = (p.S + BN - 1) >> 6;
-    const int f = q0 - p.W - (BN - 1);                          // tile j is distant for the first row too if 64 j <= f
-    dis_b = max(dis_a, min(f < 0 ? 0 : (f >> 6) + 1, low_b));
+    low_b = max(low_a, min(e < 0 ? 0 : e / BN + 1, n_tiles));
+    dis_a = (p.S + BN - 1) / BN;
+    const int f = q0 - p.W - (BN - 1);                          // tile j is distant for the first row too if 128 j <= f
+    dis_b = max(dis_a, min(f < 0 ? 0 : f / BN + 1, low_b));
   }
   const int n_low = low_b - low_a, n_skip = dis_b - dis_a;
   const int n_pass = n_low + n_tiles - n_skip;
@@ -234,27 +247,8 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   bool fail = false;
 
   if (loader) {
-    // ---- load warp: one thread requests Q, then keeps the two rings full --------------------------------
+    // ---- load warp: one thread requests Q, then keeps the ring full: load 2 v is K of pass v, 2 v + 1 its V ----
     if ((tid & 31) == 0) {
-      int kl = 0, vl = 0;                                       // next pass whose keys / values are requested
-      auto load_k = [&]() {
-        if (kl >= n_pass) return;
-        const Pass c = pass_of(kl);
-        const uint32_t dst = sb + OFF_K + (kl % NRING) * KV_B, bar = bar_kfull + (kl % NRING) * 8;
-        bar_expect_tx(bar, KV_B);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) tma_load_3d(dst + h * (KV_B / 2), c.low ? &tmKl : &tmK, h * 64, kvh, c.j * BN, bar);
-        ++kl;
-      };
-      auto load_v = [&]() {
-        if (vl >= n_pass) return;
-        const Pass c = pass_of(vl);
-        const uint32_t dst = sb + OFF_V + (vl % NRING) * KV_B, bar = bar_vfull + (vl % NRING) * 8;
-        bar_expect_tx(bar, KV_B);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) tma_load_3d(dst + h * (KV_B / 2), &tmV, h * 64, kvh, c.j * BN, bar);
-        ++vl;
-      };
       auto load_q = [&](bool low) {
         bar_expect_tx(bar_q, NG * Q_B);
 #pragma unroll
@@ -264,75 +258,76 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             tma_load_3d(sb + OFF_Q + g * Q_B + h * (Q_B / 2), low ? &tmQl : &tmQ, h * 64, hq, q0 + g * BM, bar_q);
       };
       load_q(n_low > 0);
-      for (int i = 0; i < NRING; ++i) { load_k(); load_v(); }
-      for (int v = 0; v < n_pass && !fail; ++v) {
-        const bool q_switch = n_low > 0 && v + 1 == n_low;      // pass v is the last with the lowest layer's product
-        if (q_switch || kl < n_pass) {                          // both products of pass v are done: its key slot is free,
-          fail = !bar_wait(bar_kfree + (v % NRING) * 8, (v / NRING) & 1);
+      const int n_loads = 2 * n_pass;
+      const int i_switch = n_low > 0 ? 2 * (n_low - 1) : -1;    // the last load whose product reads the lowest layer's Q
+      bool switched = n_low == 0;
+      for (int i = 0; i < n_loads && !fail; ++i) {
+        const int slot = i % NRING;
+        if (i >= NRING) {                                       // the slot's previous tile (load i - 5) has been used
+          fail = !bar_wait(bar_free + slot * 8, ((i / NRING) - 1) & 1);
           if (fail) break;
-          if (q_switch) load_q(false);                          // and after the last such pass nothing reads Q_a any more
-          load_k();
+          if (i - NRING == i_switch) { load_q(false); switched = true; }   // both groups' last products with Q_a are done
         }
-        if (vl < n_pass) {                                      // the value slot of pass v is free once its P V are done
-          fail = !bar_wait(bar_vfree + (v % NRING) * 8, (v / NRING) & 1);
-          if (fail) break;
-          load_v();
-        }
+        const Pass c = pass_of(i >> 1);
+        const CUtensorMap* map = (i & 1) ? &tmV : (c.low ? &tmKl : &tmK);
+        const uint32_t dst = sb + OFF_RING + slot * KV_B, bar = bar_full + slot * 8;
+        bar_expect_tx(bar, KV_B);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) tma_load_3d(dst + h * (KV_B / 2), map, h * 64, kvh, c.j * BN, bar);
+      }
+      if (!fail && !switched) {                                 // the ring never came back to that slot
+        fail = !bar_wait(bar_free + (i_switch % NRING) * 8, (i_switch / NRING) & 1);
+        if (!fail) load_q(false);
       }
       if (fail) atomicExch(p.err_flag, 1);
     }
   } else if (producer) {
     // ---- tensor-core warp: one thread issues every product -------------------------------------------------
     if ((tid & 31) == 0) {
-      constexpr uint32_t IDESC_S = instr_desc(BN, false), IDESC_O = instr_desc(PD, true);
+      constexpr uint32_t IDESC = instr_desc(128, false), IDESC_O = instr_desc(PD, true);
       // Descriptors of the operands' first steps, built once: a later step or slot only adds its byte offset
       // / 16 to the address field (shared-memory addresses stay below 2^18, so the field never carries).
-      const uint64_t dq0 = smem_desc(sb + OFF_Q, 16, 1024), dk0 = smem_desc(sb + OFF_K, 16, 1024);
-      const uint64_t dp0 = smem_desc(sb + OFF_P, 16, 1024), dv0 = smem_desc(sb + OFF_V, KV_B / 2, 1024);
-      auto issue_qk = [&](int v) {                              // S[g][v & 1] = Q_g K^T of pass v, both groups
-        const uint64_t dk = dk0 + (uint64_t)((v % NRING) * (KV_B >> 4));
-        tc_fence_after();
+      const uint64_t dq0 = smem_desc(sb + OFF_Q, 16, 1024), dk0 = smem_desc(sb + OFF_RING, 16, 1024);
+      const uint64_t dv0 = smem_desc(sb + OFF_RING, KV_B / 2, 1024);
+      auto issue_qk = [&](int g, int v) {                       // S[g] = Q_g K^T of pass v
+        const uint64_t dk = dk0 + (uint64_t)(((2 * v) % NRING) * (KV_B >> 4));
+        const uint64_t dq = dq0 + (uint64_t)(g * (Q_B >> 4));
 #pragma unroll
-        for (int g = 0; g < NG; ++g) {
-          const uint32_t ts = tm + g * TM_GROUP + (v & 1) * TM_SBUF;
-          const uint64_t dq = dq0 + (uint64_t)(g * (Q_B >> 4));
-#pragma unroll
-          for (int ks = 0; ks < PD / 16; ++ks) {                // 16 channels per step: 4 per 128-byte sub-tile
-            const uint32_t a_off = (ks >> 2) * (Q_B / 2) + (ks & 3) * 32, b_off = (ks >> 2) * (KV_B / 2) + (ks & 3) * 32;
-            umma(ts, dq + (uint64_t)(a_off >> 4), dk + (uint64_t)(b_off >> 4), IDESC_S, ks > 0);
-          }
-          umma_commit(bar_sfull + (g * 2 + (v & 1)) * 8);
+        for (int ks = 0; ks < PD / 16; ++ks) {                  // 16 channels per step: 4 per 128-byte sub-tile
+          const uint32_t a_off = (ks >> 2) * (Q_B / 2) + (ks & 3) * 32, b_off = (ks >> 2) * (KV_B / 2) + (ks & 3) * 32;
+          umma(tm + g * TM_GROUP, dq + (uint64_t)(a_off >> 4), dk + (uint64_t)(b_off >> 4), IDESC, ks > 0);
         }
-        umma_commit(bar_kfree + (v % NRING) * 8);
+        umma_commit(bar_sfull + g * 8);
+        if (g == NG - 1) umma_commit(bar_free + ((2 * v) % NRING) * 8);   // both groups are done with this K tile
       };
-      fail = !bar_wait(bar_q, 0) || !bar_wait(bar_kfull, 0);
-      if (!fail) issue_qk(0);
+      auto wait_k = [&](int v) -> bool {                        // K of pass v (and the Q it goes with) has landed
+        if (v == 0 && !bar_wait(bar_q, 0)) return false;
+        if (v == n_low && n_low > 0 && !bar_wait(bar_q, 1)) return false;
+        return bar_wait(bar_full + ((2 * v) % NRING) * 8, ((2 * v) / NRING) & 1);
+      };
+      fail = !wait_k(0);
+      if (!fail) {
+        tc_fence_after();
+        for (int g = 0; g < NG; ++g) issue_qk(g, 0);
+      }
       for (int v = 0; v < n_pass && !fail; ++v) {
-        const int b = v & 1, u = (v >> 1) & 1;
-        if (v + 1 < n_pass) {                                   // the next pass's products overlap this pass's softmax
-          const int v1 = v + 1;
-          if (v1 == n_low && n_low > 0) {                       // the passes with this layer's own product begin
-            fail = !bar_wait(bar_q, 1);
-            if (fail) break;
-          }
-          fail = !bar_wait(bar_kfull + (v1 % NRING) * 8, (v1 / NRING) & 1);
-          if (fail) break;
-          issue_qk(v1);
-        }
-        fail = !bar_wait(bar_vfull + (v % NRING) * 8, (v / NRING) & 1);
-        const uint64_t dv = dv0 + (uint64_t)((v % NRING) * (KV_B >> 4));
+        const int iv = 2 * v + 1;                               // the load that brought V of pass v
+        fail = !bar_wait(bar_full + (iv % NRING) * 8, (iv / NRING) & 1);
+        if (!fail && v + 1 < n_pass) fail = !wait_k(v + 1);
+        const uint64_t dv = dv0 + (uint64_t)((iv % NRING) * (KV_B >> 4));
 #pragma unroll
         for (int g = 0; g < NG && !fail; ++g) {
-          fail = !bar_wait(bar_pfull + (g * 2 + b) * 8, u);     // P[g][b] of pass v is written
+          fail = !bar_wait(bar_pfull + g * 8, v & 1);           // P[g] of pass v is written
           if (fail) break;
           tc_fence_after();
 #pragma unroll
           for (int ks = 0; ks < BN / 16; ++ks)                  // 16 keys per step; O accumulates over the passes
-            umma(tm + g * TM_GROUP + TM_O, dp0 + (uint64_t)((g * 2 + b) * (P_B >> 4) + ks * 2),
-                 dv + (uint64_t)(ks * (2048 >> 4)), IDESC_O, (v > 0 || ks > 0) ? 1u : 0u);
-          umma_commit(bar_pvdone + (g * 2 + b) * 8);
+            umma_ts(tm + g * TM_GROUP + TM_O, tm + g * TM_GROUP + ks * 8, dv + (uint64_t)(ks * (2048 >> 4)), IDESC_O,
+                    (v > 0 || ks > 0) ? 1u : 0u);
+          if (g == NG - 1) umma_commit(bar_free + (iv % NRING) * 8);      // both groups are done with this V tile
+          if (v + 1 < n_pass) issue_qk(g, v + 1);               // overwrites P[g]: in order behind the P V just issued
+          else umma_commit(bar_odone + g * 8);
         }
-        if (!fail) umma_commit(bar_vfree + (v % NRING) * 8);
       }
       if (fail) atomicExch(p.err_flag, 1);
     }
@@ -345,48 +340,45 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     float m_used = -INFINITY, l_row = 0.f;
     for (int v = 0; v < n_pass; ++v) {
       const Pass c = pass_of(v);
-      const int b = v & 1, u = (v >> 1) & 1;
-      fail = !bar_wait(bar_sfull + (g * 2 + b) * 8, u);
+      fail = !bar_wait(bar_sfull + g * 8, v & 1);               // S of pass v is complete, and so is every earlier P V
       if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
       tc_fence_after();
       const int k0 = c.j * BN;
-      // this row's 64 raw logits, read from TMEM once.  Interior tiles (every key visible to every row of
-      // the group) need no per-key decision; tiles on the diagonal get the causal mask, and a pass over a
-      // tile with both kinds of key keeps the kind its product is meant for.
-      float a[BN];
-      {
-        float t0[32], t1[32];
-        tmem_ld32(tmg + b * TM_SBUF, t0);
-        tmem_ld32(tmg + b * TM_SBUF + 32, t1);
-        tmem_ld_wait();
+      // Interior tiles (every key visible to every row of the group) need no per-key decision; tiles on the
+      // diagonal get the causal mask, and a pass over a tile with both kinds of key keeps the kind its
+      // product is meant for.
+      const bool masked = c.mixed || (k0 + BN - 1 > qg0);
+      auto mask32 = [&](float (&t)[32], int kbase) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) { a[i] = t0[i]; a[32 + i] = t1[i]; }
-      }
-      if (k0 + BN - 1 > qg0) {                                  // diagonal tile: keys after the row's position
-#pragma unroll
-        for (int i = 0; i < BN; ++i) a[i] = (k0 + i <= qi && k0 + i < p.T) ? a[i] : -INFINITY;
-      }
-      if (c.mixed) {
-#pragma unroll
-        for (int i = 0; i < BN; ++i) {
-          const int kj = k0 + i;
-          const bool prox = kj < p.S || kj > qi - p.W;
-          a[i] = (prox != c.low) ? a[i] : -INFINITY;            // own product: proximal keys; lowest layer's: distant keys
+        for (int i = 0; i < 32; ++i) {
+          const int kj = kbase + i;
+          bool keep = kj <= qi && kj < p.T;
+          if (c.mixed) {
+            const bool prox = kj < p.S || kj > qi - p.W;
+            keep = keep && (prox != c.low);                     // own product: proximal keys; lowest layer's: distant keys
+          }
+          t[i] = keep ? t[i] : -INFINITY;
         }
-      }
+      };
+      // first reading of the row: its maximum
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int i = 0; i < BN; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], a[i]);
+      for (int h = 0; h < 2; ++h) {
+        float t0[32], t1[32];
+        tmem_ld32(tmg + h * 64, t0);
+        tmem_ld32(tmg + h * 64 + 32, t1);
+        tmem_ld_wait();
+        if (masked) { mask32(t0, k0 + h * 64); mask32(t1, k0 + h * 64 + 32); }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(t0[i], t1[i]));
+      }
       float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       mx *= p.scale_log2;                                       // the scale is positive: it commutes with the maximum
       // raise the row's reference maximum only when the tile exceeds it by more than RESCALE_STEP
       const bool raise = mx > m_used + RESCALE_STEP || (m_used == -INFINITY && mx > -INFINITY);
       float alpha = 1.f;
       if (raise) { alpha = ex2f(m_used - mx); m_used = mx; }    // ex2(-inf) = 0 on the first tile
-      if (__any_sync(0xffffffffu, raise) && v > 0) {            // rescale this warp's rows of O in TMEM
-        fail = !bar_wait(bar_pvdone + (g * 2 + ((v - 1) & 1)) * 8, ((v - 1) >> 1) & 1);   // nothing is accumulating into O
-        if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
-        tc_fence_after();
+      if (__any_sync(0xffffffffu, raise) && v > 0) {            // rescale this warp's rows of O (nothing accumulates now)
 #pragma unroll
         for (int ch = 0; ch < PD / 32; ++ch) {
           float t[32];
@@ -396,38 +388,37 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           for (int i = 0; i < 32; ++i) t[i] *= alpha;
           tmem_st32(tmg + TM_O + ch * 32, t);
         }
-        tc_fence_before();
       }
       l_row *= alpha;
-      if (v >= 2) {                                             // P[g][b] was read by P V of pass v - 2
-        fail = !bar_wait(bar_pvdone + (g * 2 + b) * 8, u ^ 1);
-        if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
-      }
       const float m_use = (m_used == -INFINITY) ? 0.f : m_used;
+      // second reading, 32 keys at a time: P as packed bf16 pairs over columns already consumed
+      // (keys 32 c .. 32 c + 31 of S sit in columns 32 c .., their P in columns 16 c .. 16 c + 15)
       float ps4[4] = {0.f, 0.f, 0.f, 0.f};
-      unsigned char* prow = smem + OFF_P + (g * 2 + b) * P_B + r * 128;   // row r of the [128][128 B] P tile
 #pragma unroll
-      for (int c8 = 0; c8 < BN / 8; ++c8) {                     // eight keys = one 16-byte chunk of the row
-        uint32_t pk[4];
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        float t[32];
+        tmem_ld32(tmg + ch * 32, t);
+        tmem_ld_wait();
+        if (masked) mask32(t, k0 + ch * 32);
+        uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float p0 = ex2f(fmaf(a[c8 * 8 + 2 * i], p.scale_log2, -m_use));
-          const float p1 = ex2f(fmaf(a[c8 * 8 + 2 * i + 1], p.scale_log2, -m_use));
-          ps4[i] += p0 + p1;
+        for (int i = 0; i < 16; ++i) {
+          const float p0 = ex2f(fmaf(t[2 * i], p.scale_log2, -m_use));
+          const float p1 = ex2f(fmaf(t[2 * i + 1], p.scale_log2, -m_use));
+          ps4[i & 3] += p0 + p1;
           __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
           pk[i] = *reinterpret_cast<uint32_t*>(&b2);
         }
-        // 16-byte chunk c of row r lives at chunk c ^ (r & 7)
-        *reinterpret_cast<uint4*>(prow + ((c8 ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        tmem_st16(tmg + ch * 16, pk);
       }
       l_row += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor cores
+      tmem_st_wait();
       tc_fence_before();
-      bar_arrive(bar_pfull + (g * 2 + b) * 8);
+      __syncwarp();
+      if ((tid & 31) == 0) bar_arrive(bar_pfull + g * 8);
     }
     if (!fail) {
-      const int vz = n_pass - 1;
-      fail = !bar_wait(bar_pvdone + (g * 2 + (vz & 1)) * 8, (vz >> 1) & 1);
+      fail = !bar_wait(bar_odone + g * 8, 0);
       fail = __any_sync(0xffffffffu, fail);
     }
     if (fail) {
