@@ -178,6 +178,44 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
+// The passes of a CTA in the order they run.  Tiles [low_a, low_b) hold a key that is distant for some row of
+// the CTA: they get a pass with the lowest layer's product (these n_low passes come first).  Of those, tiles
+// [dis_a, dis_b) are distant for every row and get no other pass; every other tile gets a pass with the
+// layer's own product.  mixed: the tile has keys of both kinds, the pass keeps the kind its product is for.
+struct PassMap { int n_low, low_a, low_b, dis_a, dis_b; };
+struct Pass { int j; bool low, mixed; };
+__device__ __forceinline__ Pass pass_of(const PassMap m, int v) {
+  Pass c;
+  if (v < m.n_low) {
+    c.j = m.low_a + v;
+    c.low = true;
+    c.mixed = !(c.j >= m.dis_a && c.j < m.dis_b);
+  } else {
+    const int u = v - m.n_low;
+    c.j = u < m.dis_a ? u : u + (m.dis_b - m.dis_a);
+    c.low = false;
+    c.mixed = c.j >= m.low_a && c.j < m.low_b;
+  }
+  return c;
+}
+// bit i set for i < n
+__device__ __forceinline__ uint32_t low_bits(int n) { return n <= 0 ? 0u : (n >= 32 ? 0xffffffffu : (1u << n) - 1u); }
+// Bit i: the pass keeps key c0 + i for row qi.  Causal and inside the sequence; in a tile with both kinds of
+// key the own product keeps the proximal keys, the lowest layer's the distant ones (S <= key <= qi - W).
+__device__ __forceinline__ uint32_t keep_bits(int c0, int qi, int T, int S, int W, bool mixed, bool low) {
+  uint32_t keep = low_bits(min(qi, T - 1) - c0 + 1);
+  if (mixed) {
+    const uint32_t dist = low_bits(qi - W - c0 + 1) & ~low_bits(S - c0);
+    keep &= low ? dist : ~dist;
+  }
+  return keep;
+}
+// logits of keys the pass does not keep become -inf
+__device__ __forceinline__ void apply_bits(float (&t)[32], uint32_t bits) {
+#pragma unroll
+  for (int i = 0; i < 32; ++i) t[i] = ((bits >> i) & 1u) ? t[i] : -INFINITY;
+}
+
 __global__ void __launch_bounds__(PF_THREADS, 1)
 pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQl,
@@ -190,7 +228,10 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;          // long rows first
   const int hq = blockIdx.y, kvh = hq / (p.H_q / p.H_kv);
   const int q0 = qb * BLK;
-  const bool shares = kvh < 256 && ((p.share_mask[kvh >> 5] >> (kvh & 31)) & 1u);
+  uint32_t share_word = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) share_word = (kvh >> 5) == i ? p.share_mask[i] : share_word;
+  const bool shares = (share_word >> (kvh & 31)) & 1u;
   // mbarriers: Q landed; per ring slot: tile landed, slot free; per group: S ready, P written, O complete
   const uint32_t bar_q = sb + OFF_BAR, bar_full = bar_q + 8, bar_free = bar_q + 48, bar_sfull = bar_q + 88,
                  bar_pfull = bar_q + 104, bar_odone = bar_q + 120;
@@ -222,28 +263,18 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   // keys this CTA needs: positions [0, min(T, q0 + 256)); tile j covers [128 j, 128 j + 128)
   const int k_end = min(p.T, q0 + BLK);
   const int n_tiles = (k_end + BN - 1) / BN;
-  // Tiles [low_a, low_b) hold a key that is distant for some row of the CTA: they get a pass with the lowest
-  // layer's product.  Of those, tiles [dis_a, dis_b) are distant for every row and get no other pass.
-  int low_a = 0, low_b = 0, dis_a = 0, dis_b = 0;
+  PassMap pm{0, 0, 0, 0, 0};
   if (shares) {
-    low_a = p.S / BN;                                           // tiles before it lie inside the sink
+    pm.low_a = p.S / BN;                                        // tiles before it lie inside the sink
     const int e = q0 + BLK - 1 - p.W;                           // the last row's newest distant position
-    low_b = max(low_a, min(e < 0 ? 0 : e / BN + 1, n_tiles));
-    dis_a = (p.S + BN - 1) / BN;
+    pm.low_b = max(pm.low_a, min(e < 0 ? 0 : e / BN + 1, n_tiles));
+    pm.dis_a = (p.S + BN - 1) / BN;
     const int f = q0 - p.W - (BN - 1);                          // tile j is distant for the first row too if 128 j <= f
-    dis_b = max(dis_a, min(f < 0 ? 0 : f / BN + 1, low_b));
+    pm.dis_b = max(pm.dis_a, min(f < 0 ? 0 : f / BN + 1, pm.low_b));
+    pm.n_low = pm.low_b - pm.low_a;
   }
-  const int n_low = low_b - low_a, n_skip = dis_b - dis_a;
-  const int n_pass = n_low + n_tiles - n_skip;
-  struct Pass { int j; bool low, mixed; };
-  auto pass_of = [&](int v) -> Pass {
-    if (v < n_low) {
-      const int j = low_a + v;
-      return Pass{j, true, !(j >= dis_a && j < dis_b)};
-    }
-    const int u = v - n_low, j = u < dis_a ? u : u + n_skip;
-    return Pass{j, false, j >= low_a && j < low_b};
-  };
+  const int n_low = pm.n_low;
+  const int n_pass = n_low + n_tiles - (pm.dis_b - pm.dis_a);
   bool fail = false;
 
   if (loader) {
@@ -268,7 +299,7 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           if (fail) break;
           if (i - NRING == i_switch) { load_q(false); switched = true; }   // both groups' last products with Q_a are done
         }
-        const Pass c = pass_of(i >> 1);
+        const Pass c = pass_of(pm, i >> 1);
         const CUtensorMap* map = (i & 1) ? &tmV : (c.low ? &tmKl : &tmK);
         const uint32_t dst = sb + OFF_RING + slot * KV_B, bar = bar_full + slot * 8;
         bar_expect_tx(bar, KV_B);
@@ -339,7 +370,7 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const uint32_t tmg = tm + g * TM_GROUP + lane_base;
     float m_used = -INFINITY, l_row = 0.f;
     for (int v = 0; v < n_pass; ++v) {
-      const Pass c = pass_of(v);
+      const Pass c = pass_of(pm, v);
       fail = !bar_wait(bar_sfull + g * 8, v & 1);               // S of pass v is complete, and so is every earlier P V
       if (__any_sync(0xffffffffu, fail)) { fail = true; break; }
       tc_fence_after();
@@ -348,29 +379,33 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // diagonal get the causal mask, and a pass over a tile with both kinds of key keeps the kind its
       // product is meant for.
       const bool masked = c.mixed || (k0 + BN - 1 > qg0);
-      auto mask32 = [&](float (&t)[32], int kbase) {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int kj = kbase + i;
-          bool keep = kj <= qi && kj < p.T;
-          if (c.mixed) {
-            const bool prox = kj < p.S || kj > qi - p.W;
-            keep = keep && (prox != c.low);                     // own product: proximal keys; lowest layer's: distant keys
-          }
-          t[i] = keep ? t[i] : -INFINITY;
-        }
-      };
-      // first reading of the row: its maximum
+      // first reading of the row: its maximum.  In a masked tile most pieces of 32 keys are still all kept or
+      // all masked for the 32 rows of a warp (the boundaries move with the row); only the others are decided
+      // key by key, from the row's keep bits.  The masked tiles are few, so their loops stay rolled up and
+      // the code of the common path stays short.
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if (!masked) {
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        float t0[32], t1[32];
-        tmem_ld32(tmg + h * 64, t0);
-        tmem_ld32(tmg + h * 64 + 32, t1);
-        tmem_ld_wait();
-        if (masked) { mask32(t0, k0 + h * 64); mask32(t1, k0 + h * 64 + 32); }
+        for (int h = 0; h < 2; ++h) {
+          float t0[32], t1[32];
+          tmem_ld32(tmg + h * 64, t0);
+          tmem_ld32(tmg + h * 64 + 32, t1);
+          tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(t0[i], t1[i]));
+          for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(t0[i], t1[i]));
+        }
+      } else {
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          const uint32_t kb = keep_bits(k0 + ch * 32, qi, p.T, p.S, p.W, c.mixed, c.low);
+          if (__all_sync(0xffffffffu, kb == 0u)) continue;
+          float t[32];
+          tmem_ld32(tmg + ch * 32, t);
+          tmem_ld_wait();
+          if (!__all_sync(0xffffffffu, kb == 0xffffffffu)) apply_bits(t, kb);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], t[i]);
+        }
       }
       float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       mx *= p.scale_log2;                                       // the scale is positive: it commutes with the maximum
@@ -379,7 +414,7 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       float alpha = 1.f;
       if (raise) { alpha = ex2f(m_used - mx); m_used = mx; }    // ex2(-inf) = 0 on the first tile
       if (__any_sync(0xffffffffu, raise) && v > 0) {            // rescale this warp's rows of O (nothing accumulates now)
-#pragma unroll
+#pragma unroll 1
         for (int ch = 0; ch < PD / 32; ++ch) {
           float t[32];
           tmem_ld32(tmg + TM_O + ch * 32, t);
@@ -394,13 +429,7 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // second reading, 32 keys at a time: P as packed bf16 pairs over columns already consumed
       // (keys 32 c .. 32 c + 31 of S sit in columns 32 c .., their P in columns 16 c .. 16 c + 15)
       float ps4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        float t[32];
-        tmem_ld32(tmg + ch * 32, t);
-        tmem_ld_wait();
-        if (masked) mask32(t, k0 + ch * 32);
-        uint32_t pk[16];
+      auto exp_piece = [&](const float (&t)[32], uint32_t (&pk)[16]) {
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
           const float p0 = ex2f(fmaf(t[2 * i], p.scale_log2, -m_use));
@@ -409,7 +438,34 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
           pk[i] = *reinterpret_cast<uint32_t*>(&b2);
         }
-        tmem_st16(tmg + ch * 16, pk);
+      };
+      if (!masked) {
+#pragma unroll
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          float t[32];
+          uint32_t pk[16];
+          tmem_ld32(tmg + ch * 32, t);
+          tmem_ld_wait();
+          exp_piece(t, pk);
+          tmem_st16(tmg + ch * 16, pk);
+        }
+      } else {
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          const uint32_t kb = keep_bits(k0 + ch * 32, qi, p.T, p.S, p.W, c.mixed, c.low);
+          float t[32];
+          uint32_t pk[16];
+          if (__all_sync(0xffffffffu, kb == 0u)) {               // nothing kept: P = 0
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+          } else {
+            tmem_ld32(tmg + ch * 32, t);
+            tmem_ld_wait();
+            if (!__all_sync(0xffffffffu, kb == 0xffffffffu)) apply_bits(t, kb);
+            exp_piece(t, pk);
+          }
+          tmem_st16(tmg + ch * 16, pk);
+        }
       }
       l_row += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
       tmem_st_wait();
@@ -427,7 +483,7 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       tc_fence_after();
       const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
       uint16_t* dst = p.out + ((int64_t)qi * p.H_q + hq) * PD;
-#pragma unroll
+#pragma unroll 1
       for (int ch = 0; ch < PD / 32; ++ch) {
         float t[32];
         tmem_ld32(tmg + TM_O + ch * 32, t);                     // warp-collective: rows past T load too
