@@ -379,25 +379,59 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // diagonal get the causal mask, and a pass over a tile with both kinds of key keeps the kind its
       // product is meant for.
       const bool masked = c.mixed || (k0 + BN - 1 > qg0);
-      // first reading of the row: its maximum.  In a masked tile most pieces of 32 keys are still all kept or
-      // all masked for the 32 rows of a warp (the boundaries move with the row); only the others are decided
-      // key by key, from the row's keep bits.  The masked tiles are few, so their loops stay rolled up and
-      // the code of the common path stays short.
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      if (!masked) {
+      // Common case (no mask, not the first pass): ONE reading of the row.  The exponentials are taken against
+      // the reference maximum the row already has while the tile's own maximum is found on the side; P stays
+      // in registers until it is known that no row of the warp has to raise its reference, which is nearly
+      // always so (a raise needs a logit 8 log2 units above everything seen before).  S is still intact then,
+      // so the rare other case simply falls through to the general path below.
+      bool done = false;
+      if (!masked && v > 0) {
+        const float m_use = (m_used == -INFINITY) ? 0.f : m_used;
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t pk[BN / 32][16];
+        float ta[32], tb[32];
+        auto piece = [&](const float (&t)[32], uint32_t (&o)[16]) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          float t0[32], t1[32];
-          tmem_ld32(tmg + h * 64, t0);
-          tmem_ld32(tmg + h * 64 + 32, t1);
-          tmem_ld_wait();
+          for (int i = 0; i < 16; ++i) {
+            mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(t[2 * i], t[2 * i + 1]));
+            const float p0 = ex2f(fmaf(t[2 * i], p.scale_log2, -m_use));
+            const float p1 = ex2f(fmaf(t[2 * i + 1], p.scale_log2, -m_use));
+            ps4[i & 3] += p0 + p1;
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+            o[i] = *reinterpret_cast<uint32_t*>(&b2);
+          }
+        };
+        tmem_ld32(tmg, ta);                                     // the next piece is on its way while one is worked on
+        tmem_ld_wait();
+        tmem_ld32(tmg + 32, tb);
+        piece(ta, pk[0]);
+        tmem_ld_wait();
+        tmem_ld32(tmg + 64, ta);
+        piece(tb, pk[1]);
+        tmem_ld_wait();
+        tmem_ld32(tmg + 96, tb);
+        piece(ta, pk[2]);
+        tmem_ld_wait();
+        piece(tb, pk[3]);
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+        const bool raise = mx > m_used + RESCALE_STEP || (m_used == -INFINITY && mx > -INFINITY);
+        if (!__any_sync(0xffffffffu, raise)) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(t0[i], t1[i]));
+          for (int ch = 0; ch < BN / 32; ++ch) tmem_st16(tmg + ch * 16, pk[ch]);
+          l_row += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+          done = true;
         }
-      } else {
+      }
+      if (!done) {
+        // General path, two readings of the row: its maximum first.  In a masked tile most pieces of 32 keys
+        // are still all kept or all masked for the 32 rows of a warp (the boundaries move with the row); only
+        // the others are decided key by key, from the row's keep bits.  These passes are few, so their loops
+        // stay rolled up and the kernel's code stays short.
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
         for (int ch = 0; ch < BN / 32; ++ch) {
-          const uint32_t kb = keep_bits(k0 + ch * 32, qi, p.T, p.S, p.W, c.mixed, c.low);
+          const uint32_t kb = masked ? keep_bits(k0 + ch * 32, qi, p.T, p.S, p.W, c.mixed, c.low) : 0xffffffffu;
           if (__all_sync(0xffffffffu, kb == 0u)) continue;
           float t[32];
           tmem_ld32(tmg + ch * 32, t);
@@ -406,53 +440,31 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
           for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], t[i]);
         }
-      }
-      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      mx *= p.scale_log2;                                       // the scale is positive: it commutes with the maximum
-      // raise the row's reference maximum only when the tile exceeds it by more than RESCALE_STEP
-      const bool raise = mx > m_used + RESCALE_STEP || (m_used == -INFINITY && mx > -INFINITY);
-      float alpha = 1.f;
-      if (raise) { alpha = ex2f(m_used - mx); m_used = mx; }    // ex2(-inf) = 0 on the first tile
-      if (__any_sync(0xffffffffu, raise) && v > 0) {            // rescale this warp's rows of O (nothing accumulates now)
+        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        mx *= p.scale_log2;                                     // the scale is positive: it commutes with the maximum
+        // raise the row's reference maximum only when the tile exceeds it by more than RESCALE_STEP
+        const bool raise = mx > m_used + RESCALE_STEP || (m_used == -INFINITY && mx > -INFINITY);
+        float alpha = 1.f;
+        if (raise) { alpha = ex2f(m_used - mx); m_used = mx; }  // ex2(-inf) = 0 on the first tile
+        if (__any_sync(0xffffffffu, raise) && v > 0) {          // rescale this warp's rows of O (nothing accumulates now)
 #pragma unroll 1
-        for (int ch = 0; ch < PD / 32; ++ch) {
-          float t[32];
-          tmem_ld32(tmg + TM_O + ch * 32, t);
-          tmem_ld_wait();
+          for (int ch = 0; ch < PD / 32; ++ch) {
+            float t[32];
+            tmem_ld32(tmg + TM_O + ch * 32, t);
+            tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) t[i] *= alpha;
-          tmem_st32(tmg + TM_O + ch * 32, t);
+            for (int i = 0; i < 32; ++i) t[i] *= alpha;
+            tmem_st32(tmg + TM_O + ch * 32, t);
+          }
         }
-      }
-      l_row *= alpha;
-      const float m_use = (m_used == -INFINITY) ? 0.f : m_used;
-      // second reading, 32 keys at a time: P as packed bf16 pairs over columns already consumed
-      // (keys 32 c .. 32 c + 31 of S sit in columns 32 c .., their P in columns 16 c .. 16 c + 15)
-      float ps4[4] = {0.f, 0.f, 0.f, 0.f};
-      auto exp_piece = [&](const float (&t)[32], uint32_t (&pk)[16]) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float p0 = ex2f(fmaf(t[2 * i], p.scale_log2, -m_use));
-          const float p1 = ex2f(fmaf(t[2 * i + 1], p.scale_log2, -m_use));
-          ps4[i & 3] += p0 + p1;
-          __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-          pk[i] = *reinterpret_cast<uint32_t*>(&b2);
-        }
-      };
-      if (!masked) {
-#pragma unroll
-        for (int ch = 0; ch < BN / 32; ++ch) {
-          float t[32];
-          uint32_t pk[16];
-          tmem_ld32(tmg + ch * 32, t);
-          tmem_ld_wait();
-          exp_piece(t, pk);
-          tmem_st16(tmg + ch * 16, pk);
-        }
-      } else {
+        l_row *= alpha;
+        const float m_use = (m_used == -INFINITY) ? 0.f : m_used;
+        // second reading, 32 keys at a time: P as packed bf16 pairs over columns already consumed
+        // (keys 32 c .. 32 c + 31 of S sit in columns 32 c .., their P in columns 16 c .. 16 c + 15)
+        float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
         for (int ch = 0; ch < BN / 32; ++ch) {
-          const uint32_t kb = keep_bits(k0 + ch * 32, qi, p.T, p.S, p.W, c.mixed, c.low);
+          const uint32_t kb = masked ? keep_bits(k0 + ch * 32, qi, p.T, p.S, p.W, c.mixed, c.low) : 0xffffffffu;
           float t[32];
           uint32_t pk[16];
           if (__all_sync(0xffffffffu, kb == 0u)) {               // nothing kept: P = 0
@@ -462,12 +474,19 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             tmem_ld32(tmg + ch * 32, t);
             tmem_ld_wait();
             if (!__all_sync(0xffffffffu, kb == 0xffffffffu)) apply_bits(t, kb);
-            exp_piece(t, pk);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float p0 = ex2f(fmaf(t[2 * i], p.scale_log2, -m_use));
+              const float p1 = ex2f(fmaf(t[2 * i + 1], p.scale_log2, -m_use));
+              ps4[i & 3] += p0 + p1;
+              __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+              pk[i] = *reinterpret_cast<uint32_t*>(&b2);
+            }
           }
           tmem_st16(tmg + ch * 16, pk);
         }
+        l_row += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
       }
-      l_row += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();

@@ -100,6 +100,34 @@ def test_prefill_matches_decode_steps():
     assert cache.device_status() == B.POD_OK and B.pod_prefill_status() == B.POD_OK
 
 
+@pytest.mark.parametrize("T,S,W", [(8192, 16, 2048), (5000, 0, 1000)])
+def test_prefill_long_sequence_sampled_rows(T, S, W):
+    """A sequence of many query blocks and key tiles (the ring of K/V slots wraps many times, the passes
+    with the lowest layer's product are most of the work, Q is exchanged between the two kinds of pass):
+    both layers of a block, checked on sampled positions that the oracle computes one by one -- the first
+    rows, rows around every boundary of a 256-row block in the middle, rows whose window edge or sink edge
+    falls inside a tile, and the last rows."""
+    Hq, Hkv = 8, 2
+    q, kv = _inputs(34, T, Hq, Hkv, outliers=True)
+    Q = [q(l) for l in range(2)]
+    K = [kv(synth.TAG_K, l) for l in range(2)]
+    V = [kv(synth.TAG_V, l) for l in range(2)]
+    outs = [torch.zeros(T, Hq, 128, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    B.pod_prefill_attn(Q[0], K[0], V[0], outs[0], n_sink=S, n_recent=W)
+    B.pod_prefill_attn(Q[1], K[1], V[1], outs[1], n_sink=S, n_recent=W, q_low=Q[0], k_low=K[0])
+    torch.cuda.synchronize()
+    assert B.pod_prefill_status() == B.POD_OK
+    rows = sorted({0, 1, S, S + 1, W - 1, W, W + S - 1, W + S, W + S + 1, W + S + 127, W + S + 128, 2047, 2048, 2303, 2304,
+                   T // 2 - 1, T // 2, T // 2 + 127, T // 2 + 128, T // 2 + 255, T // 2 + 256, T - 257, T - 256, T - 129,
+                   T - 128, T - 2, T - 1} & set(range(T)))
+    f = lambda xs: np.stack([x.double().cpu().numpy() for x in xs])
+    Qn, Kn, Vn = f(Q), f(K), f(V)
+    for l in range(2):
+        ref = np.stack([O.pod_decode_layer(Qn[:, i], Kn[:, :i + 1], Vn[:, :i + 1], l, group_size=2, n_s=S, n_r=W)
+                        for i in rows])
+        _check(outs[l][rows], ref, f"T={T} layer {l} rows {rows[0]}..{rows[-1]}", V[l])
+
+
 def test_prefill_rejects_bad_arguments():
     x = torch.zeros(4, 2, 128, dtype=torch.bfloat16, device="cuda")
     y = torch.zeros(4, 2, 64, dtype=torch.bfloat16, device="cuda")
