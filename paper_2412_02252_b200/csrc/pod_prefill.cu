@@ -329,7 +329,12 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           umma(tm + g * TM_GROUP, dq + (uint64_t)(a_off >> 4), dk + (uint64_t)(b_off >> 4), IDESC, ks > 0);
         }
         umma_commit(bar_sfull + g * 8);
-        if (g == NG - 1) umma_commit(bar_free + ((2 * v) % NRING) * 8);   // both groups are done with this K tile
+        // A tcgen05.commit in the middle of a run of products costs the pipe a few hundred cycles, one that
+        // follows another commit much less: the ring slots are handed back here, next to the commit above.
+        if (g == NG - 1) {
+          umma_commit(bar_free + ((2 * v) % NRING) * 8);        // both groups are done with this K tile,
+          if (v > 0) umma_commit(bar_free + ((2 * v - 1) % NRING) * 8);   // and with V of the pass before
+        }
       };
       auto wait_k = [&](int v) -> bool {                        // K of pass v (and the Q it goes with) has landed
         if (v == 0 && !bar_wait(bar_q, 0)) return false;
@@ -355,7 +360,6 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           for (int ks = 0; ks < BN / 16; ++ks)                  // 16 keys per step; O accumulates over the passes
             umma_ts(tm + g * TM_GROUP + TM_O, tm + g * TM_GROUP + ks * 8, dv + (uint64_t)(ks * (2048 >> 4)), IDESC_O,
                     (v > 0 || ks > 0) ? 1u : 0u);
-          if (g == NG - 1) umma_commit(bar_free + (iv % NRING) * 8);      // both groups are done with this V tile
           if (v + 1 < n_pass) issue_qk(g, v + 1);               // overwrites P[g]: in order behind the P V just issued
           else umma_commit(bar_odone + g * 8);
         }
