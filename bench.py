@@ -262,6 +262,9 @@ def run_ours(args):
         assert B.pod_prefill_status() == 0
         out["tokens"] = T_
         out["peak_tflops"] = _bf16_peak()
+        out["roofline"] = {"bound": "tensor", "achieved": out["lowest_layer"]["tflops"], "peak": out["peak_tflops"],
+                           "unit": "TFLOP/s", "frac": round(out["lowest_layer"]["tflops"] / out["peak_tflops"], 4),
+                           "frac_sharing_layer": round(out["sharing_layer"]["tflops"] / out["peak_tflops"], 4)}
         out["note"] = "causal FLOPs (2 products x 2 d per visible pair) over the mean of back-to-back calls; peak = measured cuBLAS bf16 burst"
         return out
 

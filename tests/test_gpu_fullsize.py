@@ -110,3 +110,36 @@ def test_config5_ragged_serving_mix():
     live, dense = O.pod_cache_bytes([n + steps for n in lens0], n_layers=32, n_kv_heads=8, head_dim=128,
                                     group_size=2, n_s=16, n_r=2048)
     assert cache.bytes(B.POD_BYTES_LIVE) == live and cache.bytes(B.POD_BYTES_DENSE_EQUIV) == dense
+
+
+def test_prefill_attention_32k_sampled():
+    """pod_prefill_attn at the size bench.py times (32768 positions, 32/8 heads, S = 16, W = 2048, outlier
+    channels): both layers of a block; the oracle recomputes sampled (position, KV head) outputs one by one
+    as decode steps on the prefix (all four query heads of the KV head)."""
+    from oracle import pod_oracle as O
+    T, Hq, Hkv, d, S, W, seed = 32768, 32, 8, 128, 16, 2048, 2
+    gen = lambda tag, layer, h, outl: synth.gen_kv(seed, tag, layer, 0, 0, T, h, d, outliers=outl, device="cuda")
+    Q = [gen(synth.TAG_Q, l, Hq, False) for l in range(2)]
+    K = [gen(synth.TAG_K, l, Hkv, True) for l in range(2)]
+    V = [gen(synth.TAG_V, l, Hkv, True) for l in range(2)]
+    outs = [torch.zeros(T, Hq, d, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    B.pod_prefill_attn(Q[0], K[0], V[0], outs[0], n_sink=S, n_recent=W)
+    B.pod_prefill_attn(Q[1], K[1], V[1], outs[1], n_sink=S, n_recent=W, q_low=Q[0], k_low=K[0])
+    torch.cuda.synchronize()
+    assert B.pod_prefill_status() == B.POD_OK
+    assert all(torch.isfinite(o.float()).all() for o in outs)
+    r = Hq // Hkv
+    samples = [(0, 0), (17, 3), (2063, 1), (2064, 1), (2065, 6), (4095, 2), (4096, 2), (12345, 7), (16383, 0), (16384, 5),
+               (20000, 4), (32511, 3), (32512, 3), (32639, 6), (32640, 6), (32767, 0), (32767, 7)]
+    for (i, kh) in samples:
+        f = lambda xs, hs: np.stack([x[:i + 1, hs].double().cpu().numpy() for x in xs])
+        Kn, Vn = f(K, slice(kh, kh + 1)), f(V, slice(kh, kh + 1))
+        qn = np.stack([x[i, kh * r:(kh + 1) * r].double().cpu().numpy() for x in Q])
+        vmax = np.abs(Vn).max(axis=(1, 2))                                   # [L][d]
+        for l in range(2):
+            ref = O.pod_decode_layer(qn, Kn, Vn, l, group_size=2, n_s=S, n_r=W)   # [r][d]
+            got = outs[l][i, kh * r:(kh + 1) * r].double().cpu().numpy()
+            err = np.abs(got - ref)
+            bound = 1e-2 + 2.0 ** -8 * vmax[l][None]                          # as in test_gpu_prefill.py
+            rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+            assert (err <= bound).all() and rel <= 5e-3, (i, kh, l, err.max(), rel)
