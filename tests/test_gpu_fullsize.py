@@ -112,12 +112,19 @@ def test_config5_ragged_serving_mix():
     assert cache.bytes(B.POD_BYTES_LIVE) == live and cache.bytes(B.POD_BYTES_DENSE_EQUIV) == dense
 
 
-def test_prefill_attention_32k_sampled():
+@pytest.mark.parametrize("T,W,samples", [
+    (32768, 2048, [(0, 0), (17, 3), (2063, 1), (2064, 1), (2065, 6), (4095, 2), (4096, 2), (12345, 7), (16383, 0), (16384, 5),
+                   (20000, 4), (32511, 3), (32512, 3), (32639, 6), (32640, 6), (32767, 0), (32767, 7)]),
+    (131072, 4096, [(4111, 2), (4112, 2), (65535, 0), (65536, 7), (100000, 4), (130815, 1), (130816, 1), (131071, 5)])])
+def test_prefill_attention_sampled(T, W, samples):
     """pod_prefill_attn at the size bench.py times (32768 positions, 32/8 heads, S = 16, W = 2048, outlier
-    channels): both layers of a block; the oracle recomputes sampled (position, KV head) outputs one by one
-    as decode steps on the prefix (all four query heads of the KV head)."""
+    channels) and at the longest context of the configurations (131072 positions, W = 4096): both layers of a
+    block; the oracle recomputes sampled (position, KV head) outputs one by one as decode steps on the prefix
+    (all four query heads of the KV head)."""
+    if T > 65536 and _free_gb() < 12:
+        pytest.skip("needs 12 GiB of free device memory")
     from oracle import pod_oracle as O
-    T, Hq, Hkv, d, S, W, seed = 32768, 32, 8, 128, 16, 2048, 2
+    Hq, Hkv, d, S, seed = 32, 8, 128, 16, 2
     gen = lambda tag, layer, h, outl: synth.gen_kv(seed, tag, layer, 0, 0, T, h, d, outliers=outl, device="cuda")
     Q = [gen(synth.TAG_Q, l, Hq, False) for l in range(2)]
     K = [gen(synth.TAG_K, l, Hkv, True) for l in range(2)]
@@ -129,8 +136,6 @@ def test_prefill_attention_32k_sampled():
     assert B.pod_prefill_status() == B.POD_OK
     assert all(torch.isfinite(o.float()).all() for o in outs)
     r = Hq // Hkv
-    samples = [(0, 0), (17, 3), (2063, 1), (2064, 1), (2065, 6), (4095, 2), (4096, 2), (12345, 7), (16383, 0), (16384, 5),
-               (20000, 4), (32511, 3), (32512, 3), (32639, 6), (32640, 6), (32767, 0), (32767, 7)]
     for (i, kh) in samples:
         f = lambda xs, hs: np.stack([x[:i + 1, hs].double().cpu().numpy() for x in xs])
         Kn, Vn = f(K, slice(kh, kh + 1)), f(V, slice(kh, kh + 1))
