@@ -232,13 +232,15 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
   for (int i = 0; i < 8; ++i) share_word = (kvh >> 5) == i ? p.share_mask[i] : share_word;
   const bool shares = (share_word >> (kvh & 31)) & 1u;
-  // mbarriers: Q landed; per ring slot: tile landed, slot free; per group: S ready, P written, O complete
+  // mbarriers: Q landed; per ring slot: tile landed, slot free; per group: S ready, P written, O complete;
+  // the lowest layer's Q no longer needed
   const uint32_t bar_q = sb + OFF_BAR, bar_full = bar_q + 8, bar_free = bar_q + 48, bar_sfull = bar_q + 88,
-                 bar_pfull = bar_q + 104, bar_odone = bar_q + 120;
+                 bar_pfull = bar_q + 104, bar_odone = bar_q + 120, bar_qfree = bar_q + 136;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 192);
 
   if (tid == 0) {
     bar_init(bar_q, 1);
+    bar_init(bar_qfree, 1);
     for (int i = 0; i < NRING; ++i) {
       bar_init(bar_full + i * 8, 1);
       bar_init(bar_free + i * 8, 1);
@@ -294,10 +296,15 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       bool switched = n_low == 0;
       for (int i = 0; i < n_loads && !fail; ++i) {
         const int slot = i % NRING;
-        if (i >= NRING) {                                       // the slot's previous tile (load i - 5) has been used
-          fail = !bar_wait(bar_free + slot * 8, ((i / NRING) - 1) & 1);
+        if (i >= NRING) {
+          if (i - NRING == i_switch) {                          // both groups' last products with Q_a are done
+            fail = !bar_wait(bar_qfree, 0);
+            if (fail) break;
+            load_q(false);
+            switched = true;
+          }
+          fail = !bar_wait(bar_free + slot * 8, ((i / NRING) - 1) & 1);   // the slot's previous tile (load i - 5) has been used
           if (fail) break;
-          if (i - NRING == i_switch) { load_q(false); switched = true; }   // both groups' last products with Q_a are done
         }
         const Pass c = pass_of(pm, i >> 1);
         const CUtensorMap* map = (i & 1) ? &tmV : (c.low ? &tmKl : &tmK);
@@ -307,7 +314,7 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int h = 0; h < 2; ++h) tma_load_3d(dst + h * (KV_B / 2), map, h * 64, kvh, c.j * BN, bar);
       }
       if (!fail && !switched) {                                 // the ring never came back to that slot
-        fail = !bar_wait(bar_free + (i_switch % NRING) * 8, (i_switch / NRING) & 1);
+        fail = !bar_wait(bar_qfree, 0);
         if (!fail) load_q(false);
       }
       if (fail) atomicExch(p.err_flag, 1);
@@ -330,10 +337,11 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         umma_commit(bar_sfull + g * 8);
         // A tcgen05.commit in the middle of a run of products costs the pipe a few hundred cycles, one that
-        // follows another commit much less: the ring slots are handed back here, next to the commit above.
+        // follows another commit less: V of the pass before is handed back here, next to the commit above
+        // (both groups are done with it), and K without a commit at all (see the wait for P below).
         if (g == NG - 1) {
-          umma_commit(bar_free + ((2 * v) % NRING) * 8);        // both groups are done with this K tile,
-          if (v > 0) umma_commit(bar_free + ((2 * v - 1) % NRING) * 8);   // and with V of the pass before
+          if (v > 0) umma_commit(bar_free + ((2 * v - 1) % NRING) * 8);
+          if (v + 1 == n_low) umma_commit(bar_qfree);           // the last products that read the lowest layer's Q
         }
       };
       auto wait_k = [&](int v) -> bool {                        // K of pass v (and the Q it goes with) has landed
@@ -355,6 +363,9 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int g = 0; g < NG && !fail; ++g) {
           fail = !bar_wait(bar_pfull + g * 8, v & 1);           // P[g] of pass v is written
           if (fail) break;
+          // ... so S[g] of pass v was complete: once that is true of the last group, every product that read
+          // K of pass v is done and its slot goes back with a plain arrival (its next tile is not due soon)
+          if (g == NG - 1) bar_arrive(bar_free + ((2 * v) % NRING) * 8);
           tc_fence_after();
 #pragma unroll
           for (int ks = 0; ks < BN / 16; ++ks)                  // 16 keys per step; O accumulates over the passes
