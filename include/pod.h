@@ -218,7 +218,7 @@ const char* pod_strerror(int status);
  * of the head's block.  out[i][h] = one softmax over both groups applied to v.  It is what
  * pod_decode_attn returns at each step of a sequence fed token by token.
  *   q, q_low, out : device bf16 [n_tokens][n_q_heads][head_dim];  k, k_low, v : device bf16
- *                   [n_tokens][n_kv_heads][head_dim]; head_dim must be 128.
+ *                   [n_tokens][n_kv_heads][head_dim]; head_dim 64 or 128.
  *   q_low, k_low  : NULL for a layer that is the lowest of every head's block (ordinary causal attention).
  *   head_shares   : host int32 [n_kv_heads] or NULL; with q_low given, KV head h takes its distant logits
  *                   from q_low / k_low if head_shares is NULL or head_shares[h] != 0 (head-wise blocks).

@@ -208,8 +208,8 @@ class PodCache:
 
 def pod_prefill_attn(q, k, v, out, *, n_sink: int, n_recent: int, q_low=None, k_low=None, head_shares=None,
                      sm_scale: float = 0.0, stream: int = 0) -> int:
-    """PoD attention for every position (prefill) from dense bf16 projections ``q`` [T][H_q][128],
-    ``k``, ``v`` [T][H_kv][128]; ``q_low``/``k_low``: the lowest layer's, for layers that share."""
+    """PoD attention for every position (prefill) from dense bf16 projections ``q`` [T][H_q][d] (d 64 or 128),
+    ``k``, ``v`` [T][H_kv][d]; ``q_low``/``k_low``: the lowest layer's, for layers that share."""
     T, Hq, d = q.shape
     Hkv = k.shape[1]
     hs = None if head_shares is None else (c_int32 * Hkv)(*[int(x) for x in head_shares])

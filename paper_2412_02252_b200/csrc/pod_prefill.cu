@@ -43,7 +43,6 @@
 namespace pod {
 namespace {
 
-constexpr int PD = 128;                 // head_dim
 constexpr int BM = 128;                 // query rows per softmax group
 constexpr int NG = 2;                   // softmax groups per CTA
 constexpr int BLK = NG * BM;            // query rows per CTA
@@ -51,12 +50,16 @@ constexpr int BN = 128;                 // keys per tile
 constexpr int NRING = 5;                // slots of the K/V ring
 constexpr uint32_t PF_WAIT_LIMIT = 1u << 22;
 
-constexpr int Q_B = BM * PD * 2;        // 32 KiB: two [128][128 B] sub-tiles
-constexpr int KV_B = BN * PD * 2;       // 32 KiB: two [128][128 B] sub-tiles
-constexpr int OFF_Q = 0;                // per group: Q of the lowest layer, later Q of this layer
-constexpr int OFF_RING = NG * Q_B;
-constexpr int OFF_BAR = OFF_RING + NRING * KV_B;
-constexpr int PF_SMEM = OFF_BAR + 256 + 1024;
+constexpr int Q_SUB = BM * 128, KV_SUB = BN * 128;   // one [rows][128 B] sub-tile: 64 channels of every row
+// shared-memory plan for head_dim PD (64 or 128): one or two sub-tiles per operand tile
+template <int PD> struct Plan {
+  static constexpr int Q_B = BM * PD * 2;        // 32 KiB at d = 128
+  static constexpr int KV_B = BN * PD * 2;       // 32 KiB at d = 128
+  static constexpr int OFF_Q = 0;                // per group: Q of the lowest layer, later Q of this layer
+  static constexpr int OFF_RING = NG * Q_B;
+  static constexpr int OFF_BAR = OFF_RING + NRING * KV_B;
+  static constexpr int SMEM = OFF_BAR + 256 + 1024;
+};
 constexpr int PF_THREADS = BLK + 64;    // eight softmax warps, the tensor-core warp, the load warp
 constexpr int TM_COLS = 512;            // per group S / P 128 + O 128 fp32 columns
 constexpr int TM_GROUP = 256, TM_O = 128;
@@ -216,10 +219,13 @@ __device__ __forceinline__ void apply_bits(float (&t)[32], uint32_t bits) {
   for (int i = 0; i < 32; ++i) t[i] = ((bits >> i) & 1u) ? t[i] : -INFINITY;
 }
 
+template <int PD>
 __global__ void __launch_bounds__(PF_THREADS, 1)
 pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQl,
                    const __grid_constant__ CUtensorMap tmKl, const PrefillParams p) {
+  constexpr int Q_B = Plan<PD>::Q_B, KV_B = Plan<PD>::KV_B, OFF_Q = Plan<PD>::OFF_Q, OFF_RING = Plan<PD>::OFF_RING,
+                OFF_BAR = Plan<PD>::OFF_BAR;
   extern __shared__ unsigned char pf_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pf_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sb = s2u(smem);
@@ -287,8 +293,8 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
         for (int g = 0; g < NG; ++g)
 #pragma unroll
-          for (int h = 0; h < 2; ++h)
-            tma_load_3d(sb + OFF_Q + g * Q_B + h * (Q_B / 2), low ? &tmQl : &tmQ, h * 64, hq, q0 + g * BM, bar_q);
+          for (int h = 0; h < PD / 64; ++h)
+            tma_load_3d(sb + OFF_Q + g * Q_B + h * Q_SUB, low ? &tmQl : &tmQ, h * 64, hq, q0 + g * BM, bar_q);
       };
       load_q(n_low > 0);
       const int n_loads = 2 * n_pass;
@@ -311,7 +317,7 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const uint32_t dst = sb + OFF_RING + slot * KV_B, bar = bar_full + slot * 8;
         bar_expect_tx(bar, KV_B);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) tma_load_3d(dst + h * (KV_B / 2), map, h * 64, kvh, c.j * BN, bar);
+        for (int h = 0; h < PD / 64; ++h) tma_load_3d(dst + h * KV_SUB, map, h * 64, kvh, c.j * BN, bar);
       }
       if (!fail && !switched) {                                 // the ring never came back to that slot
         fail = !bar_wait(bar_qfree, 0);
@@ -326,13 +332,13 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // Descriptors of the operands' first steps, built once: a later step or slot only adds its byte offset
       // / 16 to the address field (shared-memory addresses stay below 2^18, so the field never carries).
       const uint64_t dq0 = smem_desc(sb + OFF_Q, 16, 1024), dk0 = smem_desc(sb + OFF_RING, 16, 1024);
-      const uint64_t dv0 = smem_desc(sb + OFF_RING, KV_B / 2, 1024);
+      const uint64_t dv0 = smem_desc(sb + OFF_RING, KV_SUB, 1024);
       auto issue_qk = [&](int g, int v) {                       // S[g] = Q_g K^T of pass v
         const uint64_t dk = dk0 + (uint64_t)(((2 * v) % NRING) * (KV_B >> 4));
         const uint64_t dq = dq0 + (uint64_t)(g * (Q_B >> 4));
 #pragma unroll
         for (int ks = 0; ks < PD / 16; ++ks) {                  // 16 channels per step: 4 per 128-byte sub-tile
-          const uint32_t a_off = (ks >> 2) * (Q_B / 2) + (ks & 3) * 32, b_off = (ks >> 2) * (KV_B / 2) + (ks & 3) * 32;
+          const uint32_t a_off = (ks >> 2) * Q_SUB + (ks & 3) * 32, b_off = (ks >> 2) * KV_SUB + (ks & 3) * 32;
           umma(tm + g * TM_GROUP, dq + (uint64_t)(a_off >> 4), dk + (uint64_t)(b_off >> 4), IDESC, ks > 0);
         }
         umma_commit(bar_sfull + g * 8);
@@ -554,7 +560,7 @@ struct PrefillSetup {
 PrefillSetup g_pf[64];
 std::mutex g_pf_mutex;
 
-bool encode_3d(PFN_cuTensorMapEncodeTiled_v12000 enc, CUtensorMap* tm, const void* base, int T, int H, int rows) {
+bool encode_3d(PFN_cuTensorMapEncodeTiled_v12000 enc, CUtensorMap* tm, const void* base, int T, int H, int rows, int PD) {
   cuuint64_t dims[3] = {(cuuint64_t)PD, (cuuint64_t)H, (cuuint64_t)T};
   cuuint64_t strides[2] = {(cuuint64_t)PD * 2, (cuuint64_t)H * PD * 2};
   cuuint32_t box[3] = {64u, 1u, (cuuint32_t)rows};
@@ -573,7 +579,7 @@ extern "C" int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int
                                 float sm_scale, const void* q, const void* k, const void* v, const void* q_low,
                                 const void* k_low, const int32_t* head_shares, void* out, void* cuda_stream) {
   if (!q || !k || !v || !out) return POD_ERR_INVALID;
-  if (head_dim != PD || n_tokens < 1 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads != 0) return POD_ERR_INVALID;
+  if ((head_dim != 64 && head_dim != 128) || n_tokens < 1 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads != 0) return POD_ERR_INVALID;
   if (n_sink < 0 || n_recent < 1 || !(sm_scale >= 0.f) || isinf(sm_scale)) return POD_ERR_INVALID;
   if (n_q_heads > 65535) return POD_ERR_INVALID;
   if ((q_low == nullptr) != (k_low == nullptr)) return POD_ERR_INVALID;
@@ -591,7 +597,8 @@ extern "C" int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int
           qres != cudaDriverEntryPointSuccess || fn == nullptr)
         return POD_ERR_CUDA;
       if (cudaMalloc(&su->err, 4) != cudaSuccess || cudaMemset(su->err, 0, 4) != cudaSuccess) return POD_ERR_CUDA;
-      if (cudaFuncSetAttribute(pod_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM) != cudaSuccess)
+      if (cudaFuncSetAttribute(pod_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<128>::SMEM) != cudaSuccess ||
+          cudaFuncSetAttribute(pod_prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<64>::SMEM) != cudaSuccess)
         return POD_ERR_CUDA;
       su->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
       su->ready = true;
@@ -608,12 +615,15 @@ extern "C" int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int
   CUtensorMap tq, tk, tv, tql, tkl;
   const void* ql = q_low ? q_low : q;
   const void* kl = k_low ? k_low : k;
-  if (!encode_3d(su->encode, &tq, q, n_tokens, n_q_heads, BM) || !encode_3d(su->encode, &tk, k, n_tokens, n_kv_heads, BN) ||
-      !encode_3d(su->encode, &tv, v, n_tokens, n_kv_heads, BN) || !encode_3d(su->encode, &tql, ql, n_tokens, n_q_heads, BM) ||
-      !encode_3d(su->encode, &tkl, kl, n_tokens, n_kv_heads, BN))
+  if (!encode_3d(su->encode, &tq, q, n_tokens, n_q_heads, BM, head_dim) || !encode_3d(su->encode, &tk, k, n_tokens, n_kv_heads, BN, head_dim) ||
+      !encode_3d(su->encode, &tv, v, n_tokens, n_kv_heads, BN, head_dim) || !encode_3d(su->encode, &tql, ql, n_tokens, n_q_heads, BM, head_dim) ||
+      !encode_3d(su->encode, &tkl, kl, n_tokens, n_kv_heads, BN, head_dim))
     return POD_ERR_INVALID;
   dim3 grid((n_tokens + BLK - 1) / BLK, n_q_heads);
-  pod_prefill_kernel<<<grid, PF_THREADS, PF_SMEM, static_cast<cudaStream_t>(cuda_stream)>>>(tq, tk, tv, tql, tkl, p);
+  if (head_dim == 128)
+    pod_prefill_kernel<128><<<grid, PF_THREADS, Plan<128>::SMEM, static_cast<cudaStream_t>(cuda_stream)>>>(tq, tk, tv, tql, tkl, p);
+  else
+    pod_prefill_kernel<64><<<grid, PF_THREADS, Plan<64>::SMEM, static_cast<cudaStream_t>(cuda_stream)>>>(tq, tk, tv, tql, tkl, p);
   return cudaGetLastError() == cudaSuccess ? POD_OK : POD_ERR_CUDA;
 }
 

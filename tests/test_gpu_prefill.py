@@ -128,11 +128,30 @@ def test_prefill_long_sequence_sampled_rows(T, S, W):
         _check(outs[l][rows], ref, f"T={T} layer {l} rows {rows[0]}..{rows[-1]}", V[l])
 
 
+@pytest.mark.parametrize("T,S,W", [(5, 4, 32), (300, 4, 32), (1000, 16, 200)])
+def test_prefill_head_dim_64(T, S, W):
+    """Heads of 64 channels (one 128-byte sub-tile per operand row): a lowest layer and a sharing layer."""
+    Hq, Hkv, d = 8, 2, 64
+    q, kv = _inputs(35, T, Hq, Hkv, d=d, outliers=True)
+    Q = [q(l) for l in range(2)]
+    K = [kv(synth.TAG_K, l) for l in range(2)]
+    V = [kv(synth.TAG_V, l) for l in range(2)]
+    outs = [torch.zeros(T, Hq, d, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    B.pod_prefill_attn(Q[0], K[0], V[0], outs[0], n_sink=S, n_recent=W)
+    B.pod_prefill_attn(Q[1], K[1], V[1], outs[1], n_sink=S, n_recent=W, q_low=Q[0], k_low=K[0])
+    torch.cuda.synchronize()
+    assert B.pod_prefill_status() == B.POD_OK
+    f = lambda xs: np.stack([x.double().cpu().numpy() for x in xs])
+    for l in range(2):
+        ref = O.pod_prefill_layer(f(Q), f(K), f(V), l, group_size=2, n_s=S, n_r=W)
+        _check(outs[l], ref, f"d=64 T={T} layer {l}", V[l])
+
+
 def test_prefill_rejects_bad_arguments():
     x = torch.zeros(4, 2, 128, dtype=torch.bfloat16, device="cuda")
-    y = torch.zeros(4, 2, 64, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(4, 2, 32, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(B.PodError):
-        B.pod_prefill_attn(y, y, y, y, n_sink=1, n_recent=1)                    # head_dim 64
+        B.pod_prefill_attn(y, y, y, y, n_sink=1, n_recent=1)                    # head_dim 32
     with pytest.raises(B.PodError):
         B.pod_prefill_attn(x, x, x, x, n_sink=1, n_recent=0)
     with pytest.raises(B.PodError):
