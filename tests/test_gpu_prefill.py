@@ -53,7 +53,9 @@ def test_prefill_lowest_layer_is_causal_attention(T, S, W):
 
 
 @pytest.mark.parametrize("T,S,W,shares", [(300, 4, 32, None), (700, 16, 200, None), (1000, 4, 300, [1, 0]),
-                                          (450, 0, 64, [0, 1]), (200, 130, 10, None), (90, 4, 200, None)])
+                                          (450, 0, 64, [0, 1]), (200, 130, 10, None), (90, 4, 200, None),
+                                          (600, 300, 1, None), (257, 0, 1, None), (256, 128, 128, [1, 1]), (1, 0, 1, None),
+                                          (640, 256, 127, None)])
 def test_prefill_sharing_layer(T, S, W, shares):
     """A layer whose distant logits come from the block's lowest layer (all heads, or some: head-wise
     blocks); windows that cross tile boundaries, a sink longer than a tile, a window longer than the
