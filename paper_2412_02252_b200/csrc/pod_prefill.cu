@@ -5,7 +5,8 @@
 // Position i attends to positions j <= i.  Of those the first n_s and the last n_r are proximal:
 // their logits are q_l[i] . k_l[j]; the others are distant: their logits are q_a[i] . k_a[j] with a
 // the lowest layer of the head's block (for a head whose block starts at this layer both are the
-// same product).  One softmax over both groups weighs layer l's own values.
+// same product).  One softmax over both groups weighs layer l's own values.  head_dim is 128 or 64 (a template
+// parameter; sizes in these comments are for 128).
 //
 // One CTA = 256 consecutive query positions of one query head: two softmax groups of four warps (group g
 // owns rows 128 g .. 128 g + 127, one thread per row), one warp whose lane 0 issues every tcgen05.mma and
@@ -20,8 +21,9 @@
 // and the other passes follow.  Per pass v and group g, in tensor memory (per group 128 columns for S and
 // P, 128 for O):
 //   S[128 x 128] = Q K^T  or  Q_a K_a^T      (M = 128, N = 128, K = 16 x 8 steps)
-//   each softmax thread reads its row of S (tcgen05.ld) for the maximum, reads it again in four pieces and
-//   writes P = 2^(logit - m) as packed bf16 over the columns of S it has already consumed (tcgen05.st)
+//   each softmax thread reads its row of S in four pieces (tcgen05.ld), takes P = 2^(logit - m) against the
+//   row's current reference m, and writes it as packed bf16 over the columns of S it has consumed (tcgen05.st);
+//   a first pass, a masked tile or a raise of m reads the row twice (maximum first)
 //   O[128 x 128] += P V                       (A = P from tensor memory, B = V MN-major, K = 16 x 8).
 // The tensor-core thread alternates between the groups (P V of group g, then its next Q K^T), so one group's
 // products run while the other group is in its softmax.  The reference maximum m of a row is only raised
@@ -69,7 +71,7 @@ struct PrefillParams {
   int32_t T, H_q, H_kv, S, W;
   float scale_log2;
   uint32_t share_mask[8];               // bit h: KV head h takes distant logits from the lowest layer's q, k
-  uint16_t* out;                        // [T][H_q][128] bf16
+  uint16_t* out;                        // [T][H_q][head_dim] bf16
   int32_t* err_flag;
 };
 
