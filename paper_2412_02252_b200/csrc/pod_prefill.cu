@@ -402,18 +402,18 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // diagonal get the causal mask, and a pass over a tile with both kinds of key keeps the kind its
       // product is meant for.
       const bool masked = c.mixed || (k0 + BN - 1 > qg0);
-      // Common case (no mask, not the first pass): ONE reading of the row.  The exponentials are taken against
+      // Common case (no mask): ONE reading of the row.  The exponentials are taken against
       // the reference maximum the row already has while the tile's own maximum is found on the side; P stays
       // in registers until it is known that no row of the warp has to raise its reference, which is nearly
       // always so (a raise needs a logit 8 log2 units above everything seen before).  S is still intact then,
       // so the rare other case simply falls through to the general path below.
       bool done = false;
-      if (!masked && v > 0) {
-        const float m_use = (m_used == -INFINITY) ? 0.f : m_used;
+      if (!masked) {
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         float ps4[4] = {0.f, 0.f, 0.f, 0.f};
         uint32_t pk[BN / 32][16];
         float ta[32], tb[32];
+        float m_use = 0.f;
         auto piece = [&](const float (&t)[32], uint32_t (&o)[16]) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -428,6 +428,13 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         tmem_ld32(tmg, ta);                                     // the next piece is on its way while one is worked on
         tmem_ld_wait();
         tmem_ld32(tmg + 32, tb);
+        if (m_used == -INFINITY) {                              // a row's first keys: any reference near their maximum will do
+          float m0 = ta[0];
+#pragma unroll
+          for (int i = 1; i < 32; ++i) m0 = fmaxf(m0, ta[i]);
+          m_used = m0 * p.scale_log2;                           // finite: nothing is masked in this tile; O and the sum are still 0
+        }
+        m_use = m_used;
         piece(ta, pk[0]);
         tmem_ld_wait();
         tmem_ld32(tmg + 64, ta);
