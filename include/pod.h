@@ -225,7 +225,8 @@ const char* pod_strerror(int status);
  * The cache is not touched: write k, v with pod_cache_write.  Runs on the current device; the first call
  * on a device allocates one status word and looks up the driver's tensor-map encoder.  Asynchronous on
  * cuda_stream.  Errors: INVALID, CUDA.  pod_prefill_status synchronises the device and returns
- * POD_ERR_DEVICE if a launch gave up a bounded wait since the last call (its output is then invalid). */
+ * POD_ERR_DEVICE if a launch gave up a bounded wait since the last call (its output is then invalid;
+ * until this call has read the error, further launches on the device return without computing). */
 int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, int n_sink, int n_recent,
                      float sm_scale, const void* q_device, const void* k_device, const void* v_device,
                      const void* q_low_device, const void* k_low_device, const int32_t* head_shares,

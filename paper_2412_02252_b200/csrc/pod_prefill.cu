@@ -246,6 +246,12 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                  bar_pfull = bar_q + 104, bar_odone = bar_q + 120, bar_qfree = bar_q + 136;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 192);
 
+  // A launch whose waits give up would otherwise spend seconds in every one of its thousands of CTAs: once the
+  // error word is set (by this launch or an earlier one, until pod_prefill_status reads it), CTAs return at once.
+  __shared__ int s_abort;
+  if (tid == 0) s_abort = *reinterpret_cast<volatile int32_t*>(p.err_flag);
+  __syncthreads();
+  if (s_abort != 0) return;
   if (tid == 0) {
     bar_init(bar_q, 1);
     bar_init(bar_qfree, 1);
