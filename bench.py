@@ -346,6 +346,9 @@ def run_ours(args):
             step(cache, first_step + s, two_calls)
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
+        # a kernel whose bounded waits gave up in the warm-up would make every timed launch last seconds: stop here
+        if cache.device_status() != B.POD_OK:
+            raise SystemExit("bench.py: the decode kernel reported a device-side wait limit during warm-up")
         launches[0] = 0
         t0.record()
         for s in range(steps):
