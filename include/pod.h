@@ -232,6 +232,11 @@ int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, 
                      const void* q_low_device, const void* k_low_device, const int32_t* head_shares,
                      void* out_device, void* cuda_stream);
 int pod_prefill_status(void);
+/* Fault injection from the host, for tests of that error path (the paper has no counterpart): sets the error
+ * word of the current device as a launch whose wait gave up would.  Until pod_prefill_status has read it,
+ * pod_prefill_attn launches on the device return without writing their output.  Synchronises the device.
+ * Errors: INVALID before the first pod_prefill_attn on the device, CUDA. */
+int pod_prefill_inject_error(void);
 
 /* Decode attention without any allocation.  (The paper has no counterpart of this call; it is a
  * packaging variant of pod_decode_attn for one sequence of ordinary, unshared K/V.)

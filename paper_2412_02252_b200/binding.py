@@ -60,6 +60,7 @@ def _load() -> ctypes.CDLL:
         "pod_prefill_attn": (c_int, [c_int, c_int, c_int, c_int, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p,
                                      c_void_p, c_void_p, P(c_int32), c_void_p, c_void_p]),
         "pod_prefill_status": (c_int, []),
+        "pod_prefill_inject_error": (c_int, []),
         "pod_dense_decode_attn_static": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_int,
                                                  c_int, c_float, c_void_p]),
     }
@@ -74,7 +75,8 @@ EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_required_b
            "pod_cache_create_blocks", "pod_greedy_layer_blocks", "pod_cache_destroy", "pod_cache_write",
            "pod_decode_attn", "pod_append_decode_attn", "pod_cache_set_gate_threshold", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
            "pod_cache_read_region", "pod_cache_device_status", "pod_cache_last_cuda_error",
-           "pod_cache_last_launch", "pod_strerror", "pod_prefill_attn", "pod_prefill_status", "pod_dense_decode_attn_static"]
+           "pod_cache_last_launch", "pod_strerror", "pod_prefill_attn", "pod_prefill_status", "pod_prefill_inject_error",
+           "pod_dense_decode_attn_static"]
 
 
 class PodError(RuntimeError):
@@ -219,6 +221,11 @@ def pod_prefill_attn(q, k, v, out, *, n_sink: int, n_recent: int, q_low=None, k_
 
 def pod_prefill_status() -> int:
     return lib.pod_prefill_status()
+
+
+def pod_prefill_inject_error() -> int:
+    """Sets the device's prefill error word from the host (tests of the error path)."""
+    return _check(lib.pod_prefill_inject_error(), "pod_prefill_inject_error")
 
 
 def pod_dense_decode_attn_static(kv, capacity: int, n_tokens: int, q, out, n_q_heads: int, n_kv_heads: int,

@@ -654,3 +654,15 @@ extern "C" int pod_prefill_status(void) {
   if (flag != 0 && cudaMemset(su->err, 0, 4) != cudaSuccess) return POD_ERR_CUDA;
   return flag ? POD_ERR_DEVICE : POD_OK;
 }
+
+// Sets the error word of the current device as a kernel whose wait gave up would (fault injection from the host, for
+// tests of the error path): the next launches return without computing until pod_prefill_status has been called.
+extern "C" int pod_prefill_inject_error(void) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return POD_ERR_CUDA;
+  PrefillSetup* su = &g_pf[dev];
+  if (!su->ready) return POD_ERR_INVALID;                    // no pod_prefill_attn on this device yet
+  if (cudaDeviceSynchronize() != cudaSuccess) return POD_ERR_CUDA;
+  const int32_t one = 1;
+  return cudaMemcpy(su->err, &one, 4, cudaMemcpyHostToDevice) == cudaSuccess ? POD_OK : POD_ERR_CUDA;
+}

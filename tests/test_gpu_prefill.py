@@ -158,3 +158,26 @@ def test_prefill_rejects_bad_arguments():
         B.pod_prefill_attn(x, x, x, x, n_sink=1, n_recent=0)
     with pytest.raises(B.PodError):
         B.pod_prefill_attn(x, x, x, x, n_sink=1, n_recent=1, q_low=x)           # q_low without k_low
+
+
+def test_prefill_error_word_stops_launches_until_read():
+    """The error path without any failing kernel: the error word is set from the host; launches then return
+    without touching their output, pod_prefill_status reports the error once and clears it, and the next
+    launch computes again."""
+    T, Hq, Hkv = 300, 4, 2
+    q, kv = _inputs(36, T, Hq, Hkv)
+    Q, K, V = q(0), kv(synth.TAG_K, 0), kv(synth.TAG_V, 0)
+    out = torch.zeros(T, Hq, 128, dtype=torch.bfloat16, device="cuda")
+    B.pod_prefill_attn(Q, K, V, out, n_sink=4, n_recent=32)
+    assert B.pod_prefill_status() == B.POD_OK
+    good = out.clone()
+    B.pod_prefill_inject_error()
+    out.fill_(7.0)
+    B.pod_prefill_attn(Q, K, V, out, n_sink=4, n_recent=32)
+    torch.cuda.synchronize()
+    assert (out == 7.0).all()                                   # nothing was computed
+    assert B.pod_prefill_status() == B.POD_ERR_DEVICE
+    assert B.pod_prefill_status() == B.POD_OK                   # read once, cleared
+    B.pod_prefill_attn(Q, K, V, out, n_sink=4, n_recent=32)
+    torch.cuda.synchronize()
+    assert B.pod_prefill_status() == B.POD_OK and torch.equal(out, good)
