@@ -508,6 +508,17 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     p.v_len[b] = in ? c->h_len(layer, b) : 0;
     p.v_cap_d[b] = in ? c->cv.seq_cap_d[b] : 0;
     p.v_row_base[b] = in ? c->cv.seq_row_base[b] : 0;
+    const int32_t pos = p.v_len[b] - 1;
+    p.v_ring_slot[b] = (in && pos >= g.n_sink) ? (pos - g.n_sink) % g.n_recent : 0;
+  }
+  p.heads_by_value = H <= SMALL_HEADS ? 1 : 0;
+  p.v_store_mask = 0u;
+  for (int h = 0; h < SMALL_HEADS; ++h) {
+    const bool in = p.heads_by_value && h < H;
+    p.v_low[h] = in ? c->low_of(layer, h) : 0;
+    p.v_slot[h] = in ? c->slot_of(layer, h) : 0;
+    if (in && c->bm.shared && c->low_of(layer, h) == layer && layer + 1 < g.n_layers && c->low_of(layer + 1, h) == layer)
+      p.v_store_mask |= 1u << h;
   }
   // With a gate threshold set, a layer in which some head reads its block's logits runs as two
   // launches: the proximal tokens (which decides, per query head, whether the distant tokens are

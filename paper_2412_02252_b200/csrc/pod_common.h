@@ -9,6 +9,7 @@
 namespace pod {
 
 constexpr int SMALL_BATCH = 8;        // batches up to this size pass per-sequence scalars by value
+constexpr int SMALL_HEADS = 16;       // up to this many KV heads pass the layer's rows of the block tables by value
 constexpr int MAX_SPLITS_CAP = 128;   // upper bound of splits per sequence (partial buffers, combine)
 
 // Shape of the split-K decode kernel (compile-time; -D overrides are for tuning builds).
@@ -157,7 +158,14 @@ struct DecodeParams {
   int32_t by_value;        // 1: use the arrays below instead of len / seq_row_base / seq_cap_d
   int32_t v_len[SMALL_BATCH];
   int32_t v_cap_d[SMALL_BATCH];
+  int32_t v_ring_slot[SMALL_BATCH];   // (v_len - 1 - S) mod W: ring slot of the sequence's last token (0 if it is a sink)
   int64_t v_row_base[SMALL_BATCH];
+  // Few KV heads: this layer's rows of the block tables by value (low[layer][h], slot[layer][h]) and the
+  // heads that store their distant logits in this launch (lowest layer of a block that goes on).
+  int32_t heads_by_value;
+  int32_t v_low[SMALL_HEADS];
+  int32_t v_slot[SMALL_HEADS];
+  uint32_t v_store_mask;
 };
 
 struct DecodePlan {

@@ -223,24 +223,36 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // A layer that reads the block's stored logits needs no key rows: its distant tiles hold 32
   // value rows (both halves of a stage), so the bytes in flight per stage stay the same.
   // blocks are per KV head: is this layer the lowest of this head's block, and does the block go on?
-  const int low_layer = lowest_of(y, p.layer, kvh);
-  const int kslot = slot_of(y, p.layer, kvh);
+  // (with few KV heads the host passes this layer's rows of the block tables by value: no global load
+  // stands between a CTA's start and its first tile requests)
+  int low_layer, kslot;
+  bool sc_write;
+  if (p.heads_by_value) {
+    low_layer = p.v_low[kvh];
+    kslot = p.v_slot[kvh];
+    sc_write = (p.v_store_mask >> kvh) & 1u;
+  } else {
+    low_layer = lowest_of(y, p.layer, kvh);
+    kslot = slot_of(y, p.layer, kvh);
+    sc_write = y.shared && low_layer == p.layer && p.layer + 1 < y.L && lowest_of(y, p.layer + 1, kvh) == p.layer;
+  }
   const bool is_low = low_layer == p.layer;
-  const bool sc_write = y.shared && is_low && p.layer + 1 < y.L && lowest_of(y, p.layer + 1, kvh) == p.layer;
   const bool sc_read = !is_low && kvh < 256 && ((p.score_read_mask[kvh >> 5] >> (kvh & 31)) & 1u);
   // CTAs of this head: in proportion to the rows it streams (keys and values, or values and the
-  // proximal keys only), so that heads with different roles in one launch finish together
-  const int64_t work_rows = sc_read ? (int64_t)n_p_s * 2 + n_d_s : 2 * ((int64_t)n_p_s + n_d_s);
-  const int nsplit = (int)min((int64_t)p.max_splits, (work_rows + p.split_rows - 1) / p.split_rows);
+  // proximal keys only), so that heads with different roles in one launch finish together.
+  // (a head's rows are a fraction of the arena's, which number less than 2^31: 32-bit arithmetic)
+  const uint32_t work_rows = sc_read ? (uint32_t)n_p_s * 2u + (uint32_t)n_d_s : 2u * ((uint32_t)n_p_s + (uint32_t)n_d_s);
+  const int nsplit = (int)min((uint32_t)p.max_splits, (work_rows + (uint32_t)p.split_rows - 1u) / (uint32_t)p.split_rows);
   if (split >= nsplit) return;
-  const int DT = sc_read ? 2 * TOK : TOK;         // tokens per distant tile
-  const int ntp = (n_p_s + TOK - 1) / TOK, ntd = (n_d_s + DT - 1) / DT;
+  const int DT_SH = sc_read ? 5 : 4;              // log2 of the tokens per distant tile
+  const int DT = 1 << DT_SH;
+  const int ntp = (n_p_s + TOK - 1) / TOK, ntd = (n_d_s + DT - 1) >> DT_SH;
   const int ntiles = ntp + ntd;
   const int tch = p.tiles_per_chunk;
   const int nwh = nsplit * NW;                    // warps working on this head
   const int gw = split * NW + warp;               // this warp's index among them
-  const int nchunks = (ntiles + tch - 1) / tch;
-  const int k_static = (nchunks / nwh) * p.static_eighths / 8;   // chunks per warp taken without a draw
+  const int nchunks = (int)((uint32_t)(ntiles + tch - 1) / (uint32_t)tch);
+  const int k_static = (int)((uint32_t)nchunks / (uint32_t)nwh) * p.static_eighths / 8;   // chunks per warp taken without a draw
   const int dyn_base = k_static * nwh;            // first chunk id that is drawn
   int* sched = p.sched + ((int64_t)b * y.H_kv + kvh) * SCHED_STRIDE;
 
@@ -262,15 +274,27 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     pdl_launch_dependents();
     waited = true;
   }
+  // A warp's first draw is issued when it enters the last of its fixed chunks (not at the start, where
+  // the draws of all warps of a head would queue up on one counter), and never before the wait: the
+  // previous kernel's last CTA of the head resets the counter.
   unsigned drawn = 0;                             // lane 0: result of the draw issued one chunk ahead
-  if (waited && lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+  bool drew = false;
   int c_id, c_t = 0, c_j = 0;
   bool walk_done = false;
+  auto first_draw = [&]() {
+    if (!drew && waited && c_j >= k_static - 1) {
+      if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+      drew = true;
+    }
+  };
   if (k_static > 0) {
     c_id = gw;
-  } else {
+    first_draw();
+  } else {                                        // (the wait above has happened)
+    if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
     c_id = dyn_base + (int)__shfl_sync(0xffffffffu, drawn, 0);
     if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+    drew = true;
   }
   auto next_tile = [&]() -> int {                 // virtual tile index, or -1 when the head is used up
     if (walk_done) return -1;
@@ -279,6 +303,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       ++c_j;
       if (c_j < k_static) {
         c_id = gw + c_j * nwh;
+        first_draw();
       } else {
         c_id = dyn_base + (int)__shfl_sync(0xffffffffu, drawn, 0);
         if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
@@ -329,7 +354,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     if (pos < y.S) {
       rA = pos;
     } else {
-      rA = y.S + (pos - y.S) % y.W;
+      rA = y.S + (p.by_value ? p.v_ring_slot[bv] : (pos - y.S) % y.W);
       if (pos - y.W >= y.S) rB = pos - y.W - y.S;
     }
     tA = rA / TOK; cA = rA % TOK;
@@ -349,8 +374,9 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
 #pragma unroll
       for (int s = 0; s < NSTAGE; ++s)
         if (vt_q[s] >= 0) issue(vt_q[s], s, 0, 2);
-      drawn = (unsigned)atomicAdd(sched, 1);
     }
+    waited = true;
+    first_draw();
   }
 
   // a head's lowest layer saves its queries for the other layers of the block
