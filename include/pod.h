@@ -67,7 +67,7 @@ typedef struct pod_cache pod_cache; /* opaque: host bookkeeping + device arena *
 
 typedef struct {
   int32_t n_layers;    /* L >= 1 */
-  int32_t n_q_heads;   /* H_q; H_q / H_kv must be 1, 2, 4 or 8 (grouped-query attention) */
+  int32_t n_q_heads;   /* H_q: a multiple of H_kv with H_q / H_kv <= 8 (grouped-query attention) */
   int32_t n_kv_heads;  /* H_kv */
   int32_t head_dim;    /* d: 64 or 128 */
   int32_t group_size;  /* G >= 1 layers per block (G = 1: ordinary dense attention) */
@@ -86,11 +86,17 @@ typedef struct {
 size_t pod_cache_required_bytes(const pod_config* cfg, const int32_t* seq_capacity);
 
 /* Creates a cache.  arena: device memory of at least pod_cache_required_bytes, 256-byte
- * aligned, owned by the caller and kept alive until pod_cache_destroy; or NULL to let the
- * library allocate (and later free) it with cudaMalloc.  Region contents start undefined,
- * lengths start at 0.  Synchronous.  The physical layout inside the arena is private; its
- * logical content is what pod_cache_read_region returns.  Every region starts on a
- * multiple of 128 bytes.  Errors: INVALID, ARENA, CUDA. */
+ * aligned (one row of head_dim 128), owned by the caller and kept alive until
+ * pod_cache_destroy; or NULL to let the library allocate (and later free) it with cudaMalloc.
+ * The call sets the WHOLE arena to zero, the caller's included (one synchronous cudaMemset of
+ * pod_cache_required_bytes: about 15 ms per 100 GB on a B200): the decode kernel's tiles may
+ * reach a few rows past the rows a head holds, those logits are masked, but the rows must
+ * hold finite numbers.  Rows that hold no token therefore read as zeros; lengths start at 0.
+ * Synchronous.  The physical layout inside the arena is private; its logical content is what
+ * pod_cache_read_region returns.  Every region starts on a multiple of 128 bytes.
+ * More than 256 KV heads are accepted; KV heads 256 and above never reuse stored distant
+ * logits (they score the block's keys themselves: same result, more bytes).
+ * Errors: INVALID, ARENA, CUDA. */
 int pod_cache_create(const pod_config* cfg, const int32_t* seq_capacity,
                      void* arena_device, size_t arena_bytes, pod_cache** out);
 
@@ -200,6 +206,12 @@ int pod_cache_read_region(const pod_cache* c, int region, int layer_or_block, in
  * bounded-wait limit since the last call (the flag is cleared), else POD_OK. */
 int pod_cache_device_status(pod_cache* c);
 
+/* Fault injection from the host, for tests of that error path (the paper has no counterpart): sets
+ * the cache's error word as a kernel whose bounded wait gave up would, without making any kernel
+ * fail.  The next pod_cache_device_status reports POD_ERR_DEVICE once and clears the word.
+ * Synchronises the device.  Errors: INVALID, CUDA. */
+int pod_cache_inject_error(pod_cache* c);
+
 /* Last CUDA runtime error code seen by this cache (0 if none). */
 int pod_cache_last_cuda_error(const pod_cache* c);
 
@@ -223,8 +235,9 @@ const char* pod_strerror(int status);
  *   head_shares   : host int32 [n_kv_heads] or NULL; with q_low given, KV head h takes its distant logits
  *                   from q_low / k_low if head_shares is NULL or head_shares[h] != 0 (head-wise blocks).
  * The cache is not touched: write k, v with pod_cache_write.  Runs on the current device; the first call
- * on a device allocates one status word and looks up the driver's tensor-map encoder.  Asynchronous on
- * cuda_stream.  Errors: INVALID, CUDA.  pod_prefill_status synchronises the device and returns
+ * on a device looks up the driver's tensor-map encoder and the address of the status word (a word inside the
+ * library's device image: nothing is allocated).  With q_low given at most 256 KV heads (INVALID beyond).
+ * Asynchronous on cuda_stream.  Errors: INVALID, CUDA.  pod_prefill_status synchronises the device and returns
  * POD_ERR_DEVICE if a launch gave up a bounded wait since the last call (its output is then invalid;
  * until this call has read the error, further launches on the device return without computing). */
 int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, int n_sink, int n_recent,
@@ -263,8 +276,10 @@ int pod_prefill_inject_error(void);
  * 2 * n_kv_heads * capacity < 2^31.  Shapes as for pod_config (head_dim 64 or 128, at most 8
  * query heads per KV head); other invalid arguments give POD_ERR_INVALID.
  *
- * The first call on each device looks up the array's device address (cudaGetSymbolAddress) and
- * the driver's tensor-map encoder; make that first call outside any stream capture.  All calls
+ * The pointers must belong to the current device.  The first call on each device looks up the array's
+ * device address (cudaGetSymbolAddress) and the driver's tensor-map encoder, sets the kernel's
+ * shared-memory attribute on that device and zeroes the error word; make that first call outside any
+ * stream capture.  All calls
  * on a device share the one array, which keeps the previous call's contents; the call clears
  * the counters that must start at zero on the given stream.  Two calls whose kernels may run at
  * the same time on one device (different streams, different threads) race on the array: order
@@ -273,6 +288,14 @@ int pod_prefill_inject_error(void);
 int pod_dense_decode_attn_static(const void* kv_device, int capacity, int n_tokens,
                                  const void* q_device, void* out_device, int n_q_heads,
                                  int n_kv_heads, int head_dim, float sm_scale, void* cuda_stream);
+/* Error word of the fixed array on the current device (the paper has no counterpart): synchronises the
+ * device and returns POD_ERR_DEVICE if a pod_dense_decode_attn_static kernel gave up a bounded wait since
+ * the last call (the outputs of the calls since then are invalid), else POD_OK; the word is cleared.  The
+ * calls themselves never clear it.  No allocation: one small copy through the array's address.  Call it with
+ * the device current that ran the kernels.  ..._inject_error sets the word from the host (tests of this
+ * path; no kernel is made to fail).  Errors: CUDA. */
+int pod_dense_decode_attn_static_status(void);
+int pod_dense_decode_attn_static_inject_error(void);
 
 #ifdef __cplusplus
 }

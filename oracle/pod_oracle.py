@@ -67,26 +67,30 @@ def check_lowest_map(low) -> np.ndarray:
 
 
 def greedy_layer_blocks(sim, threshold=0.5):
-    """Algorithm 1 (Section 2.1): bottom-up greedy grouping of consecutive similar layers, per head.
+    """Greedy grouping of consecutive similar layers, per head (Section 2.1, Algorithm 1).
 
     sim: [H][L][L], sim[h][a][b] = similarity of layers a and b for head h (1 = identical).
-    For each head the first layer opens a block; every next layer joins the current (last)
-    block if it is similar (>= threshold) to ALL layers already in it, else it opens a new one.
+    The rule of the algorithm: walking up from layer 0, a layer stays in the block of the layer
+    below it exactly when it is similar (>= threshold) to every layer that block holds so far;
+    otherwise it starts a block of its own.  Written here through each layer's "reach": the lowest
+    layer m such that the layer is similar to all of m .. l-1.  A layer then continues the block
+    below it iff its reach is at or below that block's first layer.
     Returns, per head, the list of blocks, each a list of 0-based layers.
     """
-    sim = np.asarray(sim, dtype=np.float64)
-    H, L, _ = sim.shape
-    head_wise_layer_blocks = []
+    similar = np.asarray(sim, dtype=np.float64) >= threshold
+    H, L, _ = similar.shape
+    result = []
     for h in range(H):
-        current_head_layer_blocks = [[0]]
+        reach = np.arange(L)
+        for l in range(L):
+            below = similar[h, l, :l][::-1]                    # l-1, l-2, ..., 0
+            run = int(np.argmin(below)) if not below.all() else l   # similar layers directly below l
+            reach[l] = l - run
+        first = np.zeros(L, dtype=np.int64)                    # first layer of the block of each layer
         for l in range(1, L):
-            current_block = current_head_layer_blocks[-1]
-            if all(sim[h, l, lh] >= threshold for lh in current_block):
-                current_block.append(l)
-            else:
-                current_head_layer_blocks.append([l])
-        head_wise_layer_blocks.append(current_head_layer_blocks)
-    return head_wise_layer_blocks
+            first[l] = first[l - 1] if reach[l] <= first[l - 1] else l
+        result.append([[int(l) for l in np.flatnonzero(first == f)] for f in np.unique(first)])
+    return result
 
 
 def lowest_map_from_blocks(head_wise_layer_blocks, n_layers: int) -> np.ndarray:

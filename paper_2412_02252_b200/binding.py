@@ -54,6 +54,7 @@ def _load() -> ctypes.CDLL:
         "pod_cache_reset": (c_int, [c_void_p, c_int]),
         "pod_cache_read_region": (c_int, [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int, c_void_p]),
         "pod_cache_device_status": (c_int, [c_void_p]),
+        "pod_cache_inject_error": (c_int, [c_void_p]),
         "pod_cache_last_cuda_error": (c_int, [c_void_p]),
         "pod_cache_last_launch": (c_int, [c_void_p, P(c_int32), P(c_int32), P(c_int32)]),
         "pod_strerror": (c_char_p, [c_int]),
@@ -63,6 +64,8 @@ def _load() -> ctypes.CDLL:
         "pod_prefill_inject_error": (c_int, []),
         "pod_dense_decode_attn_static": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_int,
                                                  c_int, c_float, c_void_p]),
+        "pod_dense_decode_attn_static_status": (c_int, []),
+        "pod_dense_decode_attn_static_inject_error": (c_int, []),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -74,9 +77,10 @@ lib = _load()
 EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_required_bytes_blocks",
            "pod_cache_create_blocks", "pod_greedy_layer_blocks", "pod_cache_destroy", "pod_cache_write",
            "pod_decode_attn", "pod_append_decode_attn", "pod_cache_set_gate_threshold", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
-           "pod_cache_read_region", "pod_cache_device_status", "pod_cache_last_cuda_error",
+           "pod_cache_read_region", "pod_cache_device_status", "pod_cache_inject_error", "pod_cache_last_cuda_error",
            "pod_cache_last_launch", "pod_strerror", "pod_prefill_attn", "pod_prefill_status", "pod_prefill_inject_error",
-           "pod_dense_decode_attn_static"]
+           "pod_dense_decode_attn_static", "pod_dense_decode_attn_static_status",
+           "pod_dense_decode_attn_static_inject_error"]
 
 
 class PodError(RuntimeError):
@@ -199,6 +203,10 @@ class PodCache:
     def device_status(self) -> int:
         return lib.pod_cache_device_status(self._h)
 
+    def inject_error(self) -> int:
+        """Sets the cache's error word from the host (tests of the error path)."""
+        return _check(lib.pod_cache_inject_error(self._h), "pod_cache_inject_error")
+
     def last_cuda_error(self) -> int:
         return lib.pod_cache_last_cuda_error(self._h)
 
@@ -237,3 +245,13 @@ def pod_dense_decode_attn_static(kv, capacity: int, n_tokens: int, q, out, n_q_h
     return _check(lib.pod_dense_decode_attn_static(_ptr(kv), capacity, n_tokens, _ptr(q), _ptr(out), n_q_heads,
                                                    n_kv_heads, head_dim, sm_scale, stream),
                   "pod_dense_decode_attn_static")
+
+
+def pod_dense_decode_attn_static_status() -> int:
+    """POD_ERR_DEVICE once if a kernel of the allocation-free entry gave up a bounded wait, else POD_OK."""
+    return lib.pod_dense_decode_attn_static_status()
+
+
+def pod_dense_decode_attn_static_inject_error() -> int:
+    """Sets that error word from the host (tests of the error path)."""
+    return _check(lib.pod_dense_decode_attn_static_inject_error(), "pod_dense_decode_attn_static_inject_error")

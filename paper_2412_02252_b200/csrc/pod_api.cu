@@ -682,6 +682,19 @@ int pod_cache_device_status(pod_cache* c) {
   return flag ? POD_ERR_DEVICE : POD_OK;
 }
 
+// Fault injection from the host (tests of the error path): sets the cache's error word as a kernel whose
+// bounded wait gave up would.  No kernel is made to fail.
+int pod_cache_inject_error(pod_cache* c) {
+  if (!c) return POD_ERR_INVALID;
+  if (c->dry) return POD_DRY_RUN;
+  const int32_t one = 1;
+  cudaError_t e = cudaSetDevice(c->cfg.device);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(c->arena + c->cv.off_err, &one, 4, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  return POD_OK;
+}
+
 int pod_cache_last_cuda_error(const pod_cache* c) { return c ? c->last_cuda : (int)cudaErrorInvalidValue; }
 
 int pod_cache_last_launch(const pod_cache* c, int32_t* split_tokens, int32_t* n_ctas, int32_t* n_kernels) {

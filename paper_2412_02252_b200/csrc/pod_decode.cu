@@ -829,12 +829,15 @@ cudaLaunchConfig_t pdl_config(cudaLaunchAttribute* attr, dim3 grid, dim3 block, 
 template <int D>
 int launch_decode_t(const CUtensorMap& tmap, const DecodeParams& p, int grid_splits, cudaStream_t s) {
   using C = Cfg<D>;
-  static bool configured = false;
-  if (!configured) {
+  // the shared-memory attribute is a per-device setting of the kernel
+  static bool configured[64] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return (int)cudaErrorInvalidDevice;
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(pod_decode_splitk_kernel<D>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return (int)e;
-    configured = true;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   cudaLaunchAttribute attr[1];
   cudaLaunchConfig_t cfg = pdl_config(attr, dim3(p.y.H_kv, grid_splits, p.y.B), dim3(C::NW * 32), C::SMEM, s);

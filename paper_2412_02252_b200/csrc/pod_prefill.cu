@@ -567,10 +567,15 @@ pod_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   }
 }
 
+// Error word of the bounded waits: one per device that loads the library, inside the device image, so that
+// nothing is allocated and nothing has to be freed.  In host code the name is only a handle for
+// cudaGetSymbolAddress.
+static __device__ int32_t g_prefill_err_word;
+
 struct PrefillSetup {
   bool ready = false;
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
-  int32_t* err = nullptr;       // device word
+  int32_t* err = nullptr;       // device address of g_prefill_err_word on that device
 };
 PrefillSetup g_pf[64];
 std::mutex g_pf_mutex;
@@ -598,6 +603,7 @@ extern "C" int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int
   if (n_sink < 0 || n_recent < 1 || !(sm_scale >= 0.f) || isinf(sm_scale)) return POD_ERR_INVALID;
   if (n_q_heads > 65535) return POD_ERR_INVALID;
   if ((q_low == nullptr) != (k_low == nullptr)) return POD_ERR_INVALID;
+  if (q_low != nullptr && n_kv_heads > 256) return POD_ERR_INVALID;     // the sharing mask holds 256 KV heads
   for (const void* ptr : {q, k, v, q_low, k_low, (const void*)out})
     if (((uintptr_t)ptr % 16) != 0) return POD_ERR_INVALID;
   int dev = 0;
@@ -611,7 +617,10 @@ extern "C" int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int
       if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
           qres != cudaDriverEntryPointSuccess || fn == nullptr)
         return POD_ERR_CUDA;
-      if (cudaMalloc(&su->err, 4) != cudaSuccess || cudaMemset(su->err, 0, 4) != cudaSuccess) return POD_ERR_CUDA;
+      void* errp = nullptr;
+      if (cudaGetSymbolAddress(&errp, g_prefill_err_word) != cudaSuccess || errp == nullptr) return POD_ERR_CUDA;
+      su->err = static_cast<int32_t*>(errp);
+      if (cudaMemset(su->err, 0, 4) != cudaSuccess) return POD_ERR_CUDA;
       if (cudaFuncSetAttribute(pod_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<128>::SMEM) != cudaSuccess ||
           cudaFuncSetAttribute(pod_prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Plan<64>::SMEM) != cudaSuccess)
         return POD_ERR_CUDA;
@@ -625,7 +634,7 @@ extern "C" int pod_prefill_attn(int n_tokens, int n_q_heads, int n_kv_heads, int
   p.out = static_cast<uint16_t*>(out);
   p.err_flag = su->err;
   if (q_low != nullptr)
-    for (int h = 0; h < n_kv_heads && h < 256; ++h)
+    for (int h = 0; h < n_kv_heads; ++h)
       if (head_shares == nullptr || head_shares[h] != 0) p.share_mask[h >> 5] |= 1u << (h & 31);
   CUtensorMap tq, tk, tv, tql, tkl;
   const void* ql = q_low ? q_low : q;

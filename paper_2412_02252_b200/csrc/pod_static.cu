@@ -36,7 +36,7 @@ struct DeviceSetup {
   bool ready = false;
   unsigned char* scratch = nullptr;   // device address of g_static_scratch on that device
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
-  int sm_count = 0, resident = 0;
+  int sm_count = 0, resident128 = 0, resident64 = 0;   // resident CTAs per SM of the kernel for head size 128 / 64
 };
 DeviceSetup g_setup[STATIC_MAX_DEVICES];
 std::mutex g_setup_mutex;
@@ -55,10 +55,16 @@ int setup_device(int dev, DeviceSetup** out) {
       return POD_ERR_CUDA;
     int sm = 0;
     if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return POD_ERR_CUDA;
+    // The kernel's shared-memory attribute is a per-device setting: both head sizes are configured here,
+    // on this device, and the occupancy the driver reports sizes the grid.
+    const int r128 = decode_resident_ctas_per_sm(128), r64 = decode_resident_ctas_per_sm(64);
+    if (r128 < 1 || r64 < 1) return POD_ERR_CUDA;
+    // the error word starts at zero; afterwards only pod_dense_decode_attn_static_status clears it
+    if (cudaMemset(static_cast<unsigned char*>(ptr) + OFF_ERR, 0, 256) != cudaSuccess) return POD_ERR_CUDA;
     s.scratch = static_cast<unsigned char*>(ptr);
     s.encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
     s.sm_count = sm;
-    s.resident = 2;
+    s.resident128 = r128; s.resident64 = r64;
     s.ready = true;
   }
   *out = &s;
@@ -102,7 +108,7 @@ extern "C" int pod_dense_decode_attn_static(const void* kv_device, int capacity,
     return POD_ERR_INVALID;
 
   // one CTA per (split, KV head): about one wave of resident CTAs, at most 64 splits
-  int k = (su->sm_count * su->resident) / n_kv_heads;
+  int k = (su->sm_count * (head_dim == 128 ? su->resident128 : su->resident64)) / n_kv_heads;
   if (k < 1) k = 1;
   if (k > STATIC_MAX_SPLITS) k = STATIC_MAX_SPLITS;
   int split_tokens = (n_tokens + k - 1) / k;
@@ -136,9 +142,39 @@ extern "C" int pod_dense_decode_attn_static(const void* kv_device, int capacity,
   p.v_len[0] = n_tokens; p.v_cap_d[0] = 0; p.v_row_base[0] = 0; p.v_ring_slot[0] = (n_tokens - 1) % capacity;
   p.heads_by_value = 0;
 
-  // The array keeps whatever the previous call left: the chunk counters, the tickets and the
-  // error flag must start at zero.
-  if (cudaMemsetAsync(su->scratch + OFF_SCHED, 0, SCHED_BYTES + 256, stream) != cudaSuccess) return POD_ERR_CUDA;
+  // The array keeps whatever the previous call left: the chunk counters and the tickets must start at
+  // zero.  The error word is left alone: only pod_dense_decode_attn_static_status reads and clears it.
+  if (cudaMemsetAsync(su->scratch + OFF_SCHED, 0, SCHED_BYTES, stream) != cudaSuccess) return POD_ERR_CUDA;
   const int e = launch_decode(tmap, p, grid_splits, stream);
   return e == 0 ? POD_OK : POD_ERR_CUDA;
+}
+
+// Reads (and clears) the error word of the fixed array on the current device.  No allocation: a plain
+// copy through the address cudaGetSymbolAddress gave.
+extern "C" int pod_dense_decode_attn_static_status(void) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) return POD_ERR_CUDA;
+  DeviceSetup* su = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!g_setup[dev].ready) return POD_OK;              // nothing has run on this device
+    su = &g_setup[dev];
+  }
+  int32_t flag = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return POD_ERR_CUDA;
+  if (cudaMemcpy(&flag, su->scratch + OFF_ERR, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return POD_ERR_CUDA;
+  if (flag != 0 && cudaMemset(su->scratch + OFF_ERR, 0, 4) != cudaSuccess) return POD_ERR_CUDA;
+  return flag ? POD_ERR_DEVICE : POD_OK;
+}
+
+// Sets that error word from the host, as a kernel whose bounded wait gave up would (tests of the error path).
+extern "C" int pod_dense_decode_attn_static_inject_error(void) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) return POD_ERR_CUDA;
+  DeviceSetup* su = nullptr;
+  const int st = setup_device(dev, &su);
+  if (st != POD_OK) return st;
+  if (cudaDeviceSynchronize() != cudaSuccess) return POD_ERR_CUDA;
+  const int32_t one = 1;
+  return cudaMemcpy(su->scratch + OFF_ERR, &one, 4, cudaMemcpyHostToDevice) == cudaSuccess ? POD_OK : POD_ERR_CUDA;
 }

@@ -279,3 +279,21 @@ def test_null_handles():
     assert B.lib.pod_decode_attn(None, 0, None, None, None) == B.POD_ERR_INVALID
     assert B.lib.pod_append_decode_attn(None, 0, None, None, None, None, None) == B.POD_ERR_INVALID
     assert B.lib.pod_cache_write(None, 0, 0, None, None, 1, None) == B.POD_ERR_INVALID
+
+
+def test_prefill_rejects_more_sharing_kv_heads_than_its_mask_holds():
+    """Argument checks come before any CUDA call, so they are testable without a GPU: with the lowest layer's
+    q, k given, more than 256 KV heads cannot be expressed in the kernel's sharing mask and are refused
+    rather than silently computed as ordinary causal attention."""
+    p = _fake_ptr()
+    call = lambda hq, hkv, ql, kl: B.lib.pod_prefill_attn(8, hq, hkv, 64, 4, 4, 0.0, p, p, p, ql, kl, None, p, None)
+    assert call(512, 512, p, p) == B.POD_ERR_INVALID
+    assert call(257, 257, p, p) == B.POD_ERR_INVALID
+    assert call(4, 2, p, None) == B.POD_ERR_INVALID             # q_low without k_low
+    assert call(4, 2, p + 8, p) == B.POD_ERR_INVALID            # misaligned
+
+
+def test_error_injection_on_a_host_only_cache_is_a_dry_run():
+    c = B.PodCache(_cfg(), [64])
+    assert c.inject_error() == B.POD_DRY_RUN
+    assert c.device_status() == B.POD_DRY_RUN

@@ -487,3 +487,20 @@ def _dense_head(case, k, q, h):
     qq = q[0, h].double().cpu().numpy()
     o, _ = O.pod_attention_joint(qq, qq, kk, kk, kk, case.S, case.W)
     return o
+
+
+def test_cache_error_word_is_reported_once_and_decoding_goes_on():
+    """The decode path's error word without any failing kernel: it is set from the host
+    (pod_cache_inject_error), pod_cache_device_status reports POD_ERR_DEVICE once and clears it, and the
+    next decode of the same cache is correct."""
+    case = Case(seed=41, L=2, G=2, Hq=8, Hkv=2, d=64, S=4, W=32, lens=[700])
+    cache = case.make_cache()
+    case.prefill(cache)
+    assert cache.device_status() == B.POD_OK
+    cache.inject_error()
+    assert cache.device_status() == B.POD_ERR_DEVICE
+    assert cache.device_status() == B.POD_OK
+    outs = case.decode_all(cache)                               # asserts POD_OK after the launches
+    for l in range(2):
+        for h in range(8):
+            assert_close(outs[l, 0, h], case.oracle_head(l, 0, h), f"layer {l} head {h} after the injected error")
