@@ -127,6 +127,24 @@ int pod_cache_create_blocks(const pod_config* cfg, const int32_t* seq_capacity,
 int pod_greedy_layer_blocks(const float* sim, int n_heads, int n_layers, float threshold,
                             int32_t* lowest_layer);
 
+/* Split of a cache over several GPUs by KV head (tensor parallelism; the paper's inference path is
+ * one GPU, its only parallelism is in training: Section 3, "Implementation Details").  Every region
+ * of the PoD layout, the query stash, the stored logits and the outputs are per KV head, and a head's
+ * attention needs nothing from another head (Eq. 1, Eq. 2), so rank r of `world` simply owns KV heads
+ * [r * H_kv / world, (r + 1) * H_kv / world) and the H_q / H_kv query heads of each: its cache is an
+ * ordinary cache with those heads, built from *local; k, v, q, out of its calls are the rank's own
+ * slices, contiguous [.][H_kv / world][d] and [B][H_q / world][d] (what column-parallel q/k/v
+ * projections produce); the ranks' outputs are disjoint slices of [B][H_q][d] starting at query head
+ * *first_q_head -- gather them, or feed them to a row-parallel output projection as they are.  No call
+ * of this library communicates between GPUs, and no kernel is ever given another GPU's memory.
+ * pod_shard_block_map cuts a head-wise map [n_layers][H_kv] down to the rank's columns
+ * [n_layers][H_kv / world].  Byte counts of the ranks add up to those of the unsplit cache.
+ * Host only.  Errors: INVALID (world does not divide H_kv, rank out of range, bad config). */
+int pod_shard_config(const pod_config* full, int rank, int world, pod_config* local,
+                     int32_t* first_kv_head, int32_t* first_q_head);
+int pod_shard_block_map(const pod_config* full, const int32_t* lowest_layer, int rank, int world,
+                        int32_t* local_lowest_layer);
+
 /* Frees host state (and the arena if the library allocated it).  Synchronises the device. */
 int pod_cache_destroy(pod_cache* c);
 
@@ -219,6 +237,18 @@ int pod_cache_last_cuda_error(const pod_cache* c);
  * tokens per split, CTAs launched, and kernels launched by that call. */
 int pod_cache_last_launch(const pod_cache* c, int32_t* split_tokens, int32_t* n_ctas,
                           int32_t* n_kernels);
+
+/* Launch trace, for benchmarks (the paper has no counterpart).  Consecutive decode launches of a stream
+ * overlap -- a launch requests its first tiles while the previous one finishes -- so CUDA events between
+ * them (which would serialise them) cannot say what one launch of a pipelined step costs.  With a trace
+ * set, each of the next n_launches kernels of pod_decode_attn / pod_append_decode_attn (a gated layer
+ * is two) writes one pair of uint64 into pairs_device: the GPU's nanosecond timer when its first CTA
+ * starts and when its last CTA ends.  pairs_device: device memory of n_launches * 16 bytes, 8-byte
+ * aligned, caller-owned; the call initialises it (synchronously).  NULL, 0 switches the trace off.
+ * pod_cache_trace_count: pairs handed out so far.  Cost when on: two atomics per CTA.
+ * Errors: INVALID, CUDA. */
+int pod_cache_set_trace(pod_cache* c, void* pairs_device, int n_launches);
+int pod_cache_trace_count(const pod_cache* c);
 
 const char* pod_strerror(int status);
 

@@ -44,6 +44,8 @@ def _load() -> ctypes.CDLL:
         "pod_cache_required_bytes_blocks": (c_size_t, [P(pod_config), P(c_int32), P(c_int32)]),
         "pod_cache_create_blocks": (c_int, [P(pod_config), P(c_int32), P(c_int32), c_void_p, c_size_t, P(c_void_p)]),
         "pod_greedy_layer_blocks": (c_int, [P(c_float), c_int, c_int, c_float, P(c_int32)]),
+        "pod_shard_config": (c_int, [P(pod_config), c_int, c_int, P(pod_config), P(c_int32), P(c_int32)]),
+        "pod_shard_block_map": (c_int, [P(pod_config), P(c_int32), c_int, c_int, P(c_int32)]),
         "pod_cache_destroy": (c_int, [c_void_p]),
         "pod_cache_write": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_void_p]),
         "pod_decode_attn": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
@@ -57,6 +59,8 @@ def _load() -> ctypes.CDLL:
         "pod_cache_inject_error": (c_int, [c_void_p]),
         "pod_cache_last_cuda_error": (c_int, [c_void_p]),
         "pod_cache_last_launch": (c_int, [c_void_p, P(c_int32), P(c_int32), P(c_int32)]),
+        "pod_cache_set_trace": (c_int, [c_void_p, c_void_p, c_int]),
+        "pod_cache_trace_count": (c_int, [c_void_p]),
         "pod_strerror": (c_char_p, [c_int]),
         "pod_prefill_attn": (c_int, [c_int, c_int, c_int, c_int, c_int, c_int, c_float, c_void_p, c_void_p, c_void_p,
                                      c_void_p, c_void_p, P(c_int32), c_void_p, c_void_p]),
@@ -75,10 +79,11 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_required_bytes_blocks",
-           "pod_cache_create_blocks", "pod_greedy_layer_blocks", "pod_cache_destroy", "pod_cache_write",
+           "pod_cache_create_blocks", "pod_greedy_layer_blocks", "pod_shard_config", "pod_shard_block_map",
+           "pod_cache_destroy", "pod_cache_write",
            "pod_decode_attn", "pod_append_decode_attn", "pod_cache_set_gate_threshold", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
            "pod_cache_read_region", "pod_cache_device_status", "pod_cache_inject_error", "pod_cache_last_cuda_error",
-           "pod_cache_last_launch", "pod_strerror", "pod_prefill_attn", "pod_prefill_status", "pod_prefill_inject_error",
+           "pod_cache_last_launch", "pod_cache_set_trace", "pod_cache_trace_count", "pod_strerror", "pod_prefill_attn", "pod_prefill_status", "pod_prefill_inject_error",
            "pod_dense_decode_attn_static", "pod_dense_decode_attn_static_status",
            "pod_dense_decode_attn_static_inject_error"]
 
@@ -138,6 +143,22 @@ def pod_greedy_layer_blocks(sim, threshold: float = 0.5):
     out = (c_int32 * (L * H))()
     _check(lib.pod_greedy_layer_blocks(flat, H, L, threshold, out), "pod_greedy_layer_blocks")
     return [[out[l * H + h] for h in range(H)] for l in range(L)]
+
+
+def pod_shard_config(cfg: pod_config, rank: int, world: int):
+    """KV-head split: returns (local config, first KV head, first query head) of ``rank``."""
+    local, kv0, q0 = pod_config(), c_int32(), c_int32()
+    _check(lib.pod_shard_config(ctypes.byref(cfg), rank, world, ctypes.byref(local), ctypes.byref(kv0), ctypes.byref(q0)),
+           "pod_shard_config")
+    return local, kv0.value, q0.value
+
+
+def pod_shard_block_map(cfg: pod_config, lowest_layer, rank: int, world: int):
+    """The rank's columns of a head-wise block map, as a list [n_layers][n_kv_heads / world]."""
+    per = cfg.n_kv_heads // max(world, 1)
+    out = (c_int32 * max(1, cfg.n_layers * per))()
+    _check(lib.pod_shard_block_map(ctypes.byref(cfg), _lowest(cfg, lowest_layer), rank, world, out), "pod_shard_block_map")
+    return [[out[l * per + h] for h in range(per)] for l in range(cfg.n_layers)]
 
 
 class PodCache:
@@ -209,6 +230,13 @@ class PodCache:
 
     def last_cuda_error(self) -> int:
         return lib.pod_cache_last_cuda_error(self._h)
+
+    def set_trace(self, pairs, n_launches: int) -> int:
+        """pairs: int64/uint64 device tensor of 2 * n_launches elements (or None, 0 to switch off)."""
+        return _check(lib.pod_cache_set_trace(self._h, _ptr(pairs), n_launches), "pod_cache_set_trace")
+
+    def trace_count(self) -> int:
+        return lib.pod_cache_trace_count(self._h)
 
     def last_launch(self):
         a, b, c = c_int32(), c_int32(), c_int32()

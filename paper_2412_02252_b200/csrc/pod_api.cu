@@ -149,6 +149,8 @@ struct pod_cache {
   float scale = 0.f;
   Layout y{};
   CUtensorMap tmap{};                  // the region rows of the arena as a [rows][d] bf16 tensor
+  unsigned long long* trace = nullptr; // caller's device buffer of (start, end) pairs, one per kernel launch
+  int trace_cap = 0, trace_n = 0;
   // last launch (diagnostics)
   int32_t last_split_tokens = 0, last_ctas = 0, last_kernels = 0;
   // planner memo
@@ -388,6 +390,33 @@ int pod_greedy_layer_blocks(const float* sim, int n_heads, int n_layers, float t
   return POD_OK;
 }
 
+// Split of one cache over `world` GPUs by KV head: rank r keeps KV heads [r * H_kv / world, (r + 1) * H_kv / world)
+// and the query heads that read them.  Every region is per KV head, so the rank's cache is an ordinary
+// cache of H_kv / world heads; outputs of the ranks are disjoint slices of [B][H_q][d].
+int pod_shard_config(const pod_config* full, int rank, int world, pod_config* local, int32_t* first_kv_head,
+                     int32_t* first_q_head) {
+  if (!config_ok(full) || !local || world < 1 || rank < 0 || rank >= world) return POD_ERR_INVALID;
+  if (full->n_kv_heads % world != 0) return POD_ERR_INVALID;
+  const int per = full->n_kv_heads / world, r = full->n_q_heads / full->n_kv_heads;
+  *local = *full;
+  local->n_kv_heads = per;
+  local->n_q_heads = per * r;
+  if (first_kv_head) *first_kv_head = rank * per;
+  if (first_q_head) *first_q_head = rank * per * r;
+  return POD_OK;
+}
+
+int pod_shard_block_map(const pod_config* full, const int32_t* lowest_layer, int rank, int world,
+                        int32_t* local_lowest_layer) {
+  if (!config_ok(full) || !lowest_layer || !local_lowest_layer || world < 1 || rank < 0 || rank >= world) return POD_ERR_INVALID;
+  if (full->n_kv_heads % world != 0) return POD_ERR_INVALID;
+  const int H = full->n_kv_heads, per = H / world;
+  for (int l = 0; l < full->n_layers; ++l)
+    for (int h = 0; h < per; ++h)
+      local_lowest_layer[(size_t)l * per + h] = lowest_layer[(size_t)l * H + rank * per + h];
+  return POD_OK;
+}
+
 int pod_cache_destroy(pod_cache* c) {
   if (!c) return POD_ERR_INVALID;
   int st = POD_OK;
@@ -547,6 +576,7 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
       p.len = c->d_len(layer);
     }
     if (plan.n_ctas == 0) continue;
+    p.trace = (c->trace != nullptr && c->trace_n < c->trace_cap) ? c->trace + 2 * (size_t)c->trace_n++ : nullptr;
     const int e = launch_decode(c->tmap, p, plan.grid_splits, s);
     if (e != 0) {
       if (fused && pass == 0) { for (int b = 0; b < g.batch; ++b) c->h_len(layer, b) -= 1; c->memo_sum = -1; }
@@ -694,6 +724,27 @@ int pod_cache_inject_error(pod_cache* c) {
   if (e != cudaSuccess) return cuda_fail(c, e);
   return POD_OK;
 }
+
+// Launch trace: the next n_launches kernels of pod_decode_attn / pod_append_decode_attn each record the GPU
+// timer at the start of their first CTA and at the end of their last one.
+int pod_cache_set_trace(pod_cache* c, void* pairs_device, int n_launches) {
+  if (!c || n_launches < 0 || (pairs_device == nullptr) != (n_launches == 0)) return POD_ERR_INVALID;
+  if (((uintptr_t)pairs_device % 8) != 0) return POD_ERR_INVALID;
+  if (c->dry) return POD_DRY_RUN;
+  c->trace = nullptr; c->trace_cap = 0; c->trace_n = 0;
+  if (pairs_device == nullptr) return POD_OK;
+  std::vector<unsigned long long> init((size_t)2 * n_launches);
+  for (int i = 0; i < n_launches; ++i) { init[2 * (size_t)i] = ~0ull; init[2 * (size_t)i + 1] = 0ull; }
+  cudaError_t e = cudaSetDevice(c->cfg.device);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(pairs_device, init.data(), init.size() * 8, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  c->trace = static_cast<unsigned long long*>(pairs_device);
+  c->trace_cap = n_launches;
+  return POD_OK;
+}
+
+int pod_cache_trace_count(const pod_cache* c) { return c ? c->trace_n : POD_ERR_INVALID; }
 
 int pod_cache_last_cuda_error(const pod_cache* c) { return c ? c->last_cuda : (int)cudaErrorInvalidValue; }
 

@@ -125,6 +125,7 @@ struct DecodeParams {
   float* part_ml;          // [B][H_q][max_splits][4]  (running max in log2 units, sum, distant part of the sum, -)
   uint16_t* out;           // [B][H_q][D]
   int32_t* err_flag;
+  unsigned long long* trace;   // nullptr, or this launch's (first CTA start, last CTA end) pair of GPU-timer nanoseconds
   int32_t* sched;          // [B][H_kv][SCHED_STRIDE] zeroed chunk counters and tickets (the kernel re-zeroes them)
   // Gate threshold (paper appendix "Computation Optimization for Distant Tokens"): a gated decode of a
   // layer is two launches.  segment 1 streams the proximal tokens only and evaluates the gate of

@@ -101,6 +101,20 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
+// Launch trace (pod_cache_set_trace): the first CTA to start and the last to finish leave the
+// GPU's nanosecond timer, so that a benchmark can see when consecutive launches of a stream, which
+// overlap, really begin and end.  Two fire-and-forget atomics per CTA, none when the trace is off.
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void trace_begin(const DecodeParams& p) {
+  if (p.trace != nullptr && threadIdx.x == 0) atomicMin(p.trace, global_timer_ns());
+}
+__device__ __forceinline__ void trace_end(const DecodeParams& p) {
+  if (p.trace != nullptr && threadIdx.x == 0) atomicMax(p.trace + 1, global_timer_ns());
+}
 __device__ __forceinline__ float lds_f32(uint32_t a) {
   float v;
   asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a));
@@ -180,6 +194,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);   // swizzle atoms are 1024 B
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  trace_begin(p);
   unsigned char* wbuf = smem + warp * C::WARP_B;
   const uint32_t wbuf_s = smem_u32(wbuf);
   const uint32_t sc0 = smem_u32(smem + C::RING_B) + warp * NSTAGE * C::SC_SLOT_B;   // this warp's logit slots
@@ -677,7 +692,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     }
   }
   __syncthreads();
-  if (!s_last) return;
+  if (!s_last) {
+    trace_end(p);
+    return;
+  }
 
   // ---- combine: every warp merges the partials of its own query heads, on its own -----------
   // The (max, sum) pairs and the partial rows of a head come into the warp's ring with bulk
@@ -805,6 +823,8 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       *reinterpret_cast<__nv_bfloat162*>(dst + j) = __floats2bfloat162_rn(acc[j] * inv, acc[j + 1] * inv);
   }
   if (cfail && lane == 0) atomicExch(p.err_flag, 1);
+  __syncthreads();
+  trace_end(p);
 }
 
 // Outputs of sequences that hold no token are zero (no split CTA exists to write them).

@@ -128,6 +128,7 @@ extern "C" int pod_dense_decode_attn_static(const void* kv_device, int capacity,
   p.part_ml = reinterpret_cast<float*>(su->scratch + OFF_PML);
   p.out = static_cast<uint16_t*>(out_device);
   p.err_flag = reinterpret_cast<int32_t*>(su->scratch + OFF_ERR);
+  p.trace = nullptr;
   p.sched = reinterpret_cast<int32_t*>(su->scratch + OFF_SCHED);
   p.layer = 0; p.split_rows = 2 * split_tokens; p.max_splits = STATIC_MAX_SPLITS;
   p.tiles_per_chunk = split_tokens / (decode_tile_tokens() * decode_warps_per_cta() * 16);
