@@ -230,6 +230,15 @@ int pod_cache_device_status(pod_cache* c);
  * Synchronises the device.  Errors: INVALID, CUDA. */
 int pod_cache_inject_error(pod_cache* c);
 
+/* Test hook (the paper has no counterpart).  Decode launches that follow a decode launch of another layer
+ * of the same cache start "optimistically": they stream with a copy of q read before the stream's
+ * previous kernel is known to have finished, wait for that kernel only before they publish anything, then
+ * read q again and compare; a head in which a copy turned out stale is recomputed by one CTA with a plain
+ * loop (exact, slow).  That path is never taken when q is complete before the call is enqueued, so this
+ * call forces it: the next pod_decode_attn / pod_append_decode_attn (not a gated one) treats every early
+ * copy as stale.  Results must not change.  Errors: INVALID. */
+int pod_cache_inject_stale_query(pod_cache* c);
+
 /* Last CUDA runtime error code seen by this cache (0 if none). */
 int pod_cache_last_cuda_error(const pod_cache* c);
 

@@ -57,6 +57,7 @@ def _load() -> ctypes.CDLL:
         "pod_cache_read_region": (c_int, [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int, c_void_p]),
         "pod_cache_device_status": (c_int, [c_void_p]),
         "pod_cache_inject_error": (c_int, [c_void_p]),
+        "pod_cache_inject_stale_query": (c_int, [c_void_p]),
         "pod_cache_last_cuda_error": (c_int, [c_void_p]),
         "pod_cache_last_launch": (c_int, [c_void_p, P(c_int32), P(c_int32), P(c_int32)]),
         "pod_cache_set_trace": (c_int, [c_void_p, c_void_p, c_int]),
@@ -82,7 +83,8 @@ EXPORTS = ["pod_cache_required_bytes", "pod_cache_create", "pod_cache_required_b
            "pod_cache_create_blocks", "pod_greedy_layer_blocks", "pod_shard_config", "pod_shard_block_map",
            "pod_cache_destroy", "pod_cache_write",
            "pod_decode_attn", "pod_append_decode_attn", "pod_cache_set_gate_threshold", "pod_cache_bytes", "pod_cache_seq_len", "pod_cache_reset",
-           "pod_cache_read_region", "pod_cache_device_status", "pod_cache_inject_error", "pod_cache_last_cuda_error",
+           "pod_cache_read_region", "pod_cache_device_status", "pod_cache_inject_error", "pod_cache_inject_stale_query",
+           "pod_cache_last_cuda_error",
            "pod_cache_last_launch", "pod_cache_set_trace", "pod_cache_trace_count", "pod_strerror", "pod_prefill_attn", "pod_prefill_status", "pod_prefill_inject_error",
            "pod_dense_decode_attn_static", "pod_dense_decode_attn_static_status",
            "pod_dense_decode_attn_static_inject_error"]
@@ -227,6 +229,10 @@ class PodCache:
     def inject_error(self) -> int:
         """Sets the cache's error word from the host (tests of the error path)."""
         return _check(lib.pod_cache_inject_error(self._h), "pod_cache_inject_error")
+
+    def inject_stale_query(self) -> int:
+        """The next decode launch recomputes every head as if its early copy of q had been stale (test hook)."""
+        return _check(lib.pod_cache_inject_stale_query(self._h), "pod_cache_inject_stale_query")
 
     def last_cuda_error(self) -> int:
         return lib.pod_cache_last_cuda_error(self._h)

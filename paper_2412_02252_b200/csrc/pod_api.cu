@@ -142,6 +142,11 @@ struct pod_cache {
   int last_decode_layer = -1;          // layer of the previous launch on this cache if it was a decode launch, else -1
   std::vector<int32_t> score_low;      // [H_kv] lowest layer whose distant logits the head's score store holds, -1 = none
   std::vector<int32_t> score_len;      // [H_kv][B] lengths at which they were stored
+  std::vector<int32_t> score_seq;      // [H_kv] sequence number of the launch that stored them
+  int32_t launch_seq = 0;              // decode kernels launched on this cache so far
+  bool optimistic = true;              // POD_OPTIMISTIC=0 switches the optimistic start off
+  bool closer = true;                  // POD_CLOSER=0: every CTA takes a counted ticket even when the grid fits the GPU
+  bool inject_stale = false;           // pod_cache_inject_stale_query: the next launch treats its early q as stale
   int force_split_tokens = 0;          // POD_SPLIT_TOKENS > 0 overrides the planner
   int force_chunk_tiles = 0;           // POD_CHUNK_TILES > 0 overrides the tiles per draw
   int static_eighths = 5;              // POD_STATIC_EIGHTHS: share of a warp's chunks assigned without a draw
@@ -303,6 +308,7 @@ static int create_impl(const pod_config* cfg, const int32_t* seq_capacity, const
   c->len_cur.assign((size_t)cfg->n_layers, 0);
   c->score_low.assign((size_t)cfg->n_kv_heads, -1);
   c->score_len.assign((size_t)cfg->n_kv_heads * cfg->batch, -1);
+  c->score_seq.assign((size_t)cfg->n_kv_heads, 0);
   c->stash_len.assign((size_t)c->bm.n_slots * cfg->batch, -1);
   c->scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)cfg->head_dim);
   c->dry = cfg->device < 0;
@@ -353,6 +359,8 @@ static int create_impl(const pod_config* cfg, const int32_t* seq_capacity, const
     const int v = atoi(se);
     if (v >= 0 && v <= 8) c->static_eighths = v;
   }
+  if (const char* op = getenv("POD_OPTIMISTIC")) c->optimistic = atoi(op) != 0;
+  if (const char* cl = getenv("POD_CLOSER")) c->closer = atoi(cl) != 0;
   const char* fst = getenv("POD_SPLIT_TOKENS");
   c->force_split_tokens = fst ? atoi(fst) : 0;
   *out = c;
@@ -548,6 +556,7 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     p.v_slot[h] = in ? c->slot_of(layer, h) : 0;
     if (in && c->bm.shared && c->low_of(layer, h) == layer && layer + 1 < g.n_layers && c->low_of(layer + 1, h) == layer)
       p.v_store_mask |= 1u << h;
+    p.v_wait_seq[h] = in ? c->score_seq[h] : 0;
   }
   // With a gate threshold set, a layer in which some head reads its block's logits runs as two
   // launches: the proximal tokens (which decides, per query head, whether the distant tokens are
@@ -576,6 +585,14 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
       p.len = c->d_len(layer);
     }
     if (plan.n_ctas == 0) continue;
+    // Optimistic start: for launches that may start early, of caches with few enough heads that the per-head
+    // sequence numbers travel by value; not for the two launches of a gated layer.
+    p.optimistic = (p.early_ok && !gated && c->optimistic && p.heads_by_value) ? 1 : 0;
+    p.seq = ++c->launch_seq;
+    // every CTA gets a slot on some SM without another CTA of the grid leaving first
+    p.closer = (c->closer && (int64_t)p.y.H_kv * plan.grid_splits * p.y.B <= (int64_t)c->sm_count * c->resident) ? 1 : 0;
+    p.force_redo = (c->inject_stale && !gated) ? 1 : 0;
+    c->inject_stale = false;
     p.trace = (c->trace != nullptr && c->trace_n < c->trace_cap) ? c->trace + 2 * (size_t)c->trace_n++ : nullptr;
     const int e = launch_decode(c->tmap, p, plan.grid_splits, s);
     if (e != 0) {
@@ -598,6 +615,7 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
   for (int h = 0; h < H; ++h) {          // heads whose block starts here and goes on: their logits are stored now
     if (c->low_of(layer, h) != layer || layer + 1 >= g.n_layers || c->low_of(layer + 1, h) != layer) continue;
     c->score_low[h] = layer;
+    c->score_seq[h] = c->launch_seq;
     for (int b = 0; b < g.batch; ++b) c->score_len[(size_t)h * g.batch + b] = c->h_len(layer, b);
   }
   c->last_decode_layer = layer;
@@ -745,6 +763,14 @@ int pod_cache_set_trace(pod_cache* c, void* pairs_device, int n_launches) {
 }
 
 int pod_cache_trace_count(const pod_cache* c) { return c ? c->trace_n : POD_ERR_INVALID; }
+
+// Test hook of the optimistic start: the next decode launch behaves as if every warp had found its early
+// copy of q stale, so every head goes through the recomputation path.  Nothing on the GPU is made to fail.
+int pod_cache_inject_stale_query(pod_cache* c) {
+  if (!c) return POD_ERR_INVALID;
+  c->inject_stale = true;
+  return c->dry ? POD_DRY_RUN : POD_OK;
+}
 
 int pod_cache_last_cuda_error(const pod_cache* c) { return c ? c->last_cuda : (int)cudaErrorInvalidValue; }
 

@@ -30,6 +30,10 @@ constexpr int DECODE_CTAS_PER_SM = POD_DECODE_CTAS_PER_SM;  // register budget o
 constexpr int SCHED_STRIDE = 32;      // int32 per (sequence, KV head)
 constexpr int SCHED_TICKET = 16;      // [0] = chunk counter, [SCHED_TICKET] = finished-CTA tickets
 constexpr int SCHED_NEED = 2;         // [SCHED_NEED] = query heads of this KV head that still need their distant tokens (gate)
+constexpr int SCHED_CTR1 = 4;         // [(seq & 1) * SCHED_CTR1] = chunk counter: launches alternate between two, because a launch
+                                      //   may draw chunks while the previous launch of the cache is still finishing
+constexpr int SCHED_EPOCH = 24;       // sequence number of the last launch whose CTAs of this head have all finished streaming
+                                      //   (its stored logits and stashed queries are complete); own 32-byte sector
 
 // Physical layout of the arena.  All offsets are in rows; one row is one head's d bf16
 // values (128 B at d = 64, 256 B at d = 128), so every region base is 128-byte aligned.
@@ -153,6 +157,20 @@ struct DecodeParams {
   // it when the stored logits are those of the head's block at these lengths), else it scores the
   // block's keys itself.  Bit h & 31 of word h >> 5; heads >= 256 never read stored logits.
   uint32_t score_read_mask[8];
+  // Optimistic start.  Launches of one cache follow each other in a stream with programmatic
+  // dependencies, and the tail of a launch (partials, tickets, the combine of the last CTA of a head)
+  // keeps memory idle.  With optimistic = 1 (implies early_ok) a CTA does not wait for the previous
+  // kernel before it streams: it reads q at once, and only before it publishes anything does it wait
+  // (griddepcontrol.wait), read q again and compare.  q is the one input that the previous kernel of
+  // the stream may still be writing (a projection of the caller's); a warp whose early copy turns out
+  // stale marks its head, and the head's last CTA recomputes it with a plain loop (slow, exact, in
+  // practice never taken).  What this launch needs from an earlier launch of the cache -- the block's
+  // stored logits and stashed queries -- is awaited per head through the head's epoch word instead.
+  int32_t optimistic;
+  int32_t closer;          // 1: every CTA of the grid is resident at once; a head's first CTA combines and waits for the others
+  int32_t seq;             // sequence number of this launch on its cache (chunk-counter parity, epoch)
+  int32_t force_redo;      // test hook set from the host: every warp behaves as if its early copy of q were stale
+  int32_t v_wait_seq[SMALL_HEADS];   // per KV head that reads stored logits: sequence number of the launch that stored them
   int32_t early_ok;        // 1: no unfinished launch writes cache rows this launch streams (the two rows a
                            //    fused launch changes itself aside): tiles may be requested before the
                            //    wait for the previous kernel of the stream

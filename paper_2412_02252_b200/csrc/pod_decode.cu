@@ -51,6 +51,8 @@ namespace {
 
 constexpr int TOK = 16;          // tokens per tile (one mma k-step of P V)
 constexpr uint32_t WAIT_LIMIT = 1u << 20;
+constexpr int REDO_MARK = 1 << 20;     // added to a head's ticket word by a warp whose early copy of q, k or v was stale
+constexpr int EPOCH_POLLS = 1 << 13;   // polls (about 0.3 us apart) of a head's epoch word before falling back to the grid wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -114,6 +116,29 @@ __device__ __forceinline__ void trace_begin(const DecodeParams& p) {
 }
 __device__ __forceinline__ void trace_end(const DecodeParams& p) {
   if (p.trace != nullptr && threadIdx.x == 0) atomicMax(p.trace + 1, global_timer_ns());
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int* a) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_gpu(int* a, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(a), "r"(v) : "memory");
+}
+// A load that may race with a store of the previous kernel (the early copies of q, k, v, checked later),
+// or that must see that kernel's stores after the grid wait: served by the L2, never by an L1 line of this
+// SM (which an earlier load of this kernel may have filled with older data).
+__device__ __forceinline__ uint4 ld_relaxed_u32x4(const void* a) {
+  uint4 v;
+  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(a) : "memory");
+  return v;
+}
+// 16 bytes global -> shared, asynchronously, through the L2 only (cp.async.cg)
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ bool differ(const uint4& a, const uint4& b) {
+  return a.x != b.x || a.y != b.y || a.z != b.z || a.w != b.w;
 }
 __device__ __forceinline__ float lds_f32(uint32_t a) {
   float v;
@@ -180,6 +205,64 @@ struct Cfg {
   static_assert(CROWS >= 8, "a warp's ring must hold a few partial rows for the combine");
   static_assert(WARP_B >= (8 * D + 24) * 4, "merge scratch must fit the warp's ring");
 };
+
+// Recomputation of one (sequence, KV head) by a single CTA with a plain loop over its tokens: the way out
+// for a head in which some warp streamed with a copy of q that the previous kernel of the stream had not
+// finished writing (optimistic start).  Exact and slow (a warp per query head, a token per trip); it reads
+// the final rows of the cache -- every CTA of the head has taken its ticket -- and the final q, and writes
+// what the fast path writes: the output, and for a block's lowest layer the distant logits and their
+// log-sum-exp.
+template <int D>
+__device__ __noinline__ void redo_head(const uint16_t* arena, const uint16_t* q_all, const uint16_t* stash, uint16_t* out,
+                                       float* dlse, float scale_log2, int64_t hq0, int r, int n_p, int n_d, int64_t rowKp,
+                                       int64_t rowVp, int64_t rowKd, int64_t rowVd, unsigned char* sc_base, int sc_group_b,
+                                       bool is_low, bool sc_write, int64_t q_own, int64_t q_st) {
+  // (plain arguments: a reference to the kernel's parameter block would force a copy of it onto the stack)
+  constexpr int CPL = D / 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const __nv_bfloat16* rows = reinterpret_cast<const __nv_bfloat16*>(arena);
+  const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(q_all);
+  const __nv_bfloat16* st = reinterpret_cast<const __nv_bfloat16*>(stash);
+  for (int h = warp; h < r; h += DECODE_WARPS) {
+    float qo[CPL], ql[CPL], acc[CPL];
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) {
+      qo[j] = __bfloat162float(q[q_own + h * D + lane * CPL + j]);
+      ql[j] = is_low ? qo[j] : __bfloat162float(st[q_st + h * D + lane * CPL + j]);
+      acc[j] = 0.f;
+    }
+    float m = -INFINITY, l = 0.f, ld = 0.f;
+    for (int t = 0; t < n_p + n_d; ++t) {
+      const bool dist = t >= n_p;
+      const int64_t kr = dist ? rowKd + (t - n_p) : rowKp + t, vr = dist ? rowVd + (t - n_p) : rowVp + t;
+      float dot = 0.f;
+#pragma unroll
+      for (int j = 0; j < CPL; ++j) dot += (dist ? ql[j] : qo[j]) * __bfloat162float(rows[kr * D + lane * CPL + j]);
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      const float a = dot * scale_log2;
+      if (dist && sc_write && lane == 0) {          // same place as the streaming path: groups of 16 tokens, fragment order
+        const int td = t - n_p, c = td & 15;
+        float* slot = reinterpret_cast<float*>(sc_base + (int64_t)(td >> 4) * sc_group_b + (h * 4 + ((c & 7) >> 1)) * 16) +
+                      ((c >> 3) * 2 + (c & 1));
+        *slot = a;
+      }
+      const float m_new = fmaxf(m, a), alpha = ex2(m - m_new), pr = ex2(a - m_new);
+      m = m_new;
+      l = l * alpha + pr;
+      ld = ld * alpha + (dist ? pr : 0.f);
+#pragma unroll
+      for (int j = 0; j < CPL; ++j) acc[j] = acc[j] * alpha + pr * __bfloat162float(rows[vr * D + lane * CPL + j]);
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    const int64_t hq = hq0 + h;
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(out) + hq * D + lane * CPL;
+#pragma unroll
+    for (int j = 0; j < CPL; j += 2)
+      *reinterpret_cast<__nv_bfloat162*>(dst + j) = __floats2bfloat162_rn(acc[j] * inv, acc[j + 1] * inv);
+    if (sc_write && lane == 0) dlse[hq] = ld > 0.f ? m + __log2f(ld) : -INFINITY;
+  }
+}
 
 template <int D>
 __global__ void __launch_bounds__(DECODE_WARPS * 32, DECODE_CTAS_PER_SM)
@@ -270,6 +353,28 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int k_static = (int)((uint32_t)nchunks / (uint32_t)nwh) * p.static_eighths / 8;   // chunks per warp taken without a draw
   const int dyn_base = k_static * nwh;            // first chunk id that is drawn
   int* sched = p.sched + ((int64_t)b * y.H_kv + kvh) * SCHED_STRIDE;
+  int* ctr = sched + (p.seq & 1) * SCHED_CTR1;    // this launch's chunk counter
+  // Optimistic start (see DecodeParams): no wait for the previous kernel before streaming.  Heads that
+  // must score the block's keys with the stashed queries themselves (their stored logits were
+  // overwritten) are rare and wait as usual.
+  const bool opt = p.optimistic && !waited && (is_low || sc_read);
+  bool late_pending = opt;                        // the grid wait is still to come
+  const int64_t q_own = ((int64_t)b * y.H_q + kvh * r) * D;         // this head's r query rows in q
+  const int64_t q_st = ((int64_t)kslot * y.B + b) * r * D;          // and in the stash of its block
+  constexpr int QS = D + 8;                       // row stride in elements: the fragment reads hit 32 banks
+  __shared__ __align__(16) uint16_t s_q[8 * QS];
+  auto load_q = [&]() {
+    if (warp == 0) {
+      for (int i = lane; i < r * (D / 8); i += 32) {
+        const int h = i / (D / 8), c8 = i % (D / 8);
+        *reinterpret_cast<uint4*>(&s_q[h * QS + c8 * 8]) = ld_relaxed_u32x4(p.q + q_own + h * D + c8 * 8);
+      }
+    }
+  };
+  // q is requested before the tiles when it may be read already (the tile requests of a whole SM would
+  // be served first otherwise): the launch has waited, or starts optimistically
+  const bool q_loaded = waited || opt;
+  if (q_loaded) load_q();
 
   // arena rows of this (sequence, layer, head): tile coordinates of the tensor map
   const int rowKp = (int)(seq_row + prox_row(y, p.layer, 0, kvh));
@@ -284,21 +389,23 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   if (p.segment == 2 && sched[SCHED_NEED] == 0) return;   // every query head of this KV head skipped: no distant work
 
   // ---- the warp's walk over its chunks (all values uniform across the warp) -----------------
-  if (!waited && k_static * tch < NSTAGE) {       // the first tiles need draws: no early start
+  if (!waited && !opt && k_static * tch < NSTAGE) {   // the first tiles need draws: no early start
     pdl_wait();
     pdl_launch_dependents();
     waited = true;
   }
   // A warp's first draw is issued when it enters the last of its fixed chunks (not at the start, where
-  // the draws of all warps of a head would queue up on one counter), and never before the wait: the
-  // previous kernel's last CTA of the head resets the counter.
+  // the draws of all warps of a head would queue up on one counter).  Consecutive launches use different
+  // counters, and a launch starts only after the launch before the previous one has ended (every launch
+  // lets its dependents go only after its own grid wait), so a counter is zero and unused when its launch
+  // starts; without the optimistic start nothing is drawn before the wait all the same.
   unsigned drawn = 0;                             // lane 0: result of the draw issued one chunk ahead
   bool drew = false;
   int c_id, c_t = 0, c_j = 0;
   bool walk_done = false;
   auto first_draw = [&]() {
-    if (!drew && waited && c_j >= k_static - 1) {
-      if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+    if (!drew && (waited || opt) && c_j >= k_static - 1) {
+      if (lane == 0) drawn = (unsigned)atomicAdd(ctr, 1);
       drew = true;
     }
   };
@@ -306,9 +413,9 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     c_id = gw;
     first_draw();
   } else {                                        // (the wait above has happened)
-    if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+    if (lane == 0) drawn = (unsigned)atomicAdd(ctr, 1);
     c_id = dyn_base + (int)__shfl_sync(0xffffffffu, drawn, 0);
-    if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+    if (lane == 0) drawn = (unsigned)atomicAdd(ctr, 1);
     drew = true;
   }
   auto next_tile = [&]() -> int {                 // virtual tile index, or -1 when the head is used up
@@ -321,7 +428,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
         first_draw();
       } else {
         c_id = dyn_base + (int)__shfl_sync(0xffffffffu, drawn, 0);
-        if (lane == 0) drawn = (unsigned)atomicAdd(sched, 1);
+        if (lane == 0) drawn = (unsigned)atomicAdd(ctr, 1);
       }
     }
     const int64_t vt = (int64_t)c_id * tch + c_t;
@@ -383,9 +490,33 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, 0, waited ? 0 : 1);
   }
   if (!waited) {
-    pdl_wait();
-    pdl_launch_dependents();
+    if (!opt) {
+      pdl_wait();
+      pdl_launch_dependents();
+    } else if (sc_read && warp == 0) {
+      // The block's logits (and stashed queries) come from an earlier launch of this cache, possibly the
+      // one still running: its last CTA of this head publishes the launch's sequence number once all of
+      // the head's CTAs have finished streaming.  One lane of the CTA polls (the barrier below passes the
+      // news on).  Bounded; after the limit the grid wait settles it.
+      const int want = p.v_wait_seq[kvh];
+      bool ready = false;
+      for (int it = 0; it < EPOCH_POLLS && !ready; ++it) {
+        int seen = 0;
+        if (lane == 0) seen = ld_acquire_gpu(sched + SCHED_EPOCH);
+        ready = (int)(__shfl_sync(0xffffffffu, seen, 0) - want) >= 0;
+        if (!ready) __nanosleep(128);
+      }
+      if (!ready) {                     // (the grid wait again later, in late_wait, returns at once)
+        pdl_wait();
+        pdl_launch_dependents();
+      }
+    }
+  }
+  if (!q_loaded) load_q();              // (a launch that had to wait first reads q only now)
+  __syncthreads();                      // q in shared memory; the head's logits known to be complete
+  if (!waited) {
     if (lane == 0) {
+      if (opt && sc_read) fence_async_global();     // the logits are read through the async proxy
 #pragma unroll
       for (int s = 0; s < NSTAGE; ++s)
         if (vt_q[s] >= 0) issue(vt_q[s], s, 0, 2);
@@ -395,27 +526,32 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   }
 
   // a head's lowest layer saves its queries for the other layers of the block
-  const int64_t q_own = ((int64_t)b * y.H_q + kvh * r) * D;         // this head's r query rows in q
-  const int64_t q_st = ((int64_t)kslot * y.B + b) * r * D;          // and in the stash of its block
-  if (sc_write && split == 0 && warp == 0 && lane < D / 8) {
-    for (int h = 0; h < r; ++h)
-      *reinterpret_cast<uint4*>(p.stash + q_st + h * D + lane * 8) =
-          *reinterpret_cast<const uint4*>(p.q + q_own + h * D + lane * 8);
-  }
+  auto stash_q = [&]() {
+    if (sc_write && split == 0 && warp == 0 && lane < D / 8) {
+      for (int h = 0; h < r; ++h)
+        *reinterpret_cast<uint4*>(p.stash + q_st + h * D + lane * 8) =
+            *reinterpret_cast<const uint4*>(p.q + q_own + h * D + lane * 8);
+    }
+  };
+  if (!late_pending) stash_q();          // (an optimistic launch stashes after its wait: q may still change)
 
   // ---- per-lane state -------------------------------------------------------------------
   const int qrow = lane >> 2;          // query head (row of S) owned by this lane's quad
   const int qcol = (lane & 3) * 2;     // first of the two columns this lane holds in a fragment
+  // The CTA's copy of its query rows: read once, by warp 0 and past the L1 (when the launch is optimistic
+  // the previous kernel may still be writing q, and the copy is compared with a second reading after the
+  // grid wait: neither reading may come out of a stale L1 line), then shared by the warps.
   uint32_t qp[D / 16][2], qd[D / 16][2];   // A fragments of Q (rows 0..7; rows 8..15 are zero):
   {                                        // own query (proximal tiles), lowest layer's (distant)
-    const uint16_t* qo = p.q + q_own + qrow * D + qcol;
-    const uint16_t* ql = is_low ? qo : p.stash + q_st + qrow * D + qcol;
+    const uint16_t* qo = s_q + qrow * QS + qcol;
+    const uint16_t* ql = p.stash + q_st + qrow * D + qcol;
 #pragma unroll
     for (int kk = 0; kk < D / 16; ++kk) {
       qp[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(qo + kk * 16) : 0u;
       qp[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(qo + kk * 16 + 8) : 0u;
-      qd[kk][0] = qrow < r ? *reinterpret_cast<const uint32_t*>(ql + kk * 16) : 0u;
-      qd[kk][1] = qrow < r ? *reinterpret_cast<const uint32_t*>(ql + kk * 16 + 8) : 0u;
+      // (the stash of a block that started lower is complete: it was awaited above)
+      qd[kk][0] = is_low ? qp[kk][0] : (qrow < r ? *reinterpret_cast<const uint32_t*>(ql + kk * 16) : 0u);
+      qd[kk][1] = is_low ? qp[kk][1] : (qrow < r ? *reinterpret_cast<const uint32_t*>(ql + kk * 16 + 8) : 0u);
     }
   }
   // O^T accumulators: ot[cb][0], [1] = channel cb*16 + qrow of heads qcol, qcol + 1;
@@ -429,7 +565,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   uint32_t round = 0;                     // stage s holds its (round)-th tile: barrier parity round & 1
   int fail_stage = 0;
 
+  uint4 nw_early = make_uint4(0u, 0u, 0u, 0u);     // warp 0 of the head's first CTA: its early copy of the new k / v row
   // ---- fused append: warp 0 of the head's first CTA moves the rows and adds their terms ------
+  // (An optimistic launch does this with copies of k and v read before its wait, like q; they are checked
+  // with q.  Every streaming warp masks the two rows, and the layer's rows are read by no other launch
+  // until the layer's next step, so a stale row harms nobody before the head is redone.)
   if (fused && split == 0 && warp == 0) {
     __shared__ __align__(16) uint16_t s_sp[4][128];     // new K, new V, displaced K, displaced V
     constexpr int LPR = D / 8;                          // lanes per row, 16 bytes each
@@ -438,7 +578,8 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     if (lane < 2 * LPR) {
       const bool isv = lane >= LPR;
       const int sub = lane % LPR;
-      const uint4 nw = *reinterpret_cast<const uint4*>((isv ? p.new_v : p.new_k) + ((int64_t)b * y.H_kv + kvh) * D + sub * 8);
+      const uint4 nw = ld_relaxed_u32x4((isv ? p.new_v : p.new_k) + ((int64_t)b * y.H_kv + kvh) * D + sub * 8);
+      nw_early = nw;
       uint4* slot = reinterpret_cast<uint4*>(arena_w + ((int64_t)(isv ? rowVp : rowKp) + rA) * D + sub * 8);
       if (rB >= 0) {
         // The slot's occupant leaves the window: its value row moves to the layer's distant values,
@@ -504,6 +645,46 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // V (transposed): matrices (tokens 0-7, chunk 2cb), (0-7, 2cb+1), (8-15, 2cb), (8-15, 2cb+1):
   // the A fragments a0..a3 of V^T [16 channels x 16 tokens]
   const int v_tok = (lm >> 1) * 8 + lr, v_chunk = lm & 1;
+
+  // ---- optimistic start: the wait for the previous kernel, and the check of the early copies ----
+  // Called when the warp has requested its last tile (the reads below then hide behind the tiles still in
+  // flight), at the latest after the loop.  Dependents are let go only now, so that the launch after the
+  // next cannot start before the previous one has ended (they would share a chunk counter).
+  // The second reading of q (and of the new k, v rows) goes into a stage the warp no longer needs as an
+  // asynchronous copy (L2 to shared memory), so that nobody waits for it; it is compared after the loop.
+  int check_stage = -1;
+  auto late_wait = [&]() {
+    pdl_wait();
+    pdl_launch_dependents();
+    late_pending = false;
+    if (warp != 0) return;                 // the CTA's copies were made, and are checked, by warp 0
+#pragma unroll
+    for (int s = 0; s < NSTAGE; ++s)
+      if (check_stage < 0 && vt_q[s] < 0) check_stage = s;
+    if (check_stage < 0) return;           // (not reached: the walk is over, so some stage is free)
+    const uint32_t dst = wbuf_s + check_stage * C::STAGE_B;
+    for (int i = lane; i < r * (D / 8); i += 32) cp_async_16(dst + i * 16, p.q + q_own + (int64_t)i * 8);
+    if (fused && split == 0 && lane < D / 4)
+      cp_async_16(dst + 8 * D * 2 + lane * 16,
+                  (lane >= D / 8 ? p.new_v : p.new_k) + ((int64_t)b * y.H_kv + kvh) * D + (lane % (D / 8)) * 8);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  auto late_check = [&]() {                // after the loop: compare, mark the head if a copy was stale
+    if (warp != 0 || check_stage < 0) return;
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    const unsigned char* got = wbuf + check_stage * C::STAGE_B;
+    bool stale = false;
+    for (int i = lane; i < r * (D / 8); i += 32) {
+      const int h = i / (D / 8), c8 = i % (D / 8);
+      stale = stale || differ(*reinterpret_cast<const uint4*>(&s_q[h * QS + c8 * 8]), *reinterpret_cast<const uint4*>(got + i * 16));
+    }
+    if (fused && split == 0 && lane < D / 4)
+      stale = stale || differ(nw_early, *reinterpret_cast<const uint4*>(got + 8 * D * 2 + lane * 16));
+    // a mark is a large number added to the head's ticket word: the CTA that draws the last ticket sees it
+    if (__any_sync(0xffffffffu, stale) && lane == 0) atomicAdd(sched + SCHED_TICKET, REDO_MARK);
+    stash_q();
+  };
 
   for (bool more = true; more && !failed; ++round) {
 #pragma unroll
@@ -621,7 +802,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
                    (s1[1] + t1[1]) * p.scale_log2, min(TOK, rem), mtile, fb, store, dist);
       }
     }
+    if (late_pending && walk_done) late_wait();
   }
+  if (late_pending) late_wait();
+  late_check();
+  if (p.force_redo && p.segment == 0 && threadIdx.x == 0) atomicAdd(sched + SCHED_TICKET, REDO_MARK);
 
   if (failed) {
     if (lane == 0) atomicExch(p.err_flag, 1);
@@ -679,20 +864,66 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // ---- ticket: the CTA that publishes the last partial of this (sequence, KV head) combines ----
   // The barrier orders every thread's partial stores before thread 0's release at GPU scope
   // (cumulative), and the winner's acquire orders them before its reads.
+  // Two forms.  General: every CTA takes a ticket and learns from the returned count whether it is the
+  // last.  When the whole grid is resident at once (the host knows: closer = 1), the head's first CTA is
+  // the one that combines: the others add their ticket without asking for the count and leave at once --
+  // their slot on the SM goes to the next kernel a memory round trip earlier -- and the first CTA waits
+  // (bounded) until the count is complete.  It cannot wait for a CTA that has no slot yet, because in that
+  // mode every CTA of the grid gets one without anyone leaving.
   __shared__ int s_last;
   fence_async_global();                  // the partials are read back through the async proxy
   __syncthreads();
+  if (p.closer && split != 0) {
+    if (threadIdx.x == 0)
+      asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(sched + SCHED_TICKET) : "memory");
+    trace_end(p);
+    return;
+  }
   if (threadIdx.x == 0) {
     int got;
-    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(got) : "l"(sched + SCHED_TICKET) : "memory");
-    s_last = (got == nsplit - 1);
-    if (s_last) {                                            // ready for the next launch
-      sched[SCHED_TICKET] = 0; sched[0] = 0;
-      if (p.segment == 1) sched[SCHED_NEED] = 0;             // this CTA's warps set the bits below
+    if (p.closer) {
+      got = 0;
+      bool all = nsplit == 1;
+      for (uint32_t it = 0; it < WAIT_LIMIT && !all; ++it) {
+        got = ld_acquire_gpu(sched + SCHED_TICKET);
+        all = (got & (REDO_MARK - 1)) == nsplit - 1;
+        if (!all) __nanosleep(64);
+      }
+      if (!all) atomicExch(p.err_flag, 1);                   // (the outputs of this head are then invalid)
+      if (nsplit == 1) got = ld_acquire_gpu(sched + SCHED_TICKET);   // this CTA's own marks
+    } else {
+      asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(got) : "l"(sched + SCHED_TICKET) : "memory");
     }
+    int last = (p.closer || (got & (REDO_MARK - 1)) == nsplit - 1) ? 1 : 0;
+    if (last) {                                              // ready for the next launch
+      sched[SCHED_TICKET] = 0; *ctr = 0;
+      if (p.segment == 1) sched[SCHED_NEED] = 0;             // this CTA's warps set the bits below
+      // Every CTA of the head has finished streaming: its stored logits, stashed queries and cache rows are
+      // complete, which is what a later launch waits for -- unless a warp found its early copies stale (it added
+      // its mark to this word before its CTA took its ticket); then the head is redone first.
+      if (got >= REDO_MARK) last = 2;
+      else st_release_gpu(sched + SCHED_EPOCH, p.seq);
+    }
+    s_last = last;
   }
   __syncthreads();
   if (!s_last) {
+    trace_end(p);
+    return;
+  }
+  if (s_last == 2) {
+    if (fused && warp == 0 && lane < D / 4) {     // the new token's rows again, from the final k and v
+      const bool isv = lane >= D / 8;
+      const int sub = lane % (D / 8);
+      *reinterpret_cast<uint4*>(const_cast<uint16_t*>(p.arena) + ((int64_t)(isv ? rowVp : rowKp) + rA) * D + sub * 8) =
+          *reinterpret_cast<const uint4*>((isv ? p.new_v : p.new_k) + ((int64_t)b * y.H_kv + kvh) * D + sub * 8);
+    }
+    __syncthreads();
+    redo_head<D>(p.arena, p.q, p.stash, p.out, p.dlse, p.scale_log2, (int64_t)b * y.H_q + kvh * r, r, n_p, n_d, rowKp, rowVp,
+                 rowKd, rowVd, sc_base, sc_group_b, is_low, sc_write, q_own, q_st);
+    fence_async_global();
+    __syncthreads();
+    if (threadIdx.x == 0) st_release_gpu(sched + SCHED_EPOCH, p.seq);
     trace_end(p);
     return;
   }

@@ -504,3 +504,41 @@ def test_cache_error_word_is_reported_once_and_decoding_goes_on():
     for l in range(2):
         for h in range(8):
             assert_close(outs[l, 0, h], case.oracle_head(l, 0, h), f"layer {l} head {h} after the injected error")
+
+
+@pytest.mark.parametrize("d,G,Hq,Hkv", [(128, 2, 8, 2), (64, 3, 8, 1)])
+def test_stale_query_path_recomputes_heads_exactly(d, G, Hq, Hkv):
+    """Launches that follow a decode launch of another layer stream with an early copy of q and check it
+    after waiting for the stream's previous kernel; a head whose copy was stale is recomputed by one CTA.
+    The test forces that path from the host (pod_cache_inject_stale_query) for lowest layers (which also
+    store the distant logits that the block's next layers then consume) and for sharing layers, over
+    steps that fill the sink, fill the ring and wrap it: outputs against the oracle, cache contents bit
+    for bit against the oracle's layout."""
+    S, W = 4, 16
+    lens0 = [70, 3, 21]
+    case = Case(seed=23, L=6, G=G, Hq=Hq, Hkv=Hkv, d=d, S=S, W=W, lens=lens0, caps=[n + 24 for n in lens0])
+    cache = case.make_cache()
+    case.prefill(cache)
+    ocs = [_oracle_cache(case, b) for b in range(case.B)]
+    for b, oc in enumerate(ocs):
+        for l in range(case.L):
+            oc.write(l, synth.bf16_bits(case.kv(synth.TAG_K, l, b, 0, lens0[b], "cpu")),
+                     synth.bf16_bits(case.kv(synth.TAG_V, l, b, 0, lens0[b], "cpu")))
+    stream = torch.cuda.current_stream().cuda_stream
+    for step in range(1, 24):
+        lens = [n + step for n in lens0]
+        outs = torch.empty(case.L, case.B, case.Hq, case.d, dtype=torch.bfloat16, device="cuda")
+        for l in range(case.L):
+            k = torch.stack([case.kv(synth.TAG_K, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            v = torch.stack([case.kv(synth.TAG_V, l, b, lens[b] - 1, lens[b], "cuda")[0] for b in range(case.B)])
+            if (step + l) % 3 == 0:                     # lowest and sharing layers alike, a different set every step
+                cache.inject_stale_query()
+            cache.append_decode_attn(l, k, v, case.q(l, step, "cuda"), outs[l], stream)
+            kb, vb = synth.bf16_bits(k), synth.bf16_bits(v)
+            for b, oc in enumerate(ocs):
+                oc.append(l, kb[b], vb[b])
+        torch.cuda.synchronize()
+        _check_all_heads(case, outs, step=step, lens=lens)
+        if step in (1, 2, 13, 14, 23):
+            _compare_layout(case, cache, ocs)
+    assert cache.device_status() == B.POD_OK
