@@ -143,6 +143,8 @@ struct pod_cache {
   std::vector<int32_t> score_low;      // [H_kv] lowest layer whose distant logits the head's score store holds, -1 = none
   std::vector<int32_t> score_len;      // [H_kv][B] lengths at which they were stored
   std::vector<int32_t> score_seq;      // [H_kv] sequence number of the launch that stored them
+  std::vector<uint32_t> done_total;    // [B][H_kv] what the head's DONE word reads when all launches so far are through with it
+  std::vector<uint32_t> score_done;    // [B][H_kv] done_total right after the launch that stored the head's logits
   int32_t launch_seq = 0;              // decode kernels launched on this cache so far
   bool optimistic = true;              // POD_OPTIMISTIC=0 switches the optimistic start off
   bool closer = true;                  // POD_CLOSER=0: every CTA takes a counted ticket even when the grid fits the GPU
@@ -309,6 +311,8 @@ static int create_impl(const pod_config* cfg, const int32_t* seq_capacity, const
   c->score_low.assign((size_t)cfg->n_kv_heads, -1);
   c->score_len.assign((size_t)cfg->n_kv_heads * cfg->batch, -1);
   c->score_seq.assign((size_t)cfg->n_kv_heads, 0);
+  c->done_total.assign((size_t)cfg->n_kv_heads * cfg->batch, 0u);
+  c->score_done.assign((size_t)cfg->n_kv_heads * cfg->batch, 0u);
   c->stash_len.assign((size_t)c->bm.n_slots * cfg->batch, -1);
   c->scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)cfg->head_dim);
   c->dry = cfg->device < 0;
@@ -545,8 +549,6 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     p.v_len[b] = in ? c->h_len(layer, b) : 0;
     p.v_cap_d[b] = in ? c->cv.seq_cap_d[b] : 0;
     p.v_row_base[b] = in ? c->cv.seq_row_base[b] : 0;
-    const int32_t pos = p.v_len[b] - 1;
-    p.v_ring_slot[b] = (in && pos >= g.n_sink) ? (pos - g.n_sink) % g.n_recent : 0;
   }
   p.heads_by_value = H <= SMALL_HEADS ? 1 : 0;
   p.v_store_mask = 0u;
@@ -556,7 +558,6 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     p.v_slot[h] = in ? c->slot_of(layer, h) : 0;
     if (in && c->bm.shared && c->low_of(layer, h) == layer && layer + 1 < g.n_layers && c->low_of(layer + 1, h) == layer)
       p.v_store_mask |= 1u << h;
-    p.v_wait_seq[h] = in ? c->score_seq[h] : 0;
   }
   // With a gate threshold set, a layer in which some head reads its block's logits runs as two
   // launches: the proximal tokens (which decides, per query head, whether the distant tokens are
@@ -570,10 +571,33 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     plan = plan_decode(c, layer, n_light, p.segment);
     p.split_rows = plan.split_rows;
     {
-      // A warp sees about split_rows / (2 x tile tokens x warps) tiles; it should make a dozen draws.
-      int tch = plan.split_rows / (2 * decode_tile_tokens() * decode_warps_per_cta() * 16);
+      // A warp sees about split_rows / (2 x tile tokens x warps) tiles; it should make a dozen draws, of two
+      // tiles at least (consecutive rows; measured: 0.9 us per launch at 32K against single tiles) unless it
+      // has only a handful of tiles.
+      const int per_warp = plan.split_rows / (2 * decode_tile_tokens() * decode_warps_per_cta());
+      int tch = per_warp / 16;
+      if (tch < 2 && per_warp >= 6) tch = 2;
       if (c->force_chunk_tiles > 0) tch = c->force_chunk_tiles;
       p.tiles_per_chunk = tch < 1 ? 1 : (tch > 256 ? 256 : tch);
+    }
+    // Small launches carry the plan of every (sequence, KV head) by value.
+    p.plans_by_value = (g.batch * H <= SMALL_PLANS) ? 1 : 0;
+    if (p.plans_by_value) {
+      PlanInputs in;
+      in.layer = layer; in.segment = p.segment; in.fused = (fused && pass == 0) ? 1 : 0; in.max_splits = p.max_splits;
+      in.split_rows = p.split_rows; in.tiles_per_chunk = p.tiles_per_chunk; in.static_eighths = p.static_eighths;
+      in.tile_tokens = decode_tile_tokens(); in.warps = decode_warps_per_cta();
+      for (int b = 0; b < g.batch; ++b)
+        for (int h = 0; h < H; ++h) {
+          const int low = c->low_of(layer, h);
+          const bool store = c->bm.shared && low == layer && layer + 1 < g.n_layers && c->low_of(layer + 1, h) == layer;
+          const bool read = low != layer && h < 256 && ((p.score_read_mask[h >> 5] >> (h & 31)) & 1u);
+          HeadPlan& hp = p.v_plan[b * H + h];
+          hp = make_head_plan(p.y, in, h, c->h_len(layer, b), c->cv.seq_cap_d[b], c->cv.seq_row_base[b], low,
+                              c->slot_of(layer, h), store, read);
+          hp.wait_done = (int32_t)c->score_done[(size_t)b * H + h];
+          hp.wait_seq = c->score_seq[h];
+        }
     }
     // A launch that appends and attends streams only rows written before this step (the new token's
     // and the displaced token's rows are handled apart); the one launch that may still be running is
@@ -587,7 +611,7 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     if (plan.n_ctas == 0) continue;
     // Optimistic start: for launches that may start early, of caches with few enough heads that the per-head
     // sequence numbers travel by value; not for the two launches of a gated layer.
-    p.optimistic = (p.early_ok && !gated && c->optimistic && p.heads_by_value) ? 1 : 0;
+    p.optimistic = (p.early_ok && !gated && c->optimistic && p.plans_by_value) ? 1 : 0;
     p.seq = ++c->launch_seq;
     // every CTA gets a slot on some SM without another CTA of the grid leaving first
     p.closer = (c->closer && (int64_t)p.y.H_kv * plan.grid_splits * p.y.B <= (int64_t)c->sm_count * c->resident) ? 1 : 0;
@@ -601,6 +625,9 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     }
     ++kernels;
     if (fused && pass == 0) c->len_cur[layer] ^= 1;
+    if (p.plans_by_value)                 // every CTA of a head that stores its logits adds one to the head's DONE word
+      for (int i = 0; i < g.batch * H; ++i)
+        if (p.v_plan[i].flags & HP_STORE) c->done_total[i] += (uint32_t)p.v_plan[i].nsplit;
   }
   {
     bool any_empty = false;
@@ -616,6 +643,7 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     if (c->low_of(layer, h) != layer || layer + 1 >= g.n_layers || c->low_of(layer + 1, h) != layer) continue;
     c->score_low[h] = layer;
     c->score_seq[h] = c->launch_seq;
+    for (int b = 0; b < g.batch; ++b) c->score_done[(size_t)b * H + h] = c->done_total[(size_t)b * H + h];
     for (int b = 0; b < g.batch; ++b) c->score_len[(size_t)h * g.batch + b] = c->h_len(layer, b);
   }
   c->last_decode_layer = layer;

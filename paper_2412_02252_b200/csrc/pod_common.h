@@ -32,6 +32,8 @@ constexpr int SCHED_TICKET = 16;      // [0] = chunk counter, [SCHED_TICKET] = f
 constexpr int SCHED_NEED = 2;         // [SCHED_NEED] = query heads of this KV head that still need their distant tokens (gate)
 constexpr int SCHED_CTR1 = 4;         // [(seq & 1) * SCHED_CTR1] = chunk counter: launches alternate between two, because a launch
                                       //   may draw chunks while the previous launch of the cache is still finishing
+constexpr int SCHED_DONE = 28;        // CTAs of this head, over all launches that store logits, whose warps have finished streaming
+constexpr int SCHED_POISON = 29;      // highest sequence number of a launch in which a CTA of this head found its copy of q stale
 constexpr int SCHED_EPOCH = 24;       // sequence number of the last launch whose CTAs of this head have all finished streaming
                                       //   (its stored logits and stashed queries are complete); own 32-byte sector
 
@@ -103,6 +105,74 @@ __host__ __device__ inline int64_t score_row(const Layout& y, int head, int64_t 
          head * score_rows_per_head(y, cap_d);
 }
 
+// What one (sequence, KV head) of a decode launch needs to know before it can request its first tile.
+// The same function fills it on the host (small launches: it then travels by value with the launch, so
+// that a CTA's first requests are a handful of instructions away from its start) and on the device.
+struct HeadPlan {
+  int32_t n, n_p, n_d;                     // tokens held, proximal, distant
+  int32_t ntp, ntd;                        // tiles of the proximal / distant tokens this launch streams
+  int32_t nsplit, k_static;                // CTAs of the head; chunks per warp taken without a draw
+  int32_t rowKp, rowVp, rowKd, rowVd;      // arena rows: proximal keys / values, the block's distant keys, distant values
+  int32_t score_row;                       // arena row where the head's stored logits start
+  int32_t kslot;                           // key store (and query stash) of the head's block
+  int32_t flags;                           // HP_*
+  int32_t rA, rB;                          // a launch that appends: proximal row of the new token, distant row of the
+                                           // token it pushes out of the window (-1 = none)
+  int32_t wait_done, wait_seq;             // a head that reads stored logits: what its DONE word reads once the launch
+                                           // that stored them is through with the head, and that launch's sequence number
+};
+constexpr int HP_LOW = 1;                  // this layer is the lowest of the head's block
+constexpr int HP_STORE = 2;                // ... and the block goes on: the head stores its distant logits
+constexpr int HP_READ = 4;                 // the head reads its block's stored logits instead of the keys
+constexpr int SMALL_PLANS = 16;            // launches with up to this many (sequence, KV head) pairs carry their plans
+
+struct PlanInputs {                        // per launch
+  int32_t layer, segment, fused, max_splits, split_rows, tiles_per_chunk, static_eighths, tile_tokens, warps;
+};
+__host__ __device__ inline HeadPlan make_head_plan(const Layout& y, const PlanInputs& in, int kvh, int n, int64_t cap_d,
+                                                   int64_t seq_row, int low_layer, int kslot, bool store, bool read) {
+  HeadPlan hp;
+  const int TOKS = in.tile_tokens;
+  hp.n = n;
+  hp.n_p = n < y.S + y.W ? n : y.S + y.W;
+  hp.n_d = n - hp.n_p;
+  // a gated decode streams the proximal tokens (segment 1) and the distant tokens (segment 2) in two launches
+  const int n_p_s = in.segment == 2 ? 0 : hp.n_p, n_d_s = in.segment == 1 ? 0 : hp.n_d;
+  const bool is_low = low_layer == in.layer;
+  hp.flags = (is_low ? HP_LOW : 0) | (store ? HP_STORE : 0) | (read ? HP_READ : 0);
+  hp.kslot = kslot;
+  // CTAs of this head: in proportion to the rows it streams (keys and values, or values and the
+  // proximal keys only), so that heads with different roles in one launch finish together.
+  // (a head's rows are a fraction of the arena's, which number less than 2^31: 32-bit arithmetic)
+  const uint32_t work_rows = read ? (uint32_t)n_p_s * 2u + (uint32_t)n_d_s : 2u * ((uint32_t)n_p_s + (uint32_t)n_d_s);
+  const uint32_t ns = (work_rows + (uint32_t)in.split_rows - 1u) / (uint32_t)in.split_rows;
+  hp.nsplit = (int32_t)(ns < (uint32_t)in.max_splits ? ns : (uint32_t)in.max_splits);
+  // A head that reads stored logits needs no key rows: its distant tiles hold twice the value rows
+  const int DT = read ? 2 * TOKS : TOKS;
+  hp.ntp = (n_p_s + TOKS - 1) / TOKS;
+  hp.ntd = (n_d_s + DT - 1) / DT;
+  const uint32_t nchunks = (uint32_t)(hp.ntp + hp.ntd + in.tiles_per_chunk - 1) / (uint32_t)in.tiles_per_chunk;
+  const uint32_t nwh = (uint32_t)(hp.nsplit > 0 ? hp.nsplit : 1) * (uint32_t)in.warps;
+  hp.k_static = (int32_t)(nchunks / nwh) * in.static_eighths / 8;
+  hp.rowKp = (int32_t)(seq_row + prox_row(y, in.layer, 0, kvh));
+  hp.rowVp = (int32_t)(seq_row + prox_row(y, in.layer, 1, kvh));
+  hp.rowKd = (int32_t)(seq_row + distk_row(y, kslot, cap_d));
+  hp.rowVd = (int32_t)(seq_row + distv_row(y, in.layer, kvh, cap_d));
+  hp.score_row = (int32_t)(seq_row + score_row(y, kvh, cap_d));
+  hp.wait_done = 0; hp.wait_seq = 0;
+  hp.rA = -1; hp.rB = -1;
+  if (in.fused) {
+    const int pos = n - 1;
+    if (pos < y.S) {
+      hp.rA = pos;
+    } else {
+      hp.rA = y.S + (pos - y.S) % y.W;
+      if (pos - y.W >= y.S) hp.rB = pos - y.W - y.S;
+    }
+  }
+  return hp;
+}
+
 struct WriteParams {
   Layout y;
   uint16_t* arena;       // bf16 bit patterns
@@ -170,14 +240,12 @@ struct DecodeParams {
   int32_t closer;          // 1: every CTA of the grid is resident at once; a head's first CTA combines and waits for the others
   int32_t seq;             // sequence number of this launch on its cache (chunk-counter parity, epoch)
   int32_t force_redo;      // test hook set from the host: every warp behaves as if its early copy of q were stale
-  int32_t v_wait_seq[SMALL_HEADS];   // per KV head that reads stored logits: sequence number of the launch that stored them
   int32_t early_ok;        // 1: no unfinished launch writes cache rows this launch streams (the two rows a
                            //    fused launch changes itself aside): tiles may be requested before the
                            //    wait for the previous kernel of the stream
   int32_t by_value;        // 1: use the arrays below instead of len / seq_row_base / seq_cap_d
   int32_t v_len[SMALL_BATCH];
   int32_t v_cap_d[SMALL_BATCH];
-  int32_t v_ring_slot[SMALL_BATCH];   // (v_len - 1 - S) mod W: ring slot of the sequence's last token (0 if it is a sink)
   int64_t v_row_base[SMALL_BATCH];
   // Few KV heads: this layer's rows of the block tables by value (low[layer][h], slot[layer][h]) and the
   // heads that store their distant logits in this launch (lowest layer of a block that goes on).
@@ -185,6 +253,8 @@ struct DecodeParams {
   int32_t v_low[SMALL_HEADS];
   int32_t v_slot[SMALL_HEADS];
   uint32_t v_store_mask;
+  int32_t plans_by_value;                  // 1: v_plan[b * H_kv + h] holds the plan of every (sequence, KV head)
+  HeadPlan v_plan[SMALL_PLANS];
 };
 
 struct DecodePlan {

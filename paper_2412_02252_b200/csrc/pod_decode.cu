@@ -315,42 +315,43 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   }
 
   // ---- tiles and chunks of this (sequence, KV head) -----------------------------------------
-  const int n_p = min(n, y.S + y.W), n_d = n - n_p;
-  // a gated decode streams the proximal tokens (segment 1) and the distant tokens (segment 2) in two launches
-  const int n_p_s = p.segment == 2 ? 0 : n_p, n_d_s = p.segment == 1 ? 0 : n_d;
-  // A layer that reads the block's stored logits needs no key rows: its distant tiles hold 32
-  // value rows (both halves of a stage), so the bytes in flight per stage stay the same.
-  // blocks are per KV head: is this layer the lowest of this head's block, and does the block go on?
-  // (with few KV heads the host passes this layer's rows of the block tables by value: no global load
-  // stands between a CTA's start and its first tile requests)
-  int low_layer, kslot;
-  bool sc_write;
-  if (p.heads_by_value) {
-    low_layer = p.v_low[kvh];
-    kslot = p.v_slot[kvh];
-    sc_write = (p.v_store_mask >> kvh) & 1u;
+  // The plan comes with the launch when the launch is small (no arithmetic and no load between a CTA's
+  // start and its first tile requests); otherwise it is worked out here, by the same function.
+  HeadPlan hp;
+  if (p.plans_by_value) {
+    hp = p.v_plan[b * y.H_kv + kvh];
   } else {
-    low_layer = lowest_of(y, p.layer, kvh);
-    kslot = slot_of(y, p.layer, kvh);
-    sc_write = y.shared && low_layer == p.layer && p.layer + 1 < y.L && lowest_of(y, p.layer + 1, kvh) == p.layer;
+    int low_layer, kslot_;
+    bool store;
+    if (p.heads_by_value) {
+      low_layer = p.v_low[kvh];
+      kslot_ = p.v_slot[kvh];
+      store = (p.v_store_mask >> kvh) & 1u;
+    } else {
+      low_layer = lowest_of(y, p.layer, kvh);
+      kslot_ = slot_of(y, p.layer, kvh);
+      store = y.shared && low_layer == p.layer && p.layer + 1 < y.L && lowest_of(y, p.layer + 1, kvh) == p.layer;
+    }
+    const bool read = low_layer != p.layer && kvh < 256 && ((p.score_read_mask[kvh >> 5] >> (kvh & 31)) & 1u);
+    PlanInputs in;
+    in.layer = p.layer; in.segment = p.segment; in.fused = fused ? 1 : 0; in.max_splits = p.max_splits;
+    in.split_rows = p.split_rows; in.tiles_per_chunk = p.tiles_per_chunk; in.static_eighths = p.static_eighths;
+    in.tile_tokens = TOK; in.warps = NW;
+    hp = make_head_plan(y, in, kvh, n, cap_d, seq_row, low_layer, kslot_, store, read);
   }
-  const bool is_low = low_layer == p.layer;
-  const bool sc_read = !is_low && kvh < 256 && ((p.score_read_mask[kvh >> 5] >> (kvh & 31)) & 1u);
-  // CTAs of this head: in proportion to the rows it streams (keys and values, or values and the
-  // proximal keys only), so that heads with different roles in one launch finish together.
-  // (a head's rows are a fraction of the arena's, which number less than 2^31: 32-bit arithmetic)
-  const uint32_t work_rows = sc_read ? (uint32_t)n_p_s * 2u + (uint32_t)n_d_s : 2u * ((uint32_t)n_p_s + (uint32_t)n_d_s);
-  const int nsplit = (int)min((uint32_t)p.max_splits, (work_rows + (uint32_t)p.split_rows - 1u) / (uint32_t)p.split_rows);
+  const int n_p = hp.n_p, n_d = hp.n_d;
+  const int kslot = hp.kslot;
+  const bool is_low = hp.flags & HP_LOW, sc_write = hp.flags & HP_STORE, sc_read = hp.flags & HP_READ;
+  const int nsplit = hp.nsplit;
   if (split >= nsplit) return;
   const int DT_SH = sc_read ? 5 : 4;              // log2 of the tokens per distant tile
   const int DT = 1 << DT_SH;
-  const int ntp = (n_p_s + TOK - 1) / TOK, ntd = (n_d_s + DT - 1) >> DT_SH;
+  const int ntp = hp.ntp, ntd = hp.ntd;
   const int ntiles = ntp + ntd;
   const int tch = p.tiles_per_chunk;
   const int nwh = nsplit * NW;                    // warps working on this head
   const int gw = split * NW + warp;               // this warp's index among them
-  const int nchunks = (int)((uint32_t)(ntiles + tch - 1) / (uint32_t)tch);
-  const int k_static = (int)((uint32_t)nchunks / (uint32_t)nwh) * p.static_eighths / 8;   // chunks per warp taken without a draw
+  const int k_static = hp.k_static;               // chunks per warp taken without a draw
   const int dyn_base = k_static * nwh;            // first chunk id that is drawn
   int* sched = p.sched + ((int64_t)b * y.H_kv + kvh) * SCHED_STRIDE;
   int* ctr = sched + (p.seq & 1) * SCHED_CTR1;    // this launch's chunk counter
@@ -377,14 +378,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   if (q_loaded) load_q();
 
   // arena rows of this (sequence, layer, head): tile coordinates of the tensor map
-  const int rowKp = (int)(seq_row + prox_row(y, p.layer, 0, kvh));
-  const int rowVp = (int)(seq_row + prox_row(y, p.layer, 1, kvh));
-  const int rowKd = (int)(seq_row + distk_row(y, kslot, cap_d));
-  const int rowVd = (int)(seq_row + distv_row(y, p.layer, kvh, cap_d));
+  const int rowKp = hp.rowKp, rowVp = hp.rowVp, rowKd = hp.rowKd, rowVd = hp.rowVd;
   // shared distant logits of this head: groups of 16 tokens x r heads, fp32, fragment order
   const int sc_group_b = score_group_bytes(y);
-  unsigned char* sc_base = reinterpret_cast<unsigned char*>(const_cast<uint16_t*>(p.arena)) +
-                           (seq_row + score_row(y, kvh, cap_d)) * (int64_t)(D * 2);
+  unsigned char* sc_base = reinterpret_cast<unsigned char*>(const_cast<uint16_t*>(p.arena)) + (int64_t)hp.score_row * (D * 2);
 
   if (p.segment == 2 && sched[SCHED_NEED] == 0) return;   // every query head of this KV head skipped: no distant work
 
@@ -470,40 +467,52 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // Rows that change in a fused launch are masked in the streamed tiles and added by one warp
   // from registers: the new token's proximal row, and the distant row of the token it pushes
   // out of the recent window.
-  int tA = -1, cA = 0, tB = -1, cB = 0, rA = -1, rB = -1;
+  int tA = -1, cA = 0, tB = -1, cB = 0;
+  const int rA = hp.rA, rB = hp.rB;
   if (fused) {
-    const int pos = n - 1;
-    if (pos < y.S) {
-      rA = pos;
-    } else {
-      rA = y.S + (p.by_value ? p.v_ring_slot[bv] : (pos - y.S) % y.W);
-      if (pos - y.W >= y.S) rB = pos - y.W - y.S;
-    }
     tA = rA / TOK; cA = rA % TOK;
-    if (rB >= 0) { tB = ntp + rB / DT; cB = rB % DT; }
+    if (rB >= 0) { tB = ntp + (rB >> DT_SH); cB = rB & (DT - 1); }
   }
 
+  // The block's logits (and stashed queries) come from an earlier launch of this cache, possibly the one
+  // still running.  Every CTA of that launch adds one to the head's DONE word when its warps have finished
+  // streaming (all logits of theirs are stored); the host knows what the word reads once the head is
+  // complete.  If a CTA of that launch found its copy of q stale, the logits are rewritten by the head's
+  // recomputation, which the head's epoch word announces: the POISON word says whether to wait for that.
+  auto scores_complete = [&]() -> bool {          // lane 0's view, passed to the warp
+    int ok = 0;
+    if (lane == 0) {
+      ok = (int)(ld_acquire_gpu(sched + SCHED_DONE) - hp.wait_done) >= 0;
+      if (ok && (int)(ld_acquire_gpu(sched + SCHED_POISON) - hp.wait_seq) >= 0)
+        ok = (int)(ld_acquire_gpu(sched + SCHED_EPOCH) - hp.wait_seq) >= 0;
+    }
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+  };
+  // An optimistic launch that reads stored logits looks before its tile requests go out (behind them an
+  // answer takes microseconds).  CTAs that start after the head is complete then request whole tiles at
+  // once and never poll; the others request one stage (values only) and poll.
+  const bool scores_done = opt && sc_read && scores_complete();
+  if (scores_done && lane == 0) fence_async_global();       // the logits are read through the async proxy
+  const int n_prime = (opt && sc_read && !scores_done) ? 1 : NSTAGE;
   int vt_q[NSTAGE];                               // tile held by each stage, -1 = none
 #pragma unroll
   for (int s = 0; s < NSTAGE; ++s) {
-    vt_q[s] = next_tile();
-    if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, 0, waited ? 0 : 1);
+    vt_q[s] = -1;
+    if (s < n_prime) {
+      vt_q[s] = next_tile();
+      if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, 0, (waited || scores_done) ? 0 : 1);
+    }
   }
   if (!waited) {
     if (!opt) {
       pdl_wait();
       pdl_launch_dependents();
-    } else if (sc_read && warp == 0) {
-      // The block's logits (and stashed queries) come from an earlier launch of this cache, possibly the
-      // one still running: its last CTA of this head publishes the launch's sequence number once all of
-      // the head's CTAs have finished streaming.  One lane of the CTA polls (the barrier below passes the
-      // news on).  Bounded; after the limit the grid wait settles it.
-      const int want = p.v_wait_seq[kvh];
+    } else if (sc_read && warp == 0 && !scores_done) {
+      // One warp of the CTA polls (the barrier below passes the news on).  Bounded; after the limit the
+      // grid wait settles it.
       bool ready = false;
       for (int it = 0; it < EPOCH_POLLS && !ready; ++it) {
-        int seen = 0;
-        if (lane == 0) seen = ld_acquire_gpu(sched + SCHED_EPOCH);
-        ready = (int)(__shfl_sync(0xffffffffu, seen, 0) - want) >= 0;
+        ready = scores_complete();
         if (!ready) __nanosleep(128);
       }
       if (!ready) {                     // (the grid wait again later, in late_wait, returns at once)
@@ -515,14 +524,20 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   if (!q_loaded) load_q();              // (a launch that had to wait first reads q only now)
   __syncthreads();                      // q in shared memory; the head's logits known to be complete
   if (!waited) {
-    if (lane == 0) {
+    if (lane == 0 && !scores_done) {
       if (opt && sc_read) fence_async_global();     // the logits are read through the async proxy
 #pragma unroll
       for (int s = 0; s < NSTAGE; ++s)
-        if (vt_q[s] >= 0) issue(vt_q[s], s, 0, 2);
+        if (s < n_prime && vt_q[s] >= 0) issue(vt_q[s], s, 0, 2);
     }
     waited = true;
     first_draw();
+#pragma unroll
+    for (int s = 0; s < NSTAGE; ++s)
+      if (s >= n_prime) {
+        vt_q[s] = next_tile();
+        if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, 0, 0);
+      }
   }
 
   // a head's lowest layer saves its queries for the other layers of the block
@@ -682,7 +697,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     if (fused && split == 0 && lane < D / 4)
       stale = stale || differ(nw_early, *reinterpret_cast<const uint4*>(got + 8 * D * 2 + lane * 16));
     // a mark is a large number added to the head's ticket word: the CTA that draws the last ticket sees it
-    if (__any_sync(0xffffffffu, stale) && lane == 0) atomicAdd(sched + SCHED_TICKET, REDO_MARK);
+    if (__any_sync(0xffffffffu, stale) && lane == 0) {
+      atomicMax(sched + SCHED_POISON, p.seq);
+      atomicAdd(sched + SCHED_TICKET, REDO_MARK);
+    }
     stash_q();
   };
 
@@ -806,7 +824,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   }
   if (late_pending) late_wait();
   late_check();
-  if (p.force_redo && p.segment == 0 && threadIdx.x == 0) atomicAdd(sched + SCHED_TICKET, REDO_MARK);
+  if (p.force_redo && p.segment == 0 && threadIdx.x == 0) {
+    atomicMax(sched + SCHED_POISON, p.seq);
+    atomicAdd(sched + SCHED_TICKET, REDO_MARK);
+  }
 
   if (failed) {
     if (lane == 0) atomicExch(p.err_flag, 1);
@@ -838,7 +859,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     }
   }
   if ((lane & 3) == 0) { mine[8 * D + qrow] = m_row; mine[8 * D + 8 + qrow] = l_row; mine[8 * D + 16 + qrow] = ld_row; }
+  if (sc_write) fence_async_global();    // the stored logits are read through the async proxy
   __syncthreads();
+  // all warps of the CTA have finished streaming: its share of the head's logits is stored (see scores_complete)
+  if (sc_write && threadIdx.x == 0)
+    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(sched + SCHED_DONE) : "memory");
 
   for (int idx = threadIdx.x; idx < r * D; idx += NW * 32) {
     const int h = idx / D, c = idx % D;

@@ -140,8 +140,8 @@ extern "C" int pod_dense_decode_attn_static(const void* kv_device, int capacity,
   p.early_ok = 0; p.optimistic = 0; p.closer = 0; p.seq = 0; p.force_redo = 0;
   p.segment = 0; p.gate_tau = 2.f; p.dlse = nullptr; p.state_acc = nullptr; p.state_ml = nullptr;
   p.by_value = 1;
-  p.v_len[0] = n_tokens; p.v_cap_d[0] = 0; p.v_row_base[0] = 0; p.v_ring_slot[0] = (n_tokens - 1) % capacity;
-  p.heads_by_value = 0;
+  p.v_len[0] = n_tokens; p.v_cap_d[0] = 0; p.v_row_base[0] = 0;
+  p.heads_by_value = 0; p.plans_by_value = 0;
 
   // The array keeps whatever the previous call left: the chunk counters and the tickets must start at
   // zero.  The error word is left alone: only pod_dense_decode_attn_static_status reads and clears it.
