@@ -2,6 +2,9 @@
 and compute oracle outputs for selected (sequence, layer, head) triples on the host."""
 from __future__ import annotations
 
+import concurrent.futures as cf
+import os
+
 import numpy as np
 import torch
 
@@ -87,3 +90,89 @@ def assert_close(got_bf16, ref_f64, what=""):
     rel = np.linalg.norm(got - ref) / denom if denom > 0 else np.linalg.norm(got - ref)
     assert max_abs <= MAX_ABS and rel <= REL_L2, f"{what}: max_abs={max_abs:.3e} rel_l2={rel:.3e}"
     return max_abs, rel
+
+
+class KVHeadChecker:
+    """Oracle comparison of whole KV-head groups at sizes where every (sequence, layer, head) is checked.
+
+    The r query heads of a KV head share K_l, K_a and V_l, so these are regenerated once per group (on the
+    GPU, by the seeded generator, and copied to the host as fp32, which holds bf16 exactly); the oracle
+    function itself runs unchanged, once per query head, in fp64 on the host.  Groups are computed by a
+    pool of host threads (numpy releases the interpreter lock) while the main thread regenerates inputs.
+    """
+
+    def __init__(self, case, workers=None, max_pending=24):
+        self.case = case
+        self.pool = cf.ThreadPoolExecutor(max_workers=workers or max(2, min(16, (os.cpu_count() or 4))))
+        try:                                   # one BLAS thread per pool thread instead of a pool of pools
+            from threadpoolctl import threadpool_limits
+            self._blas = threadpool_limits(limits=1)
+        except Exception:
+            self._blas = None
+        self.pending, self.max_pending = [], max_pending
+        self.worst = [0.0, 0.0]
+        self.checked = 0
+
+    def _inputs(self, layer, b, kvh, n, step):
+        c = self.case
+        r = c.Hq // c.Hkv
+        low = c.lowest[layer][kvh]
+        f = lambda tag, l: c.kv(tag, l, b, 0, n, "cuda", heads=[kvh])[:, 0].float().cpu().numpy()
+        K_l, V_l = f(synth.TAG_K, layer), f(synth.TAG_V, layer)
+        K_a = K_l if low == layer else f(synth.TAG_K, low)
+        q_l = c.q(layer, step, "cpu")[b, kvh * r:(kvh + 1) * r].double().numpy()
+        q_a = c.q(low, step, "cpu")[b, kvh * r:(kvh + 1) * r].double().numpy()
+        return K_l, K_a, V_l, q_l, q_a, low != layer
+
+    def _work(self, inp, got, what, tau):
+        K_l, K_a, V_l, q_l, q_a, shares = inp
+        c = self.case
+        K_l64, V_l64 = K_l.astype(np.float64), V_l.astype(np.float64)
+        K_a64 = K_l64 if K_a is K_l else K_a.astype(np.float64)
+        scale = c.scale if c.scale > 0 else None
+        res = []
+        for i in range(q_l.shape[0]):
+            ref, _ = O.pod_attention_joint(q_l[i], q_a[i], K_l64, K_a64, V_l64, c.S, c.W, scale=scale)
+            ok = _close(got[i], ref)
+            if tau is not None and shares:
+                # a head of a sharing layer under a gate threshold: the oracle's decision decides, except within
+                # 0.01 of the threshold (the device takes it in fp32), where either candidate is a valid result
+                alt, g, skipped = O.pod_attention_gate_skip(q_l[i], q_a[i], K_l64, K_a64, V_l64, c.S, c.W, tau, scale=scale)
+                ok_alt = _close(got[i], alt)
+                if abs(g - tau) >= 0.01:
+                    ok = ok_alt
+                elif ok_alt[0]:
+                    ok = ok_alt
+            res.append((ok, f"{what} head {i}"))
+        return res
+
+    def submit(self, outs, layer, b, kvh, n, step=0, tau=None):
+        """outs: bf16 device tensor [L][B][Hq][d] (or the same on the host)."""
+        r = self.case.Hq // self.case.Hkv
+        got = outs[layer, b, kvh * r:(kvh + 1) * r].double().cpu().numpy()
+        inp = self._inputs(layer, b, kvh, n, step)
+        self.pending.append(self.pool.submit(self._work, inp, got, f"seq {b} layer {layer} kv head {kvh} step {step}", tau))
+        if len(self.pending) >= self.max_pending:
+            self._drain(self.max_pending // 2)
+
+    def _drain(self, keep):
+        while len(self.pending) > keep:
+            for (ok, max_abs, rel), what in self.pending.pop(0).result():
+                assert ok, f"{what}: max_abs={max_abs:.3e} rel_l2={rel:.3e}"
+                self.worst = [max(self.worst[0], max_abs), max(self.worst[1], rel)]
+                self.checked += 1
+
+    def finish(self):
+        self._drain(0)
+        self.pool.shutdown()
+        if self._blas is not None:
+            self._blas.restore_original_limits()
+        return self.worst
+
+
+def _close(got, ref):
+    g, r = np.asarray(got).reshape(-1), np.asarray(ref).reshape(-1)
+    max_abs = float(np.abs(g - r).max())
+    denom = np.linalg.norm(r)
+    rel = float(np.linalg.norm(g - r) / denom) if denom > 0 else float(np.linalg.norm(g - r))
+    return (max_abs <= MAX_ABS and rel <= REL_L2), max_abs, rel

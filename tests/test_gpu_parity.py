@@ -389,7 +389,9 @@ def test_custom_scale():
 @pytest.mark.parametrize("layer", [0, 1])
 def test_planted_key_at_every_boundary(layer):
     """A key aligned with the query that scores it dominates the softmax: the output must be
-    that token's value row of the decoded layer.  Planted at region and split boundaries."""
+    that token's value row of the decoded layer.  Planted at the region boundaries and at the edges of the
+    kernel's tiles (16 rows; 32 distant rows for a layer that reads stored logits) and chunks (runs of a few
+    tiles) in the order the kernel walks a head: sink rows, ring slots, then distant rows."""
     L, G, Hq, Hkv, d, S, W, n = 2, 2, 4, 1, 128, 16, 64, 3000
     seed = 9
     cfg = B.make_config(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, group_size=G, n_sink=S,
@@ -400,17 +402,19 @@ def test_planted_key_at_every_boundary(layer):
     # make all four query heads of the group identical so one planted key serves them all
     for l in range(L):
         q[l][:, :] = q[l][:, :1]
-    ring_slot0 = next(p for p in range(n - W, n) if (p - S) % W == 0)
-    positions = [0, S - 1, S, S + 1, n - W - 1, n - W, n - 1, ring_slot0, ring_slot0 - 1,
-                 S + W - 1, S + W, 1500, 1501]
+    in_slot = lambda slot: next(p for p in range(n - W, n) if (p - S) % W == slot)
+    positions = [0, S - 1, S, S + 1, n - W - 1, n - W, n - 1, S + W - 1, S + W]
+    positions += [in_slot(x) for x in (0, 15, 16, 31, 32, 47, 48, 63)]     # tile edges among the ring slots
+    n_d = n - S - W
+    last16, last32 = (n_d - 1) // 16 * 16, (n_d - 1) // 32 * 32
+    dist_edges = [0, 15, 16, 31, 32, 33, 47, 48, 63, 64, 95, 96, 511, 512, 527, 528, 1023, 1024, 1471, 1472, 1500,
+                  last16 - 1, last16, last32 - 1, last32, n_d - 1]
+    positions += [S + t for t in dist_edges]                                 # tile and chunk edges among the distant rows
     cache = B.PodCache(cfg, [n])
     for l in range(L):
         cache.write(l, 0, K[l], V[l], n)
     out = torch.empty(1, Hq, d, dtype=torch.bfloat16, device="cuda")
     tmp = torch.empty(1, Hq, d, dtype=torch.bfloat16, device="cuda")
-    cache.decode_attn(0, q[0], tmp)
-    st = cache.last_launch()["split_tokens"]
-    positions += [st - 1, st, 2 * st - 1, 2 * st]           # virtual split boundaries (approximate)
     for pos in sorted(set(p for p in positions if 0 <= p < n)):
         distant = S <= pos < n - W
         src = 0 if (distant and layer == 1) else layer
@@ -542,3 +546,42 @@ def test_stale_query_path_recomputes_heads_exactly(d, G, Hq, Hkv):
         if step in (1, 2, 13, 14, 23):
             _compare_layout(case, cache, ocs)
     assert cache.device_status() == B.POD_OK
+
+
+def test_kv_head_shards_reproduce_the_unsplit_attention():
+    """The KV-head split for several GPUs, run here on one: the cache of each "rank" is built from
+    pod_shard_config / pod_shard_block_map with the rank's slices of k, v and q (contiguous, as column-parallel
+    projections produce them); the ranks' outputs, put side by side at their first query head, are the
+    unsplit attention -- checked head by head against the oracle -- and the ranks' bytes add up."""
+    lens0 = [300, 77]
+    case = Case(seed=29, L=6, G=2, Hq=16, Hkv=4, d=64, S=4, W=16, lens=lens0, caps=[n + 4 for n in lens0], lowest=HEAD_WISE)
+    world, r = 2, 4
+    stream = torch.cuda.current_stream().cuda_stream
+    outs = torch.zeros(case.L, case.B, case.Hq, case.d, dtype=torch.bfloat16, device="cuda")
+    live = 0
+    for rank in range(world):
+        local, kv0, q0 = B.pod_shard_config(case.cfg, rank, world)
+        heads = list(range(kv0, kv0 + local.n_kv_heads))
+        cache = B.PodCache(local, case.caps, lowest_layer=B.pod_shard_block_map(case.cfg, case.lowest, rank, world))
+        for l in range(case.L):
+            for b in range(case.B):
+                k = case.kv(synth.TAG_K, l, b, 0, lens0[b], "cuda", heads=heads)
+                v = case.kv(synth.TAG_V, l, b, 0, lens0[b], "cuda", heads=heads)
+                cache.write(l, b, k, v, lens0[b], stream)
+        for step in (1, 2):                                   # the one-launch form, two steps
+            lens = [n + step for n in lens0]
+            for l in range(case.L):
+                k = torch.stack([case.kv(synth.TAG_K, l, b, lens[b] - 1, lens[b], "cuda", heads=heads)[0] for b in range(case.B)])
+                v = torch.stack([case.kv(synth.TAG_V, l, b, lens[b] - 1, lens[b], "cuda", heads=heads)[0] for b in range(case.B)])
+                q = case.q(l, step, "cuda")[:, q0:q0 + local.n_q_heads].contiguous()
+                o = torch.empty_like(q)
+                cache.append_decode_attn(l, k, v, q, o, stream)
+                outs[l, :, q0:q0 + local.n_q_heads] = o
+        torch.cuda.synchronize()
+        assert cache.device_status() == B.POD_OK
+        live += cache.bytes(B.POD_BYTES_LIVE)
+        cache.destroy()
+    _check_all_heads(case, outs, step=2, lens=[n + 2 for n in lens0])
+    whole, _ = O.pod_cache_bytes([n + 2 for n in lens0], n_layers=case.L, n_kv_heads=case.Hkv, head_dim=case.d,
+                                 group_size=case.G, n_s=case.S, n_r=case.W, lowest=case.lowest)
+    assert live == whole
