@@ -511,6 +511,20 @@ def run_ours(args):
         if rank == 0:
             print(json.dumps({"prefill_attn": time_prefill_attn(B, synth, w, seed, dev, stream, args)}), flush=True)
         return
+    if args.only == "decode-steps":
+        # warm-up and one region of the headline steps, nothing else: the command profilers are pointed at
+        run = Runner(args.workload, w, B=B, synth=synth, dev=dev, local=local, seed=seed, dist=dist, heads=heads,
+                     reserve_steps=args.warmup + args.steps + 8)
+        run.build()
+        for _ in range(args.warmup):
+            run.step()
+        ms = run.region(args.steps)
+        assert run.cache.device_status() == B.POD_OK
+        if rank == 0:
+            print(json.dumps({"decode_steps": {"us_per_layer_step": round(ms * 1e3 / (args.steps * L), 3), "steps": args.steps,
+                                               "launches": run.launches}}), flush=True)
+        run.destroy()
+        return
 
     steps = w.get("steps", args.steps)
     regions = max(1, args.regions)
@@ -813,7 +827,7 @@ def main():
     ap.add_argument("--gate-tau", type=float, default=None, help=argparse.SUPPRESS)
     ap.add_argument("--prefill-tokens", type=int, default=32768,
                     help="positions of the prefill-attention leg (capped at the workload's context)")
-    ap.add_argument("--only", default=None, choices=["prefill-attn"],
+    ap.add_argument("--only", default=None, choices=["prefill-attn", "decode-steps"],
                     help="run one side leg alone and print its object (for profiling)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":

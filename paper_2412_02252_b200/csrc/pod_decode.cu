@@ -206,6 +206,50 @@ struct Cfg {
   static_assert(WARP_B >= (8 * D + 24) * 4, "merge scratch must fit the warp's ring");
 };
 
+// Everything a warp needs to request a tile; filled once per warp.
+struct TileSource {
+  const CUtensorMap* tmap;
+  uint64_t policy;
+  unsigned char* sc_base;           // the head's stored logits
+  uint32_t bar0, ring, sc0;         // shared-memory addresses: first stage barrier, first stage, first logit slot
+  int32_t ntp, rowKp, rowVp, rowKd, rowVd, sc_group_b;
+  int32_t dt_shift;                 // log2 of the tokens of a distant tile
+  int32_t from_scores;              // the head reads stored logits instead of distant keys
+};
+// Requests virtual tile vt into a stage (lane 0 only).  Rows past the segment are other (finite) cache rows,
+// or zero fill past the arena; their logits are masked.  `dep` is zero; it carries a register dependency.
+// part 0: the whole tile; 1: all but the stored logits (before the head's logits are known to be complete);
+// 2: the logits alone.  Not inlined: it is called from a dozen places, none of them hot.
+template <int D>
+__device__ __noinline__ void issue_tile(const TileSource t, int vt, int stage, int dep, int part) {
+  using C = Cfg<D>;
+  const bool dist = vt >= t.ntp;
+  const uint32_t bar = t.bar0 + stage * 8;
+  const uint32_t dst = t.ring + stage * C::STAGE_B;
+  if (dist && t.from_scores) {        // 32 value rows + their logits; no key rows
+    const int yv0 = t.rowVd + ((vt - t.ntp) << t.dt_shift) + dep;
+    if (part != 2) mbar_expect_tx(bar, C::STAGE_B + 2 * t.sc_group_b);
+    if (part != 1)
+      bulk_load(t.sc0 + stage * C::SC_SLOT_B, t.sc_base + (int64_t)(vt - t.ntp) * 2 * t.sc_group_b, 2 * t.sc_group_b, bar);
+    if (part == 2) return;
+#pragma unroll
+    for (int s = 0; s < C::NSUB; ++s) {
+      tma_load_2d(dst + s * C::SUB_B, t.tmap, s * 64, yv0, bar, t.policy);
+      tma_load_2d(dst + C::TILE_B + s * C::SUB_B, t.tmap, s * 64, yv0 + TOK, bar, t.policy);
+    }
+    return;
+  }
+  if (part == 2) return;
+  const int yk = (dist ? t.rowKd + (vt - t.ntp) * TOK : t.rowKp + vt * TOK) + dep;
+  const int yv = dist ? t.rowVd + (vt - t.ntp) * TOK : t.rowVp + vt * TOK;
+  mbar_expect_tx(bar, C::STAGE_B);
+#pragma unroll
+  for (int s = 0; s < C::NSUB; ++s) {
+    tma_load_2d(dst + s * C::SUB_B, t.tmap, s * 64, yk, bar, t.policy);
+    tma_load_2d(dst + C::TILE_B + s * C::SUB_B, t.tmap, s * 64, yv, bar, t.policy);
+  }
+}
+
 // Recomputation of one (sequence, KV head) by a single CTA with a plain loop over its tokens: the way out
 // for a head in which some warp streamed with a copy of q that the previous kernel of the stream had not
 // finished writing (optimistic start).  Exact and slow (a warp per query head, a token per trip); it reads
@@ -433,36 +477,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     if (vt >= ntiles) { walk_done = true; return -1; }
     return (int)vt;
   };
-  // lane 0 only.  Rows past the segment are other (finite) cache rows, or zero fill past the
-  // arena; their logits are masked.  `dep` is zero; it carries a register dependency.
-  // part 0: the whole tile; 1: all but the stored logits (before the wait); 2: the logits alone
-  auto issue = [&](int vt, int stage, int dep, int part) {
-    const bool dist = vt >= ntp;
-    const uint32_t bar = bar0 + stage * 8;
-    const uint32_t dst = wbuf_s + stage * C::STAGE_B;
-    if (dist && sc_read) {            // 32 value rows + their logits; no key rows
-      const int yv0 = rowVd + (vt - ntp) * DT + dep;
-      if (part != 2) mbar_expect_tx(bar, C::STAGE_B + 2 * sc_group_b);
-      if (part != 1)
-        bulk_load(sc0 + stage * C::SC_SLOT_B, sc_base + (int64_t)(vt - ntp) * 2 * sc_group_b, 2 * sc_group_b, bar);
-      if (part == 2) return;
-#pragma unroll
-      for (int s = 0; s < C::NSUB; ++s) {
-        tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yv0, bar, pol_stream);
-        tma_load_2d(dst + C::TILE_B + s * C::SUB_B, &tmap, s * 64, yv0 + TOK, bar, pol_stream);
-      }
-      return;
-    }
-    if (part == 2) return;
-    const int yk = (dist ? rowKd + (vt - ntp) * TOK : rowKp + vt * TOK) + dep;
-    const int yv = dist ? rowVd + (vt - ntp) * TOK : rowVp + vt * TOK;
-    mbar_expect_tx(bar, C::STAGE_B);
-#pragma unroll
-    for (int s = 0; s < C::NSUB; ++s) {
-      tma_load_2d(dst + s * C::SUB_B, &tmap, s * 64, yk, bar, pol_stream);
-      tma_load_2d(dst + C::TILE_B + s * C::SUB_B, &tmap, s * 64, yv, bar, pol_stream);
-    }
-  };
+  TileSource src;
+  src.tmap = &tmap; src.policy = pol_stream; src.sc_base = sc_base; src.bar0 = bar0; src.ring = wbuf_s; src.sc0 = sc0;
+  src.ntp = ntp; src.rowKp = rowKp; src.rowVp = rowVp; src.rowKd = rowKd; src.rowVd = rowVd; src.sc_group_b = sc_group_b;
+  src.dt_shift = DT_SH; src.from_scores = sc_read ? 1 : 0;
+  auto issue = [&](int vt, int stage, int dep, int part) { issue_tile<D>(src, vt, stage, dep, part); };
 
   // Rows that change in a fused launch are masked in the streamed tiles and added by one warp
   // from registers: the new token's proximal row, and the distant row of the token it pushes
@@ -668,15 +687,12 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // The second reading of q (and of the new k, v rows) goes into a stage the warp no longer needs as an
   // asynchronous copy (L2 to shared memory), so that nobody waits for it; it is compared after the loop.
   int check_stage = -1;
-  auto late_wait = [&]() {
+  auto late_wait = [&](int free_stage) {   // free_stage: a stage of this warp that no tile will use any more
     pdl_wait();
     pdl_launch_dependents();
     late_pending = false;
     if (warp != 0) return;                 // the CTA's copies were made, and are checked, by warp 0
-#pragma unroll
-    for (int s = 0; s < NSTAGE; ++s)
-      if (check_stage < 0 && vt_q[s] < 0) check_stage = s;
-    if (check_stage < 0) return;           // (not reached: the walk is over, so some stage is free)
+    check_stage = free_stage;
     const uint32_t dst = wbuf_s + check_stage * C::STAGE_B;
     for (int i = lane; i < r * (D / 8); i += 32) cp_async_16(dst + i * 16, p.q + q_own + (int64_t)i * 8);
     if (fused && split == 0 && lane < D / 4)
@@ -704,13 +720,16 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     stash_q();
   };
 
-  for (bool more = true; more && !failed; ++round) {
-#pragma unroll
-    for (int s = 0; s < NSTAGE; ++s) {
-      if (!more || failed) continue;
-      const int vt = vt_q[s];
-      if (vt < 0) { more = false; continue; }
-      if (!__all_sync(0xffffffffu, mbar_wait(bar0 + s * 8, round & 1))) { failed = true; fail_stage = s; continue; }
+  // One tile per trip, the stages in turn (the loop is not unrolled over the stages: the code of a trip is
+  // large, and three copies of it did not fit the instruction cache with the rest of the kernel).  v0 is the
+  // tile in stage s, v1 and v2 the tiles in the two stages after it.
+  int v0 = vt_q[0], v1 = NSTAGE > 1 ? vt_q[1] : -1, v2 = NSTAGE > 2 ? vt_q[2] : -1;
+  static_assert(NSTAGE <= 3, "the tile rotation below holds three stages");
+  int s = 0;
+  while (v0 >= 0) {
+    {
+      const int vt = v0;
+      if (!__all_sync(0xffffffffu, mbar_wait(bar0 + s * 8, round & 1))) { failed = true; fail_stage = s; break; }
       const bool dist = vt >= ntp;
       const bool from_scores = dist && sc_read;
       const int rem = dist ? n_d - (vt - ntp) * DT : n_p - vt * TOK;      // valid rows from the tile's start
@@ -750,8 +769,8 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       int dep;
       asm volatile("and.b32 %0, %1, 0;" : "=r"(dep) : "r"(fb[D / 16 - 1][3]));
       __syncwarp();
-      vt_q[s] = next_tile();
-      if (lane == 0 && vt_q[s] >= 0) issue(vt_q[s], s, dep, 0);
+      const int v_new = next_tile();
+      if (lane == 0 && v_new >= 0) issue(v_new, s, dep, 0);
 
       // one online-softmax step (base 2) over 16 tokens: logits l (log2 units; tokens qcol, +1,
       // +8, +9 of head qrow), `cnt` valid tokens, token `mcol` left out, value fragments vf
@@ -819,10 +838,13 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
         softmax_pv((s0[0] + t0[0]) * p.scale_log2, (s0[1] + t0[1]) * p.scale_log2, (s1[0] + t1[0]) * p.scale_log2,
                    (s1[1] + t1[1]) * p.scale_log2, min(TOK, rem), mtile, fb, store, dist);
       }
+      // the stage just used holds the new tile, or is free from now on
+      if (NSTAGE == 3) { v0 = v1; v1 = v2; v2 = v_new; } else if (NSTAGE == 2) { v0 = v1; v1 = v_new; } else { v0 = v_new; }
+      if (late_pending && walk_done) late_wait(s);
+      if (++s == NSTAGE) { s = 0; ++round; }
     }
-    if (late_pending && walk_done) late_wait();
   }
-  if (late_pending) late_wait();
+  if (late_pending) late_wait(0);
   late_check();
   if (p.force_redo && p.segment == 0 && threadIdx.x == 0) {
     atomicMax(sched + SCHED_POISON, p.seq);
@@ -831,13 +853,14 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
 
   if (failed) {
     if (lane == 0) atomicExch(p.err_flag, 1);
-    // `round` was advanced once after the failing pass.  Drain the copies this warp still has in
-    // flight before its shared memory is reused: stages before the failing one were refilled in
-    // that pass, the others still hold that pass's tile.
-    const uint32_t fr = round - 1;
-#pragma unroll
-    for (int s = 0; s < NSTAGE; ++s)
-      if (vt_q[s] >= 0) mbar_wait(bar0 + s * 8, (s < fail_stage ? fr + 1 : fr) & 1);
+    // Drain the copies this warp still has in flight before its shared memory is reused: v0, v1, v2 sit in
+    // the failing stage and the ones after it; stages before the failing one were refilled in this round
+    // (next parity), the others still hold this round's tile.
+    const int vq[3] = {v0, v1, v2};
+    for (int i = 0; i < NSTAGE; ++i) {
+      const int st = (fail_stage + i) % NSTAGE;
+      if (vq[i] >= 0) mbar_wait(bar0 + st * 8, (st < fail_stage ? round + 1 : round) & 1);
+    }
   }
 
   // ---- merge the warps of the CTA -------------------------------------------------------------
