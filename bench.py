@@ -506,6 +506,13 @@ def run_ours(args):
         heads = list(range(kv0, kv0 + local_cfg.n_kv_heads))
     elif world > 1:
         seed = rank_seed(seed, rank)
+    elif args.one_shard_of > 1:
+        # one GPU doing the work of one rank of a KV-head split (rank 0 of --one-shard-of ranks): what a rank's
+        # launches cost, without the other ranks -- not a multi-GPU measurement
+        cfg_full = B.make_config(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, group_size=w["G"], n_sink=S,
+                                 n_recent=W, batch=w["B"], device=local)
+        local_cfg, kv0, _ = B.pod_shard_config(cfg_full, 0, args.one_shard_of)
+        heads = list(range(kv0, kv0 + local_cfg.n_kv_heads))
 
     if args.only == "prefill-attn":
         if rank == 0:
@@ -579,7 +586,7 @@ def run_ours(args):
 
     # ---- the other configurations of the scope table, one after the other (each frees its cache) ----
     others = {}
-    if world == 1 and not args.no_extra and args.workload == "llama3-8b-32k":
+    if world == 1 and not args.no_extra and args.workload == "llama3-8b-32k" and args.one_shard_of <= 1:
         for name in EXTRA_WORKLOADS:
             free_gib = torch.cuda.mem_get_info()[0] / 2 ** 30
             wx = dict(WORKLOADS[name])
@@ -649,7 +656,10 @@ def run_ours(args):
         "two_call_us_per_layer_step": res.get("two_call_us_per_layer_step"),
         "dense_kv_baseline_us_per_layer_step": dense_us,
     }
-    if not args.no_cpu and world == 1 and "head_wise_new_block_p" not in w and not w.get("ragged"):
+    if args.one_shard_of > 1:
+        line["config"]["shard"] = "rank 0 of a %d-way KV-head split, alone on one GPU (%d of %d KV heads)" % (
+            args.one_shard_of, len(heads), Hkv)
+    if not args.no_cpu and world == 1 and "head_wise_new_block_p" not in w and not w.get("ragged") and args.one_shard_of <= 1:
         line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_budget)
     print(json.dumps(line))
     if dist is not None:
@@ -820,6 +830,8 @@ def main():
     ap.add_argument("--workload", default="llama3-8b-32k", choices=sorted(WORKLOADS))
     ap.add_argument("--shard", default="sequence", choices=["sequence", "kv-head"],
                     help="with several GPUs: independent sequences per rank, or H_kv / N KV heads of the same sequences per rank")
+    ap.add_argument("--one-shard-of", type=int, default=1,
+                    help="on one GPU: run rank 0's share of a KV-head split over this many ranks (what one rank's launches cost)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-KV baseline legs")
     ap.add_argument("--no-extra", action="store_true", help="skip the 128K, batch-16 and ragged workloads")
