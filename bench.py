@@ -694,6 +694,21 @@ def time_prefill_write(B, synth, w, seed, dev, local, stream, reps=6):
         # and the W rows per head and kind that leave the ring; written: the same rows at their new places
         rows = T_ * Hkv + T_ * keeps + W * (Hkv - keeps) + W * (Hkv + keeps)
         out[name] = {"us": round(us, 2), "gbs": round(2 * rows * row / (us * 1e-6) / 1e9, 1)}
+        # yardstick: a plain device-to-device copy of as many bytes, issued the same way (the copy rate the
+        # roofline uses is that of much larger buffers; at this size a launch's ramp and tail weigh more)
+        nb = rows * row
+        srcs = [torch.empty(nb, dtype=torch.uint8, device=dev).fill_(i) for i in range(2)]
+        dsts = [torch.empty(nb, dtype=torch.uint8, device=dev) for _ in range(reps)]
+        dsts[0].copy_(srcs[0])
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(reps):
+            dsts[i].copy_(srcs[i % 2])
+        e1.record()
+        torch.cuda.synchronize()
+        cus = e0.elapsed_time(e1) * 1e3 / reps
+        out[name]["device_copy_same_bytes"] = {"us": round(cus, 2), "gbs": round(2 * nb / (cus * 1e-6) / 1e9, 1)}
+        del srcs, dsts
     pc.destroy()
     out["tokens_per_call"] = T_
     out["note"] = "bytes read + written per call over the mean of back-to-back calls"

@@ -142,7 +142,6 @@ struct pod_cache {
   int last_decode_layer = -1;          // layer of the previous launch on this cache if it was a decode launch, else -1
   std::vector<int32_t> score_low;      // [H_kv] lowest layer whose distant logits the head's score store holds, -1 = none
   std::vector<int32_t> score_len;      // [H_kv][B] lengths at which they were stored
-  std::vector<int32_t> score_seq;      // [H_kv] sequence number of the launch that stored them
   std::vector<uint32_t> done_total;    // [B][H_kv] what the head's DONE word reads when all launches so far are through with it
   std::vector<uint32_t> score_done;    // [B][H_kv] done_total right after the launch that stored the head's logits
   int32_t launch_seq = 0;              // decode kernels launched on this cache so far
@@ -310,7 +309,6 @@ static int create_impl(const pod_config* cfg, const int32_t* seq_capacity, const
   c->len_cur.assign((size_t)cfg->n_layers, 0);
   c->score_low.assign((size_t)cfg->n_kv_heads, -1);
   c->score_len.assign((size_t)cfg->n_kv_heads * cfg->batch, -1);
-  c->score_seq.assign((size_t)cfg->n_kv_heads, 0);
   c->done_total.assign((size_t)cfg->n_kv_heads * cfg->batch, 0u);
   c->score_done.assign((size_t)cfg->n_kv_heads * cfg->batch, 0u);
   c->stash_len.assign((size_t)c->bm.n_slots * cfg->batch, -1);
@@ -596,7 +594,6 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
           hp = make_head_plan(p.y, in, h, c->h_len(layer, b), c->cv.seq_cap_d[b], c->cv.seq_row_base[b], low,
                               c->slot_of(layer, h), store, read);
           hp.wait_done = (int32_t)c->score_done[(size_t)b * H + h];
-          hp.wait_seq = c->score_seq[h];
         }
     }
     // A launch that appends and attends streams only rows written before this step (the new token's
@@ -642,7 +639,6 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
   for (int h = 0; h < H; ++h) {          // heads whose block starts here and goes on: their logits are stored now
     if (c->low_of(layer, h) != layer || layer + 1 >= g.n_layers || c->low_of(layer + 1, h) != layer) continue;
     c->score_low[h] = layer;
-    c->score_seq[h] = c->launch_seq;
     for (int b = 0; b < g.batch; ++b) c->score_done[(size_t)b * H + h] = c->done_total[(size_t)b * H + h];
     for (int b = 0; b < g.batch; ++b) c->score_len[(size_t)h * g.batch + b] = c->h_len(layer, b);
   }

@@ -32,10 +32,8 @@ constexpr int SCHED_TICKET = 16;      // [0] = chunk counter, [SCHED_TICKET] = f
 constexpr int SCHED_NEED = 2;         // [SCHED_NEED] = query heads of this KV head that still need their distant tokens (gate)
 constexpr int SCHED_CTR1 = 4;         // [(seq & 1) * SCHED_CTR1] = chunk counter: launches alternate between two, because a launch
                                       //   may draw chunks while the previous launch of the cache is still finishing
-constexpr int SCHED_DONE = 28;        // CTAs of this head, over all launches that store logits, whose warps have finished streaming
-constexpr int SCHED_POISON = 29;      // highest sequence number of a launch in which a CTA of this head found its copy of q stale
-constexpr int SCHED_EPOCH = 24;       // sequence number of the last launch whose CTAs of this head have all finished streaming
-                                      //   (its stored logits and stashed queries are complete); own 32-byte sector
+constexpr int SCHED_DONE = 24;        // CTAs of this head, over all launches that store logits, whose warps have finished streaming
+                                      //   with valid inputs (a head that had to be recomputed counts them afterwards); own 32-byte sector
 
 // Physical layout of the arena.  All offsets are in rows; one row is one head's d bf16
 // values (128 B at d = 64, 256 B at d = 128), so every region base is 128-byte aligned.
@@ -118,8 +116,8 @@ struct HeadPlan {
   int32_t flags;                           // HP_*
   int32_t rA, rB;                          // a launch that appends: proximal row of the new token, distant row of the
                                            // token it pushes out of the window (-1 = none)
-  int32_t wait_done, wait_seq;             // a head that reads stored logits: what its DONE word reads once the launch
-                                           // that stored them is through with the head, and that launch's sequence number
+  int32_t wait_done;                       // a head that reads stored logits: what its DONE word reads once the launch
+                                           // that stored them is through with the head
 };
 constexpr int HP_LOW = 1;                  // this layer is the lowest of the head's block
 constexpr int HP_STORE = 2;                // ... and the block goes on: the head stores its distant logits
@@ -159,7 +157,7 @@ __host__ __device__ inline HeadPlan make_head_plan(const Layout& y, const PlanIn
   hp.rowKd = (int32_t)(seq_row + distk_row(y, kslot, cap_d));
   hp.rowVd = (int32_t)(seq_row + distv_row(y, in.layer, kvh, cap_d));
   hp.score_row = (int32_t)(seq_row + score_row(y, kvh, cap_d));
-  hp.wait_done = 0; hp.wait_seq = 0;
+  hp.wait_done = 0;
   hp.rA = -1; hp.rB = -1;
   if (in.fused) {
     const int pos = n - 1;
@@ -235,10 +233,10 @@ struct DecodeParams {
   // the stream may still be writing (a projection of the caller's); a warp whose early copy turns out
   // stale marks its head, and the head's last CTA recomputes it with a plain loop (slow, exact, in
   // practice never taken).  What this launch needs from an earlier launch of the cache -- the block's
-  // stored logits and stashed queries -- is awaited per head through the head's epoch word instead.
+  // stored logits and stashed queries -- is awaited per head through the head's DONE word instead.
   int32_t optimistic;
   int32_t closer;          // 1: every CTA of the grid is resident at once; a head's first CTA combines and waits for the others
-  int32_t seq;             // sequence number of this launch on its cache (chunk-counter parity, epoch)
+  int32_t seq;             // sequence number of this launch on its cache (chunk-counter parity)
   int32_t force_redo;      // test hook set from the host: every warp behaves as if its early copy of q were stale
   int32_t early_ok;        // 1: no unfinished launch writes cache rows this launch streams (the two rows a
                            //    fused launch changes itself aside): tiles may be requested before the

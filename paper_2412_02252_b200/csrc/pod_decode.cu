@@ -51,8 +51,9 @@ namespace {
 
 constexpr int TOK = 16;          // tokens per tile (one mma k-step of P V)
 constexpr uint32_t WAIT_LIMIT = 1u << 20;
-constexpr int REDO_MARK = 1 << 20;     // added to a head's ticket word by a warp whose early copy of q, k or v was stale
-constexpr int EPOCH_POLLS = 1 << 13;   // polls (about 0.3 us apart) of a head's epoch word before falling back to the grid wait
+constexpr int REDO_SHIFT = 20;
+constexpr int REDO_MARK = 1 << REDO_SHIFT;     // added to a head's ticket word by a warp whose early copy of q, k or v was stale
+constexpr int DONE_POLLS = 1 << 13;   // polls (about 0.3 us apart) of a head's DONE word before falling back to the grid wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -408,18 +409,33 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int64_t q_st = ((int64_t)kslot * y.B + b) * r * D;          // and in the stash of its block
   constexpr int QS = D + 8;                       // row stride in elements: the fragment reads hit 32 banks
   __shared__ __align__(16) uint16_t s_q[8 * QS];
-  auto load_q = [&]() {
+  // Warp 0 brings the CTA's copy of q into shared memory in two steps: the loads go out into registers,
+  // and the stores to shared memory follow where the values are first needed, so that the warp does not sit
+  // out a memory round trip between the two.
+  constexpr int QL = D / 32;                      // 16-byte pieces per lane: up to 8 heads x D / 8 pieces
+  uint4 q_reg[QL];
+  auto request_q = [&]() {
     if (warp == 0) {
-      for (int i = lane; i < r * (D / 8); i += 32) {
-        const int h = i / (D / 8), c8 = i % (D / 8);
-        *reinterpret_cast<uint4*>(&s_q[h * QS + c8 * 8]) = ld_relaxed_u32x4(p.q + q_own + h * D + c8 * 8);
+#pragma unroll
+      for (int k = 0; k < QL; ++k) {
+        const int i = lane + 32 * k;
+        if (i < r * (D / 8)) q_reg[k] = ld_relaxed_u32x4(p.q + q_own + (int64_t)i * 8);
+      }
+    }
+  };
+  auto keep_q = [&]() {
+    if (warp == 0) {
+#pragma unroll
+      for (int k = 0; k < QL; ++k) {
+        const int i = lane + 32 * k;
+        if (i < r * (D / 8)) *reinterpret_cast<uint4*>(&s_q[(i / (D / 8)) * QS + (i % (D / 8)) * 8]) = q_reg[k];
       }
     }
   };
   // q is requested before the tiles when it may be read already (the tile requests of a whole SM would
   // be served first otherwise): the launch has waited, or starts optimistically
   const bool q_loaded = waited || opt;
-  if (q_loaded) load_q();
+  if (q_loaded) request_q();
 
   // arena rows of this (sequence, layer, head): tile coordinates of the tensor map
   const int rowKp = hp.rowKp, rowVp = hp.rowVp, rowKd = hp.rowKd, rowVd = hp.rowVd;
@@ -427,7 +443,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   const int sc_group_b = score_group_bytes(y);
   unsigned char* sc_base = reinterpret_cast<unsigned char*>(const_cast<uint16_t*>(p.arena)) + (int64_t)hp.score_row * (D * 2);
 
-  if (p.segment == 2 && sched[SCHED_NEED] == 0) return;   // every query head of this KV head skipped: no distant work
+  if (p.segment == 2 && sched[SCHED_NEED] == 0) {          // every query head of this KV head skipped: no distant work
+    if (sc_write && threadIdx.x == 0) atomicAdd(sched + SCHED_DONE, 1);   // (the host counts every CTA of a storing head)
+    return;
+  }
 
   // ---- the warp's walk over its chunks (all values uniform across the warp) -----------------
   if (!waited && !opt && k_static * tch < NSTAGE) {   // the first tiles need draws: no early start
@@ -496,15 +515,11 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // The block's logits (and stashed queries) come from an earlier launch of this cache, possibly the one
   // still running.  Every CTA of that launch adds one to the head's DONE word when its warps have finished
   // streaming (all logits of theirs are stored); the host knows what the word reads once the head is
-  // complete.  If a CTA of that launch found its copy of q stale, the logits are rewritten by the head's
-  // recomputation, which the head's epoch word announces: the POISON word says whether to wait for that.
+  // complete.  A CTA that found its copy of q stale does not add its one: the CTA that recomputes the head
+  // adds the missing ones when the logits have been rewritten, so the word is complete only then.
   auto scores_complete = [&]() -> bool {          // lane 0's view, passed to the warp
     int ok = 0;
-    if (lane == 0) {
-      ok = (int)(ld_acquire_gpu(sched + SCHED_DONE) - hp.wait_done) >= 0;
-      if (ok && (int)(ld_acquire_gpu(sched + SCHED_POISON) - hp.wait_seq) >= 0)
-        ok = (int)(ld_acquire_gpu(sched + SCHED_EPOCH) - hp.wait_seq) >= 0;
-    }
+    if (lane == 0) ok = (int)(ld_acquire_gpu(sched + SCHED_DONE) - hp.wait_done) >= 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
   };
   // An optimistic launch that reads stored logits looks before its tile requests go out (behind them an
@@ -530,7 +545,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       // One warp of the CTA polls (the barrier below passes the news on).  Bounded; after the limit the
       // grid wait settles it.
       bool ready = false;
-      for (int it = 0; it < EPOCH_POLLS && !ready; ++it) {
+      for (int it = 0; it < DONE_POLLS && !ready; ++it) {
         ready = scores_complete();
         if (!ready) __nanosleep(128);
       }
@@ -540,7 +555,8 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       }
     }
   }
-  if (!q_loaded) load_q();              // (a launch that had to wait first reads q only now)
+  if (!q_loaded) request_q();           // (a launch that had to wait first reads q only now)
+  keep_q();
   __syncthreads();                      // q in shared memory; the head's logits known to be complete
   if (!waited) {
     if (lane == 0 && !scores_done) {
@@ -700,8 +716,8 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
                   (lane >= D / 8 ? p.new_v : p.new_k) + ((int64_t)b * y.H_kv + kvh) * D + (lane % (D / 8)) * 8);
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  auto late_check = [&]() {                // after the loop: compare, mark the head if a copy was stale
-    if (warp != 0 || check_stage < 0) return;
+  auto late_check = [&]() -> bool {        // after the loop: compare; true (in warp 0) if a copy was stale
+    if (warp != 0 || check_stage < 0) return false;
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncwarp();
     const unsigned char* got = wbuf + check_stage * C::STAGE_B;
@@ -712,12 +728,9 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     }
     if (fused && split == 0 && lane < D / 4)
       stale = stale || differ(nw_early, *reinterpret_cast<const uint4*>(got + 8 * D * 2 + lane * 16));
-    // a mark is a large number added to the head's ticket word: the CTA that draws the last ticket sees it
-    if (__any_sync(0xffffffffu, stale) && lane == 0) {
-      atomicMax(sched + SCHED_POISON, p.seq);
-      atomicAdd(sched + SCHED_TICKET, REDO_MARK);
-    }
+    stale = __any_sync(0xffffffffu, stale);
     stash_q();
+    return stale;
   };
 
   // One tile per trip, the stages in turn (the loop is not unrolled over the stages: the code of a trip is
@@ -845,11 +858,10 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     }
   }
   if (late_pending) late_wait(0);
-  late_check();
-  if (p.force_redo && p.segment == 0 && threadIdx.x == 0) {
-    atomicMax(sched + SCHED_POISON, p.seq);
-    atomicAdd(sched + SCHED_TICKET, REDO_MARK);
-  }
+  // A CTA with a stale copy marks the head: a large number added to the head's ticket word, which the CTA that
+  // draws the last ticket sees (this thread's ticket comes later, to the same word).
+  const bool cta_stale = late_check() || (p.force_redo && p.segment == 0);    // as seen by warp 0
+  if (cta_stale && threadIdx.x == 0) atomicAdd(sched + SCHED_TICKET, REDO_MARK);
 
   if (failed) {
     if (lane == 0) atomicExch(p.err_flag, 1);
@@ -885,7 +897,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   if (sc_write) fence_async_global();    // the stored logits are read through the async proxy
   __syncthreads();
   // all warps of the CTA have finished streaming: its share of the head's logits is stored (see scores_complete)
-  if (sc_write && threadIdx.x == 0)
+  if (sc_write && threadIdx.x == 0 && !cta_stale)
     asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(sched + SCHED_DONE) : "memory");
 
   for (int idx = threadIdx.x; idx < r * D; idx += NW * 32) {
@@ -918,7 +930,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   // their slot on the SM goes to the next kernel a memory round trip earlier -- and the first CTA waits
   // (bounded) until the count is complete.  It cannot wait for a CTA that has no slot yet, because in that
   // mode every CTA of the grid gets one without anyone leaving.
-  __shared__ int s_last;
+  __shared__ int s_last, s_marks;
   fence_async_global();                  // the partials are read back through the async proxy
   __syncthreads();
   if (p.closer && split != 0) {
@@ -950,9 +962,9 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
       // complete, which is what a later launch waits for -- unless a warp found its early copies stale (it added
       // its mark to this word before its CTA took its ticket); then the head is redone first.
       if (got >= REDO_MARK) last = 2;
-      else st_release_gpu(sched + SCHED_EPOCH, p.seq);
     }
     s_last = last;
+    s_marks = got >> REDO_SHIFT;
   }
   __syncthreads();
   if (!s_last) {
@@ -971,7 +983,9 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
                  rowKd, rowVd, sc_base, sc_group_b, is_low, sc_write, q_own, q_st);
     fence_async_global();
     __syncthreads();
-    if (threadIdx.x == 0) st_release_gpu(sched + SCHED_EPOCH, p.seq);
+    // the logits are rewritten: the DONE counts that the marked CTAs held back
+    if (threadIdx.x == 0 && sc_write)
+      asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(sched + SCHED_DONE), "r"(s_marks) : "memory");
     trace_end(p);
     return;
   }
