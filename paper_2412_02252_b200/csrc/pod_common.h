@@ -44,9 +44,12 @@ constexpr int SCHED_DONE = 24;        // CTAs of this head, over all launches th
 //   distK [n_slots][cap_d[b]]                 index p - n_s, key of a block's lowest layer; one slot per
 //                                             (head, block of that head), a head's slots adjacent
 //   guard [32]                                only when layers share: rows that stay zero
-//   score [H_kv][score_rows_per_head]         only when layers share: the distant logits of the block being
+//   score [H_kv][2][score_rows_per_head]      only when layers share: the distant logits of the block being
 //                                             decoded (fp32, log2 units), one group of 16 tokens x r
-//                                             query heads = r * 64 bytes in mma fragment order
+//                                             query heads = r * 64 bytes in mma fragment order; two stores
+//                                             per head, used in turn by the head's consecutive blocks, so
+//                                             that a launch which stores the logits of the next block never
+//                                             writes where the launch before it (possibly still running) reads
 // with cap_d[b] = max(0, capacity[b] - n_s - n_r).  Sink and ring of one (layer, head) are
 // adjacent so that the proximal tokens of a head are one contiguous stream (the softmax does
 // not care about token order, so ring slots are read in slot order).
@@ -96,11 +99,13 @@ __host__ __device__ inline int64_t score_rows_per_head(const Layout& y, int64_t 
 // separates them from the key and value rows before them.
 constexpr int SCORE_GUARD_ROWS = 32;
 __host__ __device__ inline int64_t score_rows_per_seq(const Layout& y, int64_t cap_d) {
-  return !y.shared ? 0 : SCORE_GUARD_ROWS + y.H_kv * score_rows_per_head(y, cap_d);
+  return !y.shared ? 0 : SCORE_GUARD_ROWS + 2 * y.H_kv * score_rows_per_head(y, cap_d);
 }
-__host__ __device__ inline int64_t score_row(const Layout& y, int head, int64_t cap_d) {
+// `kslot` is the key store of the head's block: a head's blocks have consecutive key stores, so its parity
+// alternates from one block of the head to the next.
+__host__ __device__ inline int64_t score_row(const Layout& y, int head, int64_t cap_d, int kslot) {
   return dist_base_row(y) + ((int64_t)y.L * y.H_kv + y.n_slots) * cap_d + SCORE_GUARD_ROWS +
-         head * score_rows_per_head(y, cap_d);
+         (2 * head + (kslot & 1)) * score_rows_per_head(y, cap_d);
 }
 
 // What one (sequence, KV head) of a decode launch needs to know before it can request its first tile.
@@ -156,7 +161,7 @@ __host__ __device__ inline HeadPlan make_head_plan(const Layout& y, const PlanIn
   hp.rowVp = (int32_t)(seq_row + prox_row(y, in.layer, 1, kvh));
   hp.rowKd = (int32_t)(seq_row + distk_row(y, kslot, cap_d));
   hp.rowVd = (int32_t)(seq_row + distv_row(y, in.layer, kvh, cap_d));
-  hp.score_row = (int32_t)(seq_row + score_row(y, kvh, cap_d));
+  hp.score_row = (int32_t)(seq_row + score_row(y, kvh, cap_d, kslot));
   hp.wait_done = 0;
   hp.rA = -1; hp.rB = -1;
   if (in.fused) {

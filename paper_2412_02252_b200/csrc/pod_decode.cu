@@ -123,9 +123,6 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* a) {
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(a) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_release_gpu(int* a, int v) {
-  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(a), "r"(v) : "memory");
-}
 // A load that may race with a store of the previous kernel (the early copies of q, k, v, checked later),
 // or that must see that kernel's stores after the grid wait: served by the L2, never by an L1 line of this
 // SM (which an earlier load of this kernel may have filled with older data).
@@ -896,10 +893,8 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   if ((lane & 3) == 0) { mine[8 * D + qrow] = m_row; mine[8 * D + 8 + qrow] = l_row; mine[8 * D + 16 + qrow] = ld_row; }
   if (sc_write) fence_async_global();    // the stored logits are read through the async proxy
   __syncthreads();
-  // all warps of the CTA have finished streaming: its share of the head's logits is stored (see scores_complete)
-  if (sc_write && threadIdx.x == 0 && !cta_stale)
-    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(sched + SCHED_DONE) : "memory");
-
+  // all warps of the CTA have finished streaming: its share of the head's logits is stored; the head's DONE
+  // count moves below, together with the CTA's ticket (see scores_complete)
   for (int idx = threadIdx.x; idx < r * D; idx += NW * 32) {
     const int h = idx / D, c = idx % D;
     float M = -INFINITY;
@@ -933,9 +928,14 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   __shared__ int s_last, s_marks;
   fence_async_global();                  // the partials are read back through the async proxy
   __syncthreads();
+  // One release for both of the head's counts: this CTA's logits and partials are visible before either moves.
+  if (threadIdx.x == 0) {
+    asm volatile("fence.acq_rel.gpu;" ::: "memory");
+    if (sc_write && !cta_stale) asm volatile("red.relaxed.gpu.global.add.s32 [%0], 1;" ::"l"(sched + SCHED_DONE) : "memory");
+  }
   if (p.closer && split != 0) {
     if (threadIdx.x == 0)
-      asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(sched + SCHED_TICKET) : "memory");
+      asm volatile("red.relaxed.gpu.global.add.s32 [%0], 1;" ::"l"(sched + SCHED_TICKET) : "memory");
     trace_end(p);
     return;
   }

@@ -241,7 +241,9 @@ def test_largest_cache_is_bounded_by_32_bit_row_indices():
     """Tile coordinates are 32-bit row indices: a cache whose regions would hold 2^31 rows or more is
     refused at creation (and sized 0), the largest one below that is accepted on a host-only cache."""
     cfg = _cfg(n_layers=32, n_q_heads=32, n_kv_heads=8, head_dim=128, group_size=2, n_sink=16, n_recent=2048)
-    rows_per_token = 32 * 8 + 16 * 8                     # value rows of every layer + key rows of every block
+    # value rows of every layer + key rows of every block + the stored logits of a distant token
+    # (two stores per KV head, 4 query heads x 4 bytes each: 8 x 2 x 16 B = one 256-byte row)
+    rows_per_token = 32 * 8 + 16 * 8 + 1
     too_many = (2 ** 31) // rows_per_token + 4096
     assert B.pod_cache_required_bytes(cfg, [too_many]) == 0
     with pytest.raises(B.PodError) as e:
