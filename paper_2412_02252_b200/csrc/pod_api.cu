@@ -139,6 +139,7 @@ struct pod_cache {
   bool dry = false;
   int last_cuda = 0;
   int sm_count = 148, resident = 2;
+  bool keep_logits = false;            // the logit stores are a small part of the L2: they are written and read with evict_last
   int last_decode_layer = -1;          // layer of the previous launch on this cache if it was a decode launch, else -1
   std::vector<int32_t> score_low;      // [H_kv] lowest layer whose distant logits the head's score store holds, -1 = none
   std::vector<int32_t> score_len;      // [H_kv][B] lengths at which they were stored
@@ -347,6 +348,8 @@ static int create_impl(const pod_config* cfg, const int32_t* seq_capacity, const
   ok = ok && cudaMemcpy(c->arena + c->cv.off_slot, c->bm.slot.data(), c->bm.slot.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess;
   int sm = 0;
   ok = ok && cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess;
+  int l2_bytes = 0;
+  ok = ok && cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, cfg->device) == cudaSuccess;
   const int res = ok ? decode_resident_ctas_per_sm(cfg->head_dim) : 0;
   ok = ok && res > 0 && cudaDeviceSynchronize() == cudaSuccess;
   if (!ok) {
@@ -356,6 +359,11 @@ static int create_impl(const pod_config* cfg, const int32_t* seq_capacity, const
     return POD_ERR_CUDA;
   }
   c->sm_count = sm; c->resident = res;
+  {                                    // all logit stores of the cache at capacity against the L2
+    int64_t rows = 0;
+    for (int b = 0; b < cfg->batch; ++b) rows += score_rows_per_seq(c->y, c->cv.seq_cap_d[b]);
+    c->keep_logits = rows > 0 && rows * cfg->head_dim * 2 <= (int64_t)l2_bytes / 8;
+  }
   if (const char* ct = getenv("POD_CHUNK_TILES")) c->force_chunk_tiles = atoi(ct);
   if (const char* se = getenv("POD_STATIC_EIGHTHS")) {
     const int v = atoi(se);
@@ -613,6 +621,7 @@ static int decode_impl(pod_cache* c, int layer, const void* k_new, const void* v
     // every CTA gets a slot on some SM without another CTA of the grid leaving first
     p.closer = (c->closer && (int64_t)p.y.H_kv * plan.grid_splits * p.y.B <= (int64_t)c->sm_count * c->resident) ? 1 : 0;
     p.force_redo = (c->inject_stale && !gated) ? 1 : 0;
+    p.keep_logits = c->keep_logits ? 1 : 0;
     c->inject_stale = false;
     p.trace = (c->trace != nullptr && c->trace_n < c->trace_cap) ? c->trace + 2 * (size_t)c->trace_n++ : nullptr;
     const int e = launch_decode(c->tmap, p, plan.grid_splits, s);

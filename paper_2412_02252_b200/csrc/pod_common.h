@@ -243,6 +243,7 @@ struct DecodeParams {
   int32_t closer;          // 1: every CTA of the grid is resident at once; a head's first CTA combines and waits for the others
   int32_t seq;             // sequence number of this launch on its cache (chunk-counter parity)
   int32_t force_redo;      // test hook set from the host: every warp behaves as if its early copy of q were stale
+  int32_t keep_logits;     // 1: the cache's logit stores are a small part of the L2: write and read them with evict_last
   int32_t early_ok;        // 1: no unfinished launch writes cache rows this launch streams (the two rows a
                            //    fused launch changes itself aside): tiles may be requested before the
                            //    wait for the previous kernel of the stream

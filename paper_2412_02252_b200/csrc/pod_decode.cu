@@ -95,6 +95,18 @@ __device__ __forceinline__ uint64_t policy_evict_first() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
   return p;
 }
+// The stored logits are written by one launch and read by the next: when all of a cache's logit stores are a
+// small part of the L2 (the host decides), they are kept there with evict_last.
+__device__ __forceinline__ uint64_t policy_logits(bool keep) {
+  uint64_t p;
+  if (keep) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void st_f32x4_hint(float* a, float4 v, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1,%2,%3,%4}, %5;"
+               ::"l"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
@@ -102,6 +114,11 @@ __device__ __forceinline__ void fence_async_global() { asm volatile("fence.proxy
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
                : "memory");
 }
 // Launch trace (pod_cache_set_trace): the first CTA to start and the last to finish leave the
@@ -207,7 +224,8 @@ struct Cfg {
 // Everything a warp needs to request a tile; filled once per warp.
 struct TileSource {
   const CUtensorMap* tmap;
-  uint64_t policy;
+  uint64_t policy;                  // of the cache rows
+  uint64_t sc_policy;               // of the stored logits
   unsigned char* sc_base;           // the head's stored logits
   uint32_t bar0, ring, sc0;         // shared-memory addresses: first stage barrier, first stage, first logit slot
   int32_t ntp, rowKp, rowVp, rowKd, rowVd, sc_group_b;
@@ -228,7 +246,8 @@ __device__ __noinline__ void issue_tile(const TileSource t, int vt, int stage, i
     const int yv0 = t.rowVd + ((vt - t.ntp) << t.dt_shift) + dep;
     if (part != 2) mbar_expect_tx(bar, C::STAGE_B + 2 * t.sc_group_b);
     if (part != 1)
-      bulk_load(t.sc0 + stage * C::SC_SLOT_B, t.sc_base + (int64_t)(vt - t.ntp) * 2 * t.sc_group_b, 2 * t.sc_group_b, bar);
+      bulk_load_hint(t.sc0 + stage * C::SC_SLOT_B, t.sc_base + (int64_t)(vt - t.ntp) * 2 * t.sc_group_b, 2 * t.sc_group_b, bar,
+                     t.sc_policy);
     if (part == 2) return;
 #pragma unroll
     for (int s = 0; s < C::NSUB; ++s) {
@@ -337,6 +356,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
   int64_t cap_d = p.v_cap_d[bv];
   int64_t seq_row = p.v_row_base[bv];
   const uint64_t pol_stream = policy_evict_first();
+  const uint64_t pol_logits = policy_logits(p.keep_logits != 0);
 
   // The wait for the previous kernel of the stream comes before anything that kernel may have
   // written is read: stash, counters, logits, the new token.  The cache rows and this layer's
@@ -494,7 +514,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
     return (int)vt;
   };
   TileSource src;
-  src.tmap = &tmap; src.policy = pol_stream; src.sc_base = sc_base; src.bar0 = bar0; src.ring = wbuf_s; src.sc0 = sc0;
+  src.tmap = &tmap; src.policy = pol_stream; src.sc_policy = pol_logits; src.sc_base = sc_base; src.bar0 = bar0; src.ring = wbuf_s; src.sc0 = sc0;
   src.ntp = ntp; src.rowKp = rowKp; src.rowVp = rowVp; src.rowKd = rowKd; src.rowVd = rowVd; src.sc_group_b = sc_group_b;
   src.dt_shift = DT_SH; src.from_scores = sc_read ? 1 : 0;
   auto issue = [&](int vt, int stage, int dep, int part) { issue_tile<D>(src, vt, stage, dep, part); };
@@ -792,7 +812,7 @@ pod_decode_splitk_kernel(const __grid_constant__ CUtensorMap tmap, const DecodeP
         float a11 = (qcol + 9 < cnt && qcol + 9 != mcol) ? l11 : -INFINITY;
         if (store != nullptr) {                        // the other layers of the block reuse these logits
           if (mcol < 0) {
-            *reinterpret_cast<float4*>(store) = make_float4(a00, a01, a10, a11);
+            st_f32x4_hint(store, make_float4(a00, a01, a10, a11), pol_logits);
           } else {                                     // the displaced token's column is written by warp 0
             if (qcol != mcol) store[0] = a00;
             if (qcol + 1 != mcol) store[1] = a01;

@@ -137,7 +137,7 @@ extern "C" int pod_dense_decode_attn_static(const void* kv_device, int capacity,
   p.static_eighths = 5;
   p.scale_log2 = (sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim)) * 1.4426950408889634f;
   for (int w = 0; w < 8; ++w) p.score_read_mask[w] = 0u;
-  p.early_ok = 0; p.optimistic = 0; p.closer = 0; p.seq = 0; p.force_redo = 0;
+  p.early_ok = 0; p.optimistic = 0; p.closer = 0; p.seq = 0; p.force_redo = 0; p.keep_logits = 0;
   p.segment = 0; p.gate_tau = 2.f; p.dlse = nullptr; p.state_acc = nullptr; p.state_ml = nullptr;
   p.by_value = 1;
   p.v_len[0] = n_tokens; p.v_cap_d[0] = 0; p.v_row_base[0] = 0;
