@@ -519,6 +519,10 @@ def run_ours(args):
         if rank == 0:
             print(json.dumps({"prefill_attn": time_prefill_attn(B, synth, w, seed, dev, stream, args)}), flush=True)
         return
+    if args.only == "prefill-write":
+        if rank == 0:
+            print(json.dumps({"prefill_write": time_prefill_write(B, synth, w, seed, dev, local, stream)}), flush=True)
+        return
     if args.only == "decode-steps":
         # warm-up and one region of the headline steps, nothing else: the command profilers are pointed at
         run = Runner(args.workload, w, B=B, synth=synth, dev=dev, local=local, seed=seed, dist=dist, heads=heads,
@@ -889,7 +893,7 @@ def main():
     ap.add_argument("--prefill-sustained-calls", type=int, default=150,
                     help="back-to-back calls of the prefill-attention leg's sustained figure (0 = skip it)")
     ap.add_argument("--no-idle", action="store_true", help="prefill-attention leg: do not idle before the timed calls")
-    ap.add_argument("--only", default=None, choices=["prefill-attn", "decode-steps"],
+    ap.add_argument("--only", default=None, choices=["prefill-attn", "prefill-write", "decode-steps"],
                     help="run one side leg alone and print its object (for profiling)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
