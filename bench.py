@@ -173,6 +173,21 @@ def reduce_max(x, dist, device):
     return float(t.item())
 
 
+def gather_outputs(dist, local, gathered):
+    """KV-head split, for a consumer that wants every head on every rank: one all-gather of the ranks'
+    output slices.  local: this rank's [B][H_q / P][d]; gathered: [P][B][H_q / P][d], slice r = rank r's heads
+    (query heads r * H_q / P onwards).  8 KiB per sequence and layer at the 8B shapes."""
+    # as bytes (every backend moves uint8), the ranks' slices one after the other along the first dimension
+    dist.all_gather_into_tensor(gathered.view(torch.uint8).flatten(0, 1), local.view(torch.uint8))
+    return gathered
+
+
+def heads_from_gathered(gathered):
+    """[P][B][H_q / P][d] as gather_outputs leaves it -> [B][H_q][d] in the order of the unsplit call."""
+    P, Bn, Hl, d = gathered.shape
+    return gathered.permute(1, 0, 2, 3).reshape(Bn, P * Hl, d)
+
+
 def aggregate(*, ms, steps, layers, batch_per_rank, world, shard="sequence"):
     """Whole-job figures from the slowest rank's time for `steps` steps.  Ranks that hold their own
     sequences (shard = "sequence") multiply the work: the job's time per layer-step is the rank's divided
@@ -260,6 +275,7 @@ class Runner:
         self.n_in = n_in
         self.reserve = reserve_steps
         self.stream = torch.cuda.current_stream().cuda_stream
+        self.gathered = None                                    # [L][P][B][H_q / P][d] when the ranks' outputs are gathered
         self.launches = 0
         self.cache = None
         self.step_no = 0
@@ -329,6 +345,8 @@ class Runner:
         elif events is None:
             for l in range(self.L):
                 c.append_decode_attn(l, kpi[l], vpi[l], qpi[l], op[l], st)
+                if self.gathered is not None:       # every rank gets every head of this layer's output
+                    gather_outputs(self.dist, self.outs[l], self.gathered[l])
             self.launches += self.L
         else:                                       # an event pair around every launch: the launches are serialised
             for l in range(self.L):
@@ -545,6 +563,10 @@ def run_ours(args):
     run = Runner(args.workload, w, B=B, synth=synth, dev=dev, local=local, seed=seed, dist=dist, heads=heads, reserve_steps=reserve)
     if args.gate_tau is not None:
         raise SystemExit("bench.py: --gate-tau is timed by tests and DESIGN.md's table, not by this line")
+    if args.gather_outputs:
+        if not (world > 1 and args.shard == "kv-head"):
+            raise SystemExit("bench.py: --gather-outputs goes with --shard kv-head on more than one GPU")
+        run.gathered = torch.empty(L, world, run.Bn, run.Hq, d, dtype=torch.bfloat16, device=dev)
     res, ms, n_launch = measure(run, args, steps=steps, warmup=args.warmup, regions=regions, primary=True, hbm_peak=hbm_peak,
                                 clocks_index=local if rank == 0 else None, dist_world=world)
 
@@ -634,6 +656,7 @@ def run_ours(args):
                    "blocks": ("head-wise, seeded" if "head_wise_new_block_p" in w else "runs of %d layers" % w["G"]) +
                              ": %d of %d (layer, KV head) pairs keep their own distant keys" % (n_low_pairs, L * Hkv),
                    "shard": args.shard if world > 1 else None,
+                   "gather_outputs": bool(args.gather_outputs),
                    "split_tokens": res["split_tokens"], "ctas": res["ctas"],
                    "timing": "value = median of %d regions of %d steps, each bracketed by barrier + synchronize" % (regions, steps)},
         "per_rank_us_per_layer_step": round(agg["per_rank_us_per_layer_step"], 3),
@@ -881,6 +904,9 @@ def main():
     ap.add_argument("--workload", default="llama3-8b-32k", choices=sorted(WORKLOADS))
     ap.add_argument("--shard", default="sequence", choices=["sequence", "kv-head"],
                     help="with several GPUs: independent sequences per rank, or H_kv / N KV heads of the same sequences per rank")
+    ap.add_argument("--gather-outputs", action="store_true",
+                    help="with --shard kv-head: all-gather every layer's output slices (NCCL) inside the timed steps, "
+                         "for a consumer that needs all heads on every rank; default: outputs stay sharded")
     ap.add_argument("--one-shard-of", type=int, default=1,
                     help="on one GPU: run rank 0's share of a KV-head split over this many ranks (what one rank's launches cost)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")

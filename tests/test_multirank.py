@@ -74,10 +74,16 @@ def _worker(rank, world, port, ret):
         ksum = torch.tensor([float(k.float().sum())], dtype=torch.float64)
         ksums = [torch.zeros(1, dtype=torch.float64) for _ in range(world)]
         dist.all_gather(ksums, ksum)
+        # outputs of a KV-head split, gathered: rank r's slice holds query heads r * H_q / P onwards
+        Bn, Hl, d = FULL["batch"], local.n_q_heads, FULL["head_dim"]
+        whole_out = torch.arange(Bn * FULL["n_q_heads"] * d, dtype=torch.float32).reshape(Bn, FULL["n_q_heads"], d).to(torch.bfloat16)
+        mine = whole_out[:, q0:q0 + Hl].contiguous()
+        got = bench.heads_from_gathered(bench.gather_outputs(dist, mine, torch.empty(world, Bn, Hl, d, dtype=torch.bfloat16)))
+        gather_ok = bool(torch.equal(got, whole_out))
         # timing: the slowest rank counts
         t = bench.reduce_max(10.0 + rank, dist, torch.device("cpu"))
         ret[rank] = dict(gathered=[g.tolist() for g in gathered], order=order, cols=cols, hw_live=int(hw_live.item()),
-                         seed=seed, ksums=[float(x) for x in ksums], t=t)
+                         seed=seed, ksums=[float(x) for x in ksums], t=t, gather_ok=gather_ok)
     finally:
         dist.destroy_process_group()
 
@@ -109,6 +115,7 @@ def test_two_ranks_split_by_kv_head_and_by_sequence():
     # by sequence
     assert r0["seed"] != r1["seed"] and r0["ksums"] == r1["ksums"] and r0["ksums"][0] != r0["ksums"][1]
     assert r0["t"] == r1["t"] == 11.0                            # max over ranks on every rank
+    assert r0["gather_ok"] and r1["gather_ok"]                   # gathered slices give the unsplit [B][H_q][d]
 
 
 def test_shard_config_rejects_what_does_not_divide():
