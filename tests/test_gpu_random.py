@@ -106,3 +106,49 @@ def test_random_configuration_decodes_like_the_oracle(seed):
     assert checked == len(CHECK_STEPS) * case.L * case.B * case.Hq
     assert cache.device_status() == B.POD_OK
     cache.destroy()
+
+
+def draw_prefill(seed):
+    rng = random.Random(7000 + seed)
+    d = rng.choice([64, 128])
+    Hkv = rng.choice([1, 2, 3])
+    r = rng.choice([1, 2, 4])
+    T = rng.choice([rng.randint(1, 40), rng.randint(100, 300), rng.randint(250, 530), rng.randint(600, 1300)])
+    S = rng.choice([0, 1, 4, 16, 130, 260])
+    W = rng.choice([1, 31, 64, 127, 128, 300, 2000])
+    sharing = rng.random() < 0.7
+    shares = None
+    if sharing and rng.random() < 0.5:
+        shares = [rng.randint(0, 1) for _ in range(Hkv)]
+    scale = rng.choice([0.0, 0.0, 0.1])
+    return dict(d=d, Hkv=Hkv, Hq=Hkv * r, T=T, S=S, W=W, sharing=sharing, shares=shares, scale=scale,
+                outliers=rng.random() < 0.5)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_configuration_prefill_like_the_oracle(seed):
+    """pod_prefill_attn on drawn lengths (ragged query blocks and key tiles), sinks longer than a tile, windows
+    shorter and longer than the sequence, plain and sharing layers, some heads sharing and some not: every
+    position, head and channel against the oracle's prefill form."""
+    c = draw_prefill(seed)
+    d, Hq, Hkv, T, S, W = c["d"], c["Hq"], c["Hkv"], c["T"], c["S"], c["W"]
+    gen = lambda tag, layer, h: synth.gen_kv(900 + seed, tag, layer, 0, 0, T, h, d,
+                                             outliers=c["outliers"] and tag != synth.TAG_Q, device="cuda")
+    Q = [gen(synth.TAG_Q, l, Hq) for l in range(2)]
+    K = [gen(synth.TAG_K, l, Hkv) for l in range(2)]
+    V = [gen(synth.TAG_V, l, Hkv) for l in range(2)]
+    out = torch.zeros(T, Hq, d, dtype=torch.bfloat16, device="cuda")
+    kw = dict(q_low=Q[0], k_low=K[0], head_shares=c["shares"]) if c["sharing"] else {}
+    B.pod_prefill_attn(Q[1], K[1], V[1], out, n_sink=S, n_recent=W, sm_scale=c["scale"], **kw)
+    torch.cuda.synchronize()
+    assert B.pod_prefill_status() == B.POD_OK
+    f = lambda xs: np.stack([x.double().cpu().numpy() for x in xs])
+    takes_low = lambda h: c["sharing"] and (c["shares"] is None or c["shares"][h])
+    low = np.array([[0] * Hkv, [0 if takes_low(h) else 1 for h in range(Hkv)]])
+    ref = O.pod_prefill_layer(f(Q), f(K), f(V), 1, lowest=low, n_s=S, n_r=W, scale=(c["scale"] if c["scale"] > 0 else None))
+    got = out.double().cpu().numpy()
+    err = np.abs(got - ref)
+    rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    vmax = V[1].double().abs().amax(dim=0).cpu().numpy()                     # [H_kv][d]
+    bound = MAX_ABS + 2.0 ** -8 * np.repeat(vmax, Hq // Hkv, axis=0)[None]   # the prefill tests' bound
+    assert (err <= bound).all() and rel <= REL_L2, f"{c}: max_abs={err.max():.3e} rel_l2={rel:.3e}"
