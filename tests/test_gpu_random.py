@@ -1,6 +1,7 @@
 """Seeded random configurations of the decode path against the oracle: shapes, block maps, window sizes, batch
 mixes, prefill chunkings and call forms drawn together, so that combinations no hand-written case lists are met.
-Every (sequence, layer, query head) of the checked steps is compared element by element."""
+Every (sequence, layer, query head) of the checked steps is compared element by element, and the cache contents
+bit for bit with the oracle's layout after the prefill and after the last step."""
 from __future__ import annotations
 
 import random
@@ -13,6 +14,7 @@ from oracle import pod_oracle as O
 from paper_2412_02252_b200 import binding as B
 from paper_2412_02252_b200 import synth
 from podtest import MAX_ABS, REL_L2, Case
+from test_gpu_parity import _compare_layout, _oracle_cache
 
 pytestmark = pytest.mark.gpu
 
@@ -82,6 +84,14 @@ def test_random_configuration_decodes_like_the_oracle(seed):
     cache = case.make_cache()
     case.prefill(cache, chunk=chunk)
     stream = torch.cuda.current_stream().cuda_stream
+    # the oracle's layout of every sequence, kept up by plain writes and appends
+    ocs = [_oracle_cache(case, b) for b in range(case.B)]
+    for b, oc in enumerate(ocs):
+        for l in range(case.L):
+            if case.lens[b]:
+                oc.write(l, synth.bf16_bits(case.kv(synth.TAG_K, l, b, 0, case.lens[b], "cpu")),
+                         synth.bf16_bits(case.kv(synth.TAG_V, l, b, 0, case.lens[b], "cpu")))
+    _compare_layout(case, cache, ocs)
     checked = 0
     for step in range(1, N_STEPS + 1):
         lens = [n + step for n in case.lens]
@@ -95,6 +105,9 @@ def test_random_configuration_decodes_like_the_oracle(seed):
             else:
                 cache.write(l, -1, k, v, 1, stream)
                 cache.decode_attn(l, q, outs[l], stream)
+            kb, vb = synth.bf16_bits(k), synth.bf16_bits(v)
+            for b, oc in enumerate(ocs):
+                oc.append(l, kb[b], vb[b])
         torch.cuda.synchronize()
         assert [cache.seq_len(b, case.L - 1) for b in range(case.B)] == lens
         if step in CHECK_STEPS:
@@ -103,6 +116,7 @@ def test_random_configuration_decodes_like_the_oracle(seed):
                 for b in range(case.B):
                     for kvh in range(case.Hkv):
                         checked += check_group(case, host, l, b, kvh, lens[b], step)
+    _compare_layout(case, cache, ocs)                          # bit for bit after the appends of both call forms
     assert checked == len(CHECK_STEPS) * case.L * case.B * case.Hq
     assert cache.device_status() == B.POD_OK
     cache.destroy()
